@@ -1,0 +1,186 @@
+/*
+ * vcas.h -- C ABI of libvcas: the variance-controlled sampled backward of one linear layer
+ * (VCAS, "Efficient Backpropagation with Variance-Controlled Adaptive Sampling",
+ * arXiv 2402.17227) as CUDA kernels for sm_100a.
+ *
+ * Notation (paper, Sec. 4): a batch has N data of T tokens, R = N*T rows.  The layer is
+ * Z = X theta^T, so W = theta is [d_out, d_in]; X is [R, d_in]; G = dY is [R, d_out].
+ * rho is the keep ratio of SampleA (data dimension), nu the keep ratio of SampleW (token
+ * dimension).
+ *
+ * Conventions for every entry point
+ *  - returns VCAS_OK (0) or a negative vcas_status; never throws, aborts or prints;
+ *  - tensor arguments are DEVICE pointers owned by the caller, row-major, contiguous,
+ *    16-byte aligned, of the dtype given at vcas_create unless stated otherwise;
+ *  - "host" in an argument comment means a host pointer;
+ *  - work is enqueued on the caller's stream and is asynchronous; no entry point except
+ *    vcas_create, vcas_destroy and vcas_last_device_status synchronises or allocates;
+ *  - a handle owns one workspace and must not be used from two streams at the same time;
+ *  - device-side failures (a bounded wait that ran out) are recorded in a status word that
+ *    vcas_last_device_status reads back.
+ *
+ * Random numbers: Philox4x32-10 (Salmon et al., SC'11) with key = (seed low, seed high),
+ * counter = (index low, index high, sampler id, 0); the top 24 bits u of output word 0
+ * decide "keep" iff u < floor(p * 2^24) with p in float32.  Sampler id 0 = SampleA (index =
+ * datum), 1 = SampleW (index = global row).
+ */
+#ifndef VCAS_H_
+#define VCAS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct vcas_handle_s* vcas_handle;
+typedef void* vcas_stream;            /* a cudaStream_t */
+
+typedef enum {
+  VCAS_OK = 0,
+  VCAS_ERR_BAD_ARG = -1,              /* null pointer, ratio outside (0, 1], M < 2, ... */
+  VCAS_ERR_SHAPE = -2,                /* unsupported sizes */
+  VCAS_ERR_DTYPE = -3,
+  VCAS_ERR_WORKSPACE = -4,            /* workspace allocation failed at vcas_create */
+  VCAS_ERR_CUDA = -5,                 /* a CUDA runtime or driver call failed */
+  VCAS_ERR_TIMEOUT = -6,              /* a device-side bounded wait ran out */
+  VCAS_ERR_INTERNAL = -7
+} vcas_status;
+
+typedef enum { VCAS_DTYPE_F32 = 0, VCAS_DTYPE_BF16 = 1 } vcas_dtype;
+
+/* Which kernels compute the two products.  AUTO picks the tensor-core (tcgen05) kernels for
+ * bf16 layers whose d_in and d_out are multiples of 64, the fp32-FMA kernels otherwise. */
+typedef enum { VCAS_GEMM_AUTO = 0, VCAS_GEMM_FMA = 1, VCAS_GEMM_TENSOR = 2 } vcas_gemm_path;
+
+typedef struct {
+  int32_t N, T, d_in, d_out;          /* d_in and d_out must be multiples of 8 */
+  int32_t dtype;                      /* vcas_dtype of X, dY, W and dX; dW is always fp32 */
+  int32_t gemm_path;                  /* vcas_gemm_path */
+} vcas_layer_desc;
+
+/* Hyper-parameters of Alg. 1.  Defaults (Sec. 6.1): tau_act = tau_w = 0.025, alpha = 0.01,
+ * beta = 0.95, M = 2; F is task dependent (App. A.3), default 100.  rho_min / nu_min are
+ * lower clips applied by vcas_update_ratios (default 0). */
+typedef struct {
+  int32_t F, M;
+  float tau_act, tau_w, alpha, beta;
+  float rho_min, nu_min;
+} vcas_config;
+
+/* Adaptation state of Alg. 1 for a stack of L layers (index 0 = the lowest layer).
+ * rho and nu are host arrays of length L owned by the caller.  Initial values: s = 1,
+ * rho = nu = 1, t = 0. */
+typedef struct {
+  float s;
+  int32_t t;
+  int32_t L;
+  float* rho;                         /* host [L] */
+  float* nu;                          /* host [L] */
+} vcas_state;
+
+/* Fills *cfg with the defaults above (host). */
+int vcas_default_config(vcas_config* cfg);
+
+/* Creates a handle for one layer shape on the current device and allocates its workspace
+ * (the only allocation the library makes).  cfg may be NULL (defaults).  Synchronous. */
+int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config* cfg);
+int vcas_destroy(vcas_handle h);
+/* Bytes of device workspace owned by the handle (host out). */
+int vcas_workspace_bytes(vcas_handle h, size_t* bytes);
+
+/*
+ * Eq. 2 for a linear layer (Sec. 4.1, 4.2, App. E):
+ *   G_hat   = SampleA(dY): data n kept with probability p_n ~ ||G_n||_F, sum p = N rho,
+ *             kept data rescaled by 1/p_n;
+ *   dX      = G_hat W                      [R, d_in], layer dtype, rows of dropped data = 0;
+ *   G_tilde = SampleW(G_hat, X): row r kept with probability q_r ~ ||G_hat_r|| ||X_r||,
+ *             sum q = nu * T * (#kept data), kept rows rescaled by 1/q_r;
+ *   dW      = G_tilde^T X                  [d_out, d_in], fp32.
+ * rho, nu in (0, 1].  With rho = nu = 1 this is exact backprop.
+ */
+int vcas_linear_bwd(vcas_handle h, const void* X, const void* dY, const void* W,
+                    float rho, float nu, uint64_t seed, void* dX, float* dW, vcas_stream stream);
+
+/* vcas_linear_bwd with optional extras, each may be NULL:
+ *   p_in [N], q_in [R] fp32: use these keep probabilities instead of computing them (q_in is
+ *   read only on rows of kept data; rows of dropped data get q = 0);
+ *   H [R, d_in], layer dtype: pre-activation of a GELU feeding this layer's input; dX is
+ *   then multiplied elementwise by GELU'(H) (App. E: non-linear layers multiply by the saved
+ *   Jacobian), erf form of GELU. */
+int vcas_linear_bwd_ex(vcas_handle h, const void* X, const void* dY, const void* W,
+                       float rho, float nu, uint64_t seed,
+                       const float* p_in, const float* q_in, const void* H,
+                       void* dX, float* dW, vcas_stream stream);
+
+/* Exact backprop dX = dY W, dW = dY^T X with the same kernels at ratio 1 and no scoring. */
+int vcas_dense_bwd(vcas_handle h, const void* X, const void* dY, const void* W,
+                   void* dX, float* dW, vcas_stream stream);
+
+/*
+ * Scores, keep probabilities, masks and compacted index lists only (Sec. 4.1, 4.2), exactly
+ * as vcas_linear_bwd computes them.  Every output may be NULL.
+ *   g [N]: ||G_n||_F;  p [N];  w [R]: ||G_hat_r|| ||X_r|| (0 on rows of dropped data);
+ *   q [R];  idxA [N]: ascending indices of kept data, cntA [1] their number;
+ *   idxW [R]: ascending global row indices kept by both samplers, cntW [1] their number.
+ */
+int vcas_score(vcas_handle h, const void* X, const void* dY, float rho, float nu, uint64_t seed,
+               float* g, float* p, float* w, float* q,
+               int32_t* idxA, int32_t* cntA, int32_t* idxW, int32_t* cntW, vcas_stream stream);
+
+/* Copies what the last vcas_linear_bwd(_ex) or vcas_score on this handle computed (same
+ * outputs as vcas_score); enqueue on the same stream. */
+int vcas_last_sampling(vcas_handle h, float* g, float* p, float* w, float* q,
+                       int32_t* idxA, int32_t* cntA, int32_t* idxW, int32_t* cntW,
+                       vcas_stream stream);
+
+/* Bernoulli mask and compaction for given probabilities (Sec. 4.1: m_i = Bern(p_i)/p_i):
+ * keep[i] = (u24(seed, sampler_id, i) < floor(p[i] 2^24)) for i < n; idx = ascending kept
+ * indices, cnt [1] their number.  keep (uint8 [n]), idx (int32 [n]) may be NULL. */
+int vcas_mask_from_probs(vcas_handle h, const float* p, int32_t n, uint64_t seed, int32_t sampler_id,
+                         uint8_t* keep, int32_t* idx, int32_t* cnt, vcas_stream stream);
+
+/*
+ * The Monte-Carlo probe of Alg. 1 at the granularity of this layer's parameter gradient.
+ * X_i, dY_i: host arrays of M device pointers (M batches); W as above.
+ * For batch i: G_s,i = dY_i^T X_i (exact).  For repetition j (seed derived from (seed, i, j)):
+ * G_act,ij = G_hat_ij^T X_i with SampleA only, and V_w,ij = Eq. 3 at ratio nu.
+ * Outputs (device fp32 scalars, any may be NULL):
+ *   V_s   = 1/(M-1) sum_i ||G_s,i - mean||_F^2,
+ *   V_act = 1/M^2 sum_ij ||G_act,ij - G_s,i||_F^2,
+ *   V_w   = 1/M^2 sum_ij V_w,ij,
+ *   p_lo, p_hi = Eq. 4's sparsity p(s - alpha), p(s + alpha) averaged over the batches
+ *   (App. D), s -+ alpha clipped to [0, 1].
+ * M >= 2 (the 1/(M-1) of V_s).  alpha comes from the handle's config.
+ */
+int vcas_variance_probe(vcas_handle h, int32_t M, const void* const* X_i, const void* const* dY_i,
+                        const void* W, float rho, float nu, float s, uint64_t seed,
+                        float* V_s, float* V_act, float* V_w, float* p_lo, float* p_hi,
+                        vcas_stream stream);
+
+/*
+ * One adaptation step of Alg. 1 (host only, all pointers host, arrays of length L):
+ *   Eq. 5: s <- clip(s + alpha sign(sum_l V_act,l - tau_act sum_l V_s,l), 0, 1), sign(0) = +1;
+ *   Eq. 4: rho_l <- max(rho_min, max_{j<=l} p_j) with p_j = p_hi[j] if s went up else p_lo[j];
+ *   Eq. 7: nu_l <- min(1, nu_l / beta) if V_w,l >= tau_w V_s,l else max(nu_min, nu_l beta).
+ * state->t is left to the training loop.
+ */
+int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const float* V_act,
+                       const float* V_w, const float* p_lo, const float* p_hi,
+                       const vcas_config* cfg);
+
+/* Synchronises the device and returns the handle's device status word in *status
+ * (VCAS_OK or VCAS_ERR_TIMEOUT / VCAS_ERR_INTERNAL); the word is then cleared. */
+int vcas_last_device_status(vcas_handle h, int32_t* status);
+
+/* Number of this library's kernel launches enqueued through the handle so far (host out). */
+int vcas_launch_count(vcas_handle h, uint64_t* launches);
+
+/* Library version, e.g. 100 for 0.1.0. */
+int vcas_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VCAS_H_ */

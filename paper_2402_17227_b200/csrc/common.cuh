@@ -1,0 +1,137 @@
+// Internal declarations shared by the kernels of libvcas (device helpers, workspace layout).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vcas.h"
+
+namespace vcas {
+
+// ---------------------------------------------------------------------------------------
+// Workspace: one allocation per handle, carved into these arrays at vcas_create.
+// ---------------------------------------------------------------------------------------
+struct Workspace {
+  // scores (Sec. 4.1, 4.2)
+  float* a;        // [R]  ||dY_r||^2
+  float* b;        // [R]  ||X_r||^2
+  float* g;        // [N]  ||G_n||_F
+  float* p;        // [N]  SampleA keep probabilities
+  float* w;        // [R]  leverage scores of G_hat
+  float* q;        // [R]  SampleW keep probabilities
+  float* scaleA;   // [N]  1/p_n for kept data, 0 for dropped data
+  float* scaleW;   // [R]  1/(p_n q_r) per compacted row
+  float* sorted;   // [N]  data norms in descending order (Eq. 4)
+  int32_t* idxA;   // [N]  kept data, ascending
+  int32_t* dropA;  // [N]  dropped data, ascending
+  int32_t* idxW;   // [R]  kept rows, ascending
+  int32_t* counts; // [8]  0: cntA, 1: cntW, 2: R (constant, for dense launches), 4: reduction ticket
+  int32_t* status; // [1]  device status word
+  double* acc;     // [16] probe accumulators (0: V_act, 1: V_w, 2: p_lo, 3: p_hi, 4: V_s)
+  double* partial; // [PARTIAL_SLOTS] block partial sums of the probe reductions
+  // compact operands of the weight-gradient product (tensor path)
+  __nv_bfloat16* packG;  // [R_pad, d_out]
+  __nv_bfloat16* packX;  // [R_pad, d_in]
+  // probe buffers (App. D: the exact gradient, its running mean and running squared deviation)
+  float* Gs;       // [d_out, d_in]
+  float* Gact;     // [d_out, d_in]
+  float* mean;     // [d_out, d_in]
+  float* m2;       // [d_out, d_in]
+};
+
+constexpr int PARTIAL_SLOTS = 4096;
+
+struct Handle {
+  vcas_layer_desc desc;
+  vcas_config cfg;
+  int device;
+  int num_sms;
+  bool tensor_path;
+  int R_pad;
+  void* base;
+  size_t bytes;
+  Workspace ws;
+  uint64_t launches;
+};
+
+// ---------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t philox_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
+
+// keep iff the 24-bit uniform of (seed, sampler, idx) is below floor(p * 2^24)
+__device__ __forceinline__ bool bernoulli_keep(float p, uint64_t seed, uint32_t sampler, uint64_t idx) {
+  const uint32_t u = philox_word0((uint32_t)idx, (uint32_t)(idx >> 32), sampler, 0u,
+                                  (uint32_t)seed, (uint32_t)(seed >> 32)) >> 8;
+  const uint32_t thr = (uint32_t)floorf(p * 16777216.0f);
+  return u < thr;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ---------------------------------------------------------------------------------------
+// Launchers (one per .cu file).  All enqueue on `st` and return a cudaError_t.
+// ---------------------------------------------------------------------------------------
+cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, cudaStream_t st);
+
+struct SamplerArgs {
+  float rho, nu;
+  uint64_t seed;
+  const float* p_in;
+  const float* q_in;
+  int sample_w;      // 1: SampleW mask applied; 0: all rows of kept data survive (probe)
+  int accumulate_vw; // 1: add Eq. 3 at ratio nu to acc[1]
+};
+cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st);
+cudaError_t launch_mask_from_probs(Handle* h, const float* p, int n, uint64_t seed, int sampler,
+                                   uint8_t* keep, int32_t* idx, int32_t* cnt, cudaStream_t st);
+
+// fp32-FMA products
+cudaError_t launch_fma_dx(Handle* h, const void* dY, const void* W, const float* scaleA,
+                          const void* H, void* dX, cudaStream_t st);
+cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_t* idx,
+                          const float* scale, const int32_t* cnt, float* dW, cudaStream_t st);
+
+// tensor-core products
+cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
+                           const void* H, void* dX, cudaStream_t st);
+cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
+// dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
+cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity,
+                           const int32_t* cnt, float* dW, cudaStream_t st);
+
+// probe reductions
+cudaError_t launch_probe_reset(Handle* h, cudaStream_t st);
+cudaError_t launch_probe_welford(Handle* h, int i, cudaStream_t st);
+cudaError_t launch_probe_sqdiff(Handle* h, cudaStream_t st);
+cudaError_t launch_probe_sparsity(Handle* h, double s_lo, double s_hi, cudaStream_t st);
+cudaError_t launch_probe_finalize(Handle* h, int M, float* V_s, float* V_act, float* V_w,
+                                  float* p_lo, float* p_hi, cudaStream_t st);
+
+}  // namespace vcas
