@@ -1,0 +1,328 @@
+// C ABI of libvcas (see vcas.h): argument checks, workspace, and the order in which the
+// kernels of Eq. 2 and Alg. 1 are enqueued.  No arithmetic of the method happens on the host
+// except vcas_update_ratios, which the paper defines on a handful of scalars.
+#include <new>
+
+#include "common.cuh"
+
+using namespace vcas;
+
+namespace {
+
+inline Handle* H(vcas_handle h) { return reinterpret_cast<Handle*>(h); }
+inline cudaStream_t S(vcas_stream s) { return reinterpret_cast<cudaStream_t>(s); }
+
+size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+template <typename T>
+T* carve(uint8_t*& cur, size_t count) {
+  T* p = reinterpret_cast<T*>(cur);
+  cur += align_up(count * sizeof(T));
+  return p;
+}
+
+bool ratio_ok(float r) { return r > 0.f && r <= 1.f; }
+
+#define VCAS_CUDA(expr)                         \
+  do {                                          \
+    if ((expr) != cudaSuccess) return VCAS_ERR_CUDA; \
+  } while (0)
+
+// Lays the workspace out from `base` (base == nullptr: only measures).
+size_t layout(Handle* h, uint8_t* base) {
+  const vcas_layer_desc& d = h->desc;
+  const size_t N = d.N, R = (size_t)d.N * d.T, DW = (size_t)d.d_out * d.d_in;
+  uint8_t* cur = base;
+  Workspace& w = h->ws;
+  w.a = carve<float>(cur, R);
+  w.b = carve<float>(cur, R);
+  w.g = carve<float>(cur, N);
+  w.p = carve<float>(cur, N);
+  w.w = carve<float>(cur, R);
+  w.q = carve<float>(cur, R);
+  w.scaleA = carve<float>(cur, N);
+  w.scaleW = carve<float>(cur, R);
+  w.sorted = carve<float>(cur, N);
+  w.idxA = carve<int32_t>(cur, N);
+  w.dropA = carve<int32_t>(cur, N);
+  w.idxW = carve<int32_t>(cur, R);
+  w.counts = carve<int32_t>(cur, 8);
+  w.status = carve<int32_t>(cur, 1);
+  w.acc = carve<double>(cur, 16);
+  w.partial = carve<double>(cur, PARTIAL_SLOTS);
+  if (h->tensor_path) {
+    w.packG = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_out);
+    w.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
+  } else {
+    w.packG = nullptr;
+    w.packX = nullptr;
+  }
+  w.Gs = carve<float>(cur, DW);
+  w.Gact = carve<float>(cur, DW);
+  w.mean = carve<float>(cur, DW);
+  w.m2 = carve<float>(cur, DW);
+  return (size_t)(cur - base);
+}
+
+int copy_out(Handle* h, float* g, float* p, float* w, float* q, int32_t* idxA, int32_t* cntA, int32_t* idxW,
+             int32_t* cntW, cudaStream_t st) {
+  const size_t N = h->desc.N, R = (size_t)h->desc.N * h->desc.T;
+  const Workspace& ws = h->ws;
+  const cudaMemcpyKind k = cudaMemcpyDeviceToDevice;
+  if (g) VCAS_CUDA(cudaMemcpyAsync(g, ws.g, N * sizeof(float), k, st));
+  if (p) VCAS_CUDA(cudaMemcpyAsync(p, ws.p, N * sizeof(float), k, st));
+  if (w) VCAS_CUDA(cudaMemcpyAsync(w, ws.w, R * sizeof(float), k, st));
+  if (q) VCAS_CUDA(cudaMemcpyAsync(q, ws.q, R * sizeof(float), k, st));
+  if (idxA) VCAS_CUDA(cudaMemcpyAsync(idxA, ws.idxA, N * sizeof(int32_t), k, st));
+  if (cntA) VCAS_CUDA(cudaMemcpyAsync(cntA, ws.counts + 0, sizeof(int32_t), k, st));
+  if (idxW) VCAS_CUDA(cudaMemcpyAsync(idxW, ws.idxW, R * sizeof(int32_t), k, st));
+  if (cntW) VCAS_CUDA(cudaMemcpyAsync(cntW, ws.counts + 1, sizeof(int32_t), k, st));
+  return VCAS_OK;
+}
+
+// dW over the rows the sampler kept (idxW / scaleW / counts[1]) into `out`
+int sampled_dw(Handle* h, const void* X, const void* dY, float* out, cudaStream_t st) {
+  if (h->tensor_path) {
+    VCAS_CUDA(launch_pack(h, dY, X, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, out, st));
+  } else {
+    VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, out, st));
+  }
+  return VCAS_OK;
+}
+
+int dense_dw(Handle* h, const void* X, const void* dY, float* out, cudaStream_t st) {
+  if (h->tensor_path) {
+    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, out, st));
+  } else {
+    VCAS_CUDA(launch_fma_dw(h, dY, X, nullptr, nullptr, h->ws.counts + 2, out, st));
+  }
+  return VCAS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int vcas_version(void) { return 100; }
+
+int vcas_default_config(vcas_config* cfg) {
+  if (cfg == nullptr) return VCAS_ERR_BAD_ARG;
+  cfg->F = 100;
+  cfg->M = 2;
+  cfg->tau_act = 0.025f;
+  cfg->tau_w = 0.025f;
+  cfg->alpha = 0.01f;
+  cfg->beta = 0.95f;
+  cfg->rho_min = 0.f;
+  cfg->nu_min = 0.f;
+  return VCAS_OK;
+}
+
+int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config* cfg) {
+  if (out == nullptr || desc == nullptr) return VCAS_ERR_BAD_ARG;
+  *out = nullptr;
+  if (desc->N <= 0 || desc->T <= 0 || desc->d_in <= 0 || desc->d_out <= 0) return VCAS_ERR_SHAPE;
+  if ((desc->d_in % 8) != 0 || (desc->d_out % 8) != 0) return VCAS_ERR_SHAPE;
+  if ((long long)desc->N * desc->T > (1ll << 30)) return VCAS_ERR_SHAPE;
+  if (desc->dtype != VCAS_DTYPE_F32 && desc->dtype != VCAS_DTYPE_BF16) return VCAS_ERR_DTYPE;
+  const bool tensor_ok = desc->dtype == VCAS_DTYPE_BF16 && (desc->d_in % 64) == 0 && (desc->d_out % 64) == 0;
+  if (desc->gemm_path == VCAS_GEMM_TENSOR && !tensor_ok) return VCAS_ERR_SHAPE;
+  if (desc->gemm_path < VCAS_GEMM_AUTO || desc->gemm_path > VCAS_GEMM_TENSOR) return VCAS_ERR_BAD_ARG;
+  Handle* h = new (std::nothrow) Handle();
+  if (h == nullptr) return VCAS_ERR_WORKSPACE;
+  h->desc = *desc;
+  if (cfg != nullptr) h->cfg = *cfg; else vcas_default_config(&h->cfg);
+  h->tensor_path = tensor_ok && desc->gemm_path != VCAS_GEMM_FMA;
+  h->R_pad = (desc->N * desc->T + 63) / 64 * 64;
+  h->launches = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&h->device) != cudaSuccess || cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
+    delete h;
+    return VCAS_ERR_CUDA;
+  }
+  h->num_sms = prop.multiProcessorCount;
+  if (h->tensor_path && prop.major != 10) { delete h; return VCAS_ERR_CUDA; }
+  h->bytes = layout(h, nullptr);
+  if (cudaMalloc(&h->base, h->bytes) != cudaSuccess) {
+    cudaGetLastError();
+    delete h;
+    return VCAS_ERR_WORKSPACE;
+  }
+  layout(h, reinterpret_cast<uint8_t*>(h->base));
+  const int32_t R = desc->N * desc->T;
+  if (cudaMemset(h->base, 0, h->bytes) != cudaSuccess ||
+      cudaMemcpy(h->ws.counts + 2, &R, sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaFree(h->base);
+    delete h;
+    return VCAS_ERR_CUDA;
+  }
+  *out = reinterpret_cast<vcas_handle>(h);
+  return VCAS_OK;
+}
+
+int vcas_destroy(vcas_handle hh) {
+  if (hh == nullptr) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  const cudaError_t e = cudaFree(h->base);
+  delete h;
+  return e == cudaSuccess ? VCAS_OK : VCAS_ERR_CUDA;
+}
+
+int vcas_workspace_bytes(vcas_handle hh, size_t* bytes) {
+  if (hh == nullptr || bytes == nullptr) return VCAS_ERR_BAD_ARG;
+  *bytes = H(hh)->bytes;
+  return VCAS_OK;
+}
+
+int vcas_launch_count(vcas_handle hh, uint64_t* launches) {
+  if (hh == nullptr || launches == nullptr) return VCAS_ERR_BAD_ARG;
+  *launches = H(hh)->launches;
+  return VCAS_OK;
+}
+
+int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void* W, float rho, float nu,
+                       uint64_t seed, const float* p_in, const float* q_in, const void* Hpre, void* dX, float* dW,
+                       vcas_stream stream) {
+  if (hh == nullptr || X == nullptr || dY == nullptr || W == nullptr || dX == nullptr || dW == nullptr)
+    return VCAS_ERR_BAD_ARG;
+  if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  cudaStream_t st = S(stream);
+  VCAS_CUDA(launch_rownorms(h, dY, X, st));
+  SamplerArgs a;
+  a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
+  VCAS_CUDA(launch_sampler(h, a, st));
+  if (h->tensor_path) {
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, st));
+  } else {
+    VCAS_CUDA(launch_fma_dx(h, dY, W, h->ws.scaleA, Hpre, dX, st));
+  }
+  return sampled_dw(h, X, dY, dW, st);
+}
+
+int vcas_linear_bwd(vcas_handle hh, const void* X, const void* dY, const void* W, float rho, float nu,
+                    uint64_t seed, void* dX, float* dW, vcas_stream stream) {
+  return vcas_linear_bwd_ex(hh, X, dY, W, rho, nu, seed, nullptr, nullptr, nullptr, dX, dW, stream);
+}
+
+int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W, void* dX, float* dW,
+                   vcas_stream stream) {
+  if (hh == nullptr || X == nullptr || dY == nullptr || W == nullptr || dX == nullptr || dW == nullptr)
+    return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  cudaStream_t st = S(stream);
+  if (h->tensor_path) {
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, st));
+  } else {
+    VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
+  }
+  return dense_dw(h, X, dY, dW, st);
+}
+
+int vcas_score(vcas_handle hh, const void* X, const void* dY, float rho, float nu, uint64_t seed, float* g,
+               float* p, float* w, float* q, int32_t* idxA, int32_t* cntA, int32_t* idxW, int32_t* cntW,
+               vcas_stream stream) {
+  if (hh == nullptr || X == nullptr || dY == nullptr) return VCAS_ERR_BAD_ARG;
+  if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  cudaStream_t st = S(stream);
+  VCAS_CUDA(launch_rownorms(h, dY, X, st));
+  SamplerArgs a;
+  a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 1; a.accumulate_vw = 0;
+  VCAS_CUDA(launch_sampler(h, a, st));
+  return copy_out(h, g, p, w, q, idxA, cntA, idxW, cntW, st);
+}
+
+int vcas_last_sampling(vcas_handle hh, float* g, float* p, float* w, float* q, int32_t* idxA, int32_t* cntA,
+                       int32_t* idxW, int32_t* cntW, vcas_stream stream) {
+  if (hh == nullptr) return VCAS_ERR_BAD_ARG;
+  return copy_out(H(hh), g, p, w, q, idxA, cntA, idxW, cntW, S(stream));
+}
+
+int vcas_mask_from_probs(vcas_handle hh, const float* p, int32_t n, uint64_t seed, int32_t sampler_id,
+                         uint8_t* keep, int32_t* idx, int32_t* cnt, vcas_stream stream) {
+  if (hh == nullptr || p == nullptr || n < 0) return VCAS_ERR_BAD_ARG;
+  if (sampler_id < 0) return VCAS_ERR_BAD_ARG;
+  VCAS_CUDA(launch_mask_from_probs(H(hh), p, n, seed, sampler_id, keep, idx, cnt, S(stream)));
+  return VCAS_OK;
+}
+
+int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const void* const* dY_i, const void* W,
+                        float rho, float nu, float s, uint64_t seed, float* V_s, float* V_act, float* V_w,
+                        float* p_lo, float* p_hi, vcas_stream stream) {
+  if (hh == nullptr || X_i == nullptr || dY_i == nullptr || W == nullptr) return VCAS_ERR_BAD_ARG;
+  if (M < 2 || !ratio_ok(rho) || !ratio_ok(nu) || !(s >= 0.f && s <= 1.f)) return VCAS_ERR_BAD_ARG;
+  for (int i = 0; i < M; ++i)
+    if (X_i[i] == nullptr || dY_i[i] == nullptr) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  cudaStream_t st = S(stream);
+  const double alpha = (double)h->cfg.alpha;
+  double s_lo = (double)s - alpha, s_hi = (double)s + alpha;
+  if (s_lo < 0.0) s_lo = 0.0;
+  if (s_hi > 1.0) s_hi = 1.0;
+  VCAS_CUDA(launch_probe_reset(h, st));
+  for (int i = 0; i < M; ++i) {
+    int rc = dense_dw(h, X_i[i], dY_i[i], h->ws.Gs, st);            // G_s,i
+    if (rc != VCAS_OK) return rc;
+    VCAS_CUDA(launch_probe_welford(h, i, st));
+    VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], st));
+    for (int j = 0; j < M; ++j) {
+      SamplerArgs a;
+      a.rho = rho; a.nu = nu; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 0; a.accumulate_vw = 1;
+      a.seed = seed + (uint64_t)(i * M + j + 1) * 0x9E3779B97F4A7C15ull;
+      VCAS_CUDA(launch_sampler(h, a, st));
+      if (j == 0) VCAS_CUDA(launch_probe_sparsity(h, s_lo, s_hi, st));
+      rc = sampled_dw(h, X_i[i], dY_i[i], h->ws.Gact, st);          // G_act,ij (SampleA only)
+      if (rc != VCAS_OK) return rc;
+      VCAS_CUDA(launch_probe_sqdiff(h, st));
+    }
+  }
+  VCAS_CUDA(launch_probe_finalize(h, M, V_s, V_act, V_w, p_lo, p_hi, st));
+  return VCAS_OK;
+}
+
+int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const float* V_act, const float* V_w,
+                       const float* p_lo, const float* p_hi, const vcas_config* cfg) {
+  if (state == nullptr || cfg == nullptr || V_s == nullptr || V_act == nullptr || V_w == nullptr ||
+      p_lo == nullptr || p_hi == nullptr || state->rho == nullptr || state->nu == nullptr)
+    return VCAS_ERR_BAD_ARG;
+  if (L <= 0 || L != state->L) return VCAS_ERR_BAD_ARG;
+  if (!(cfg->beta > 0.f && cfg->beta < 1.f) || !(cfg->alpha > 0.f)) return VCAS_ERR_BAD_ARG;
+  double sum_act = 0.0, sum_s = 0.0;
+  for (int l = 0; l < L; ++l) { sum_act += (double)V_act[l]; sum_s += (double)V_s[l]; }
+  const bool up = sum_act - (double)cfg->tau_act * sum_s >= 0.0;   // Eq. 5, sign(0) = +1
+  double s = (double)state->s + (up ? (double)cfg->alpha : -(double)cfg->alpha);
+  s = s < 0.0 ? 0.0 : (s > 1.0 ? 1.0 : s);
+  state->s = (float)s;
+  double run = 0.0;                                                  // Eq. 4: running maximum from layer 1 up
+  for (int l = 0; l < L; ++l) {
+    const double cand = (double)(up ? p_hi[l] : p_lo[l]);
+    run = cand > run ? cand : run;
+    const double r = run > (double)cfg->rho_min ? run : (double)cfg->rho_min;
+    state->rho[l] = (float)r;
+  }
+  for (int l = 0; l < L; ++l) {                                      // Eq. 7
+    double nu = (double)state->nu[l];
+    if ((double)V_w[l] - (double)cfg->tau_w * (double)V_s[l] >= 0.0) {
+      nu = nu / (double)cfg->beta;
+      if (nu > 1.0) nu = 1.0;
+    } else {
+      nu = nu * (double)cfg->beta;
+    }
+    if (nu < (double)cfg->nu_min) nu = (double)cfg->nu_min;
+    state->nu[l] = (float)nu;
+  }
+  return VCAS_OK;
+}
+
+int vcas_last_device_status(vcas_handle hh, int32_t* status) {
+  if (hh == nullptr || status == nullptr) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  VCAS_CUDA(cudaDeviceSynchronize());
+  VCAS_CUDA(cudaMemcpy(status, h->ws.status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  VCAS_CUDA(cudaMemset(h->ws.status, 0, sizeof(int32_t)));
+  return VCAS_OK;
+}
+
+}  // extern "C"
