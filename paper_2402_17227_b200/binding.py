@@ -1,0 +1,236 @@
+"""ctypes binding of libvcas.so: one Python function per C entry point of include/vcas.h.
+
+Argument marshalling only: torch tensors provide device memory and the current CUDA stream,
+every step of the method runs in the library's kernels.  If the compiled library is missing
+this module raises on first use; there is no other implementation to fall back to.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvcas.so")
+
+VCAS_OK = 0
+ERRORS = {-1: "VCAS_ERR_BAD_ARG", -2: "VCAS_ERR_SHAPE", -3: "VCAS_ERR_DTYPE", -4: "VCAS_ERR_WORKSPACE",
+          -5: "VCAS_ERR_CUDA", -6: "VCAS_ERR_TIMEOUT", -7: "VCAS_ERR_INTERNAL"}
+DTYPE_F32, DTYPE_BF16 = 0, 1
+GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
+
+EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
+           "vcas_linear_bwd_ex", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
+           "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
+           "vcas_version"]
+
+
+class VcasError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__(f"{where} failed: {ERRORS.get(code, code)}")
+        self.code = code
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("N", C.c_int32), ("T", C.c_int32), ("d_in", C.c_int32), ("d_out", C.c_int32),
+                ("dtype", C.c_int32), ("gemm_path", C.c_int32)]
+
+
+class Config(C.Structure):
+    _fields_ = [("F", C.c_int32), ("M", C.c_int32), ("tau_act", C.c_float), ("tau_w", C.c_float),
+                ("alpha", C.c_float), ("beta", C.c_float), ("rho_min", C.c_float), ("nu_min", C.c_float)]
+
+
+class State(C.Structure):
+    _fields_ = [("s", C.c_float), ("t", C.c_int32), ("L", C.c_int32),
+                ("rho", C.POINTER(C.c_float)), ("nu", C.POINTER(C.c_float))]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libvcas.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with "
+                               "`python -m paper_2402_17227_b200.build` (needs nvcc); "
+                               "there is no CPU implementation")
+        l = C.CDLL(LIB_PATH)
+        for name in EXPORTS:
+            getattr(l, name).restype = C.c_int
+        _lib = l
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != VCAS_OK:
+        raise VcasError(code, where)
+
+
+def _ptr(t):
+    if t is None:
+        return C.c_void_p(None)
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def default_config() -> Config:
+    cfg = Config()
+    _check(lib().vcas_default_config(C.byref(cfg)), "vcas_default_config")
+    return cfg
+
+
+@dataclass
+class Sampling:
+    g: torch.Tensor
+    p: torch.Tensor
+    w: torch.Tensor
+    q: torch.Tensor
+    idxA: torch.Tensor
+    cntA: int
+    idxW: torch.Tensor
+    cntW: int
+
+
+class Layer:
+    """A handle for one layer shape (vcas_create / vcas_destroy) on the current CUDA device."""
+
+    def __init__(self, N: int, T: int, d_in: int, d_out: int, dtype: torch.dtype = torch.bfloat16,
+                 gemm_path: int = GEMM_AUTO, config: Config | None = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libvcas needs a CUDA device (sm_100a); there is no CPU path")
+        self.N, self.T, self.d_in, self.d_out, self.dtype = N, T, d_in, d_out, dtype
+        self.R = N * T
+        self.config = config if config is not None else default_config()
+        desc = LayerDesc(N, T, d_in, d_out, {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[dtype], gemm_path)
+        self._h = C.c_void_p(None)
+        _check(lib().vcas_create(C.byref(self._h), C.byref(desc), C.byref(self.config)), "vcas_create")
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().vcas_destroy(self._h)
+            self._h = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ products
+    def _outs(self, dX, dW, dev):
+        if dX is None:
+            dX = torch.empty(self.R, self.d_in, dtype=self.dtype, device=dev)
+        if dW is None:
+            dW = torch.empty(self.d_out, self.d_in, dtype=torch.float32, device=dev)
+        return dX, dW
+
+    def linear_bwd(self, X, dY, W, rho: float, nu: float, seed: int, *, p_in=None, q_in=None, H=None,
+                   dX=None, dW=None):
+        dX, dW = self._outs(dX, dW, X.device)
+        rc = lib().vcas_linear_bwd_ex(self._h, _ptr(X), _ptr(dY), _ptr(W), C.c_float(rho), C.c_float(nu),
+                                      C.c_uint64(seed), _ptr(p_in), _ptr(q_in), _ptr(H), _ptr(dX), _ptr(dW),
+                                      _stream())
+        _check(rc, "vcas_linear_bwd_ex")
+        return dX, dW
+
+    def linear_bwd_plain(self, X, dY, W, rho: float, nu: float, seed: int, dX, dW):
+        """vcas_linear_bwd with caller-provided outputs (the call a training loop makes)."""
+        _check(lib().vcas_linear_bwd(self._h, _ptr(X), _ptr(dY), _ptr(W), C.c_float(rho), C.c_float(nu),
+                                     C.c_uint64(seed), _ptr(dX), _ptr(dW), _stream()), "vcas_linear_bwd")
+
+    def dense_bwd(self, X, dY, W, *, dX=None, dW=None):
+        dX, dW = self._outs(dX, dW, X.device)
+        _check(lib().vcas_dense_bwd(self._h, _ptr(X), _ptr(dY), _ptr(W), _ptr(dX), _ptr(dW), _stream()),
+               "vcas_dense_bwd")
+        return dX, dW
+
+    # ------------------------------------------------------------------ sampling
+    def _sampling_buffers(self, dev):
+        f = dict(dtype=torch.float32, device=dev)
+        i = dict(dtype=torch.int32, device=dev)
+        return (torch.empty(self.N, **f), torch.empty(self.N, **f), torch.empty(self.R, **f),
+                torch.empty(self.R, **f), torch.empty(self.N, **i), torch.zeros(1, **i),
+                torch.empty(self.R, **i), torch.zeros(1, **i))
+
+    @staticmethod
+    def _pack_sampling(b) -> Sampling:
+        g, p, w, q, idxA, cntA, idxW, cntW = b
+        ca, cw = int(cntA.item()), int(cntW.item())
+        return Sampling(g, p, w, q, idxA[:ca], ca, idxW[:cw], cw)
+
+    def score(self, X, dY, rho: float, nu: float, seed: int) -> Sampling:
+        b = self._sampling_buffers(X.device)
+        _check(lib().vcas_score(self._h, _ptr(X), _ptr(dY), C.c_float(rho), C.c_float(nu), C.c_uint64(seed),
+                                *[_ptr(t) for t in b], _stream()), "vcas_score")
+        return self._pack_sampling(b)
+
+    def last_sampling(self, device=None) -> Sampling:
+        b = self._sampling_buffers(device or torch.device("cuda", torch.cuda.current_device()))
+        _check(lib().vcas_last_sampling(self._h, *[_ptr(t) for t in b], _stream()), "vcas_last_sampling")
+        return self._pack_sampling(b)
+
+    def mask_from_probs(self, p, seed: int, sampler_id: int):
+        n = p.numel()
+        keep = torch.empty(n, dtype=torch.uint8, device=p.device)
+        idx = torch.empty(n, dtype=torch.int32, device=p.device)
+        cnt = torch.zeros(1, dtype=torch.int32, device=p.device)
+        _check(lib().vcas_mask_from_probs(self._h, _ptr(p), C.c_int32(n), C.c_uint64(seed), C.c_int32(sampler_id),
+                                          _ptr(keep), _ptr(idx), _ptr(cnt), _stream()), "vcas_mask_from_probs")
+        c = int(cnt.item())
+        return keep, idx[:c], c
+
+    # --------------------------------------------------------------------- probe
+    def variance_probe(self, Xs, dYs, W, rho: float, nu: float, s: float, seed: int, out=None):
+        """Returns a device tensor [V_s, V_act, V_w, p_lo, p_hi] (fp32), filled asynchronously."""
+        M = len(Xs)
+        if out is None:
+            out = torch.zeros(5, dtype=torch.float32, device=W.device)
+        xa = (C.c_void_p * M)(*[x.data_ptr() for x in Xs])
+        ya = (C.c_void_p * M)(*[y.data_ptr() for y in dYs])
+        base, st = out.data_ptr(), 4
+        rc = lib().vcas_variance_probe(self._h, C.c_int32(M), xa, ya, _ptr(W), C.c_float(rho), C.c_float(nu),
+                                       C.c_float(s), C.c_uint64(seed), *[C.c_void_p(base + st * k) for k in range(5)],
+                                       _stream())
+        _check(rc, "vcas_variance_probe")
+        return out
+
+    # ---------------------------------------------------------------------- misc
+    def device_status(self) -> int:
+        st = C.c_int32(0)
+        _check(lib().vcas_last_device_status(self._h, C.byref(st)), "vcas_last_device_status")
+        return st.value
+
+    def launch_count(self) -> int:
+        n = C.c_uint64(0)
+        _check(lib().vcas_launch_count(self._h, C.byref(n)), "vcas_launch_count")
+        return n.value
+
+    def workspace_bytes(self) -> int:
+        n = C.c_size_t(0)
+        _check(lib().vcas_workspace_bytes(self._h, C.byref(n)), "vcas_workspace_bytes")
+        return n.value
+
+
+def update_ratios(s: float, rho, nu, V_s, V_act, V_w, p_lo, p_hi, config: Config, t: int = 0):
+    """vcas_update_ratios on host lists of length L; returns (s, rho, nu)."""
+    L = len(rho)
+    arr = lambda v: (C.c_float * L)(*[float(x) for x in v])
+    rho_a, nu_a = arr(rho), arr(nu)
+    st = State(float(s), int(t), L, C.cast(rho_a, C.POINTER(C.c_float)), C.cast(nu_a, C.POINTER(C.c_float)))
+    rc = lib().vcas_update_ratios(C.byref(st), C.c_int32(L), arr(V_s), arr(V_act), arr(V_w), arr(p_lo), arr(p_hi),
+                                  C.byref(config))
+    _check(rc, "vcas_update_ratios")
+    return st.s, list(rho_a), list(nu_a)
+
+
+def version() -> int:
+    return lib().vcas_version()
