@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the sampled linear backward (VCAS) on B200.
+
+Workload: the BERT-base FFN up-projection layer (N=32, T=128, 768 -> 3072, bf16 inputs, fp32
+accumulation) at keep ratios rho = 0.3, nu = 0.4, with the variance probe (M = 4 Monte-Carlo
+batches) and the ratio update run once every F = 100 backward calls.
+
+One STEP = one adaptation period of Alg. 1: 1 probe + 1 ratio update + F sampled backward
+calls.  The metric is milliseconds per layer backward = step time / F (probe amortised in).
+Inputs rotate over 8 distinct (X, dY) batches (252 MB > the 126 MB L2), so every call reads
+its inputs from HBM.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = "bert_base_ffn_up"
+F_CALLS = 100
+PROBE_M = 4
+N_BATCHES = 8
+METRIC = "sampled linear-bwd ms/layer"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm=d["hbm_gbs"], tc_burst=d["bf16_tflops"], tc_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, tc_burst=1590.0, tc_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def oracle_call(case, batch=0, seed=0):
+    """One sampled backward of the workload by the CPU oracle; returns seconds."""
+    import numpy as np
+    from oracle import vcas_oracle as o
+    from paper_2402_17227_b200 import inputs
+    X, dY, W = inputs.make_layer(case, batch=batch)
+    to64 = lambda t: t.float().numpy().astype(np.float64)
+    X, dY, W = to64(X), to64(dY), to64(W)
+    t0 = time.perf_counter()
+    o.linear_bwd(X, dY, W, case.N, case.T, float(np.float32(case.rho)), float(np.float32(case.nu)), seed)
+    return time.perf_counter() - t0
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    """The oracle as it stands, on the host cores: each step is one sampled backward of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy  # noqa: F401  (loads BLAS so that the thread count can be read)
+    from paper_2402_17227_b200 import inputs
+    case = inputs.CASES[WORKLOAD]
+    for w in range(args.warmup):
+        oracle_call(case, batch=w % N_BATCHES, seed=w)
+    ts = [oracle_call(case, batch=k % N_BATCHES, seed=1000 + k) for k in range(args.steps)]
+    ms = 1e3 * sum(ts) / len(ts)
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": ms, "unit": "ms", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "N": case.N, "T": case.T, "d_in": case.d_in, "d_out": case.d_out,
+                   "rho": case.rho, "nu": case.nu, "step": "one sampled backward of the layer by the CPU oracle"},
+        "cpu_baseline": {"value": ms, "unit": "ms", "cores": cores, "kind": "oracle",
+                         "sample": f"{args.steps} full-size sampled backward calls, one per step"},
+        "e2e": {"value": ms, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="vcas", choices=["vcas", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    args.warmup = max(args.warmup, 3)
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2402_17227_b200 import binding as vb
+    from paper_2402_17227_b200 import build as vbuild
+    from paper_2402_17227_b200 import inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        vbuild.build()
+    if world > 1:
+        dist.barrier()
+    vb.lib()
+
+    case = inputs.CASES[WORKLOAD]
+    N, T, d_in, d_out, R = case.N, case.T, case.d_in, case.d_out, case.R
+    rho, nu = case.rho, case.nu
+    cfg = vb.default_config()
+    cfg.F, cfg.M = F_CALLS, PROBE_M
+    layer = vb.Layer(N, T, d_in, d_out, case.dtype, vb.GEMM_AUTO, cfg)
+
+    # rank r draws its own batches (data-parallel replicas: per-replica sampling, no exchange here)
+    host = [inputs.make_layer(case, batch=rank * N_BATCHES + b) for b in range(N_BATCHES)]
+    W = host[0][2].to(dev)
+    Xs = [h[0].to(dev) for h in host]
+    dYs = [h[1].to(dev) for h in host]
+    dX = torch.empty(R, d_in, dtype=case.dtype, device=dev)
+    dW = torch.empty(d_out, d_in, dtype=torch.float32, device=dev)
+    probe_out = torch.zeros(5, dtype=torch.float32, device=dev)
+    state = dict(s=1.0, rho=[1.0], nu=[1.0])
+    call_no = [0]
+
+    def step():
+        # Alg. 1: every F calls probe the variances on M batches and update (s, rho_l, nu_l) ...
+        layer.variance_probe(Xs[:PROBE_M], dYs[:PROBE_M], W, rho, nu, state["s"], 7777 + call_no[0], out=probe_out)
+        v = probe_out.cpu().numpy()
+        s_new, rho_new, nu_new = vb.update_ratios(state["s"], state["rho"], state["nu"], [v[0]], [v[1]], [v[2]],
+                                                  [v[3]], [v[4]], cfg)
+        state.update(s=s_new, rho=rho_new, nu=nu_new)
+        # ... then F sampled backward calls (at the workload's fixed ratios, so that every step does the same work)
+        for _ in range(F_CALLS):
+            b = call_no[0] % N_BATCHES
+            layer.linear_bwd_plain(Xs[b], dYs[b], W, rho, nu, call_no[0], dX, dW)
+            call_no[0] += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, reps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        step()
+    clocks = ClockSampler(local)
+    if rank == 0:
+        clocks.start()
+    l0 = layer.launch_count()
+    total_ms = timed(step, args.steps)
+    launches = layer.launch_count() - l0
+    clock_info = clocks.stop() if rank == 0 else None
+    ms_per_step = total_ms / args.steps
+    value = ms_per_step / (F_CALLS * world)      # whole-job: all ranks' calls per unit time
+
+    # -- the same period without the probe, the dense backward, and per-stage times (second passes)
+    def calls_only():
+        for _ in range(F_CALLS):
+            b = call_no[0] % N_BATCHES
+            layer.linear_bwd_plain(Xs[b], dYs[b], W, rho, nu, call_no[0], dX, dW)
+            call_no[0] += 1
+
+    def dense_only():
+        for _ in range(F_CALLS):
+            b = call_no[0] % N_BATCHES
+            layer.dense_bwd(Xs[b], dYs[b], W, dX=dX, dW=dW)
+            call_no[0] += 1
+
+    dense_only()
+    reps = max(1, min(args.steps, 5))
+    ms_sampled = timed(calls_only, reps) / (reps * F_CALLS)
+    ms_dense = timed(dense_only, reps) / (reps * F_CALLS)
+    layer.set_profiling(True)
+    calls_only(); dense_only()
+    stage_ms, stage_calls = layer.stage_times()
+    layer.set_profiling(False)
+    smp = layer.last_sampling()
+    kept_A, kept_W = smp.cntA * T, smp.cntW
+    assert layer.device_status() == 0, "device-side wait timed out"
+
+    # -- end to end through the C ABI from pinned host buffers (H2D of X, dY; D2H of dX, dW every call)
+    pin = [(h[0].pin_memory(), h[1].pin_memory()) for h in host[:2]]
+    hX, hdY = torch.empty_like(Xs[0]), torch.empty_like(dYs[0])
+    out_dX = torch.empty(R, d_in, dtype=case.dtype).pin_memory()
+    out_dW = torch.empty(d_out, d_in, dtype=torch.float32).pin_memory()
+
+    def e2e_calls(n):
+        for k in range(n):
+            hX.copy_(pin[k % 2][0], non_blocking=True)
+            hdY.copy_(pin[k % 2][1], non_blocking=True)
+            layer.linear_bwd_plain(hX, hdY, W, rho, nu, 424242 + k, dX, dW)
+            out_dX.copy_(dX, non_blocking=True)
+            out_dW.copy_(dW, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_calls(3)
+    n_e2e = 20
+    e2e_ms = timed(lambda: e2e_calls(n_e2e), 1) / (n_e2e * world)
+    h2d = Xs[0].numel() * 2 + dYs[0].numel() * 2
+    d2h = dX.numel() * 2 + dW.numel() * 4
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    nc = max(1, stage_calls[0])
+    per = [m / nc for m in stage_ms[:5]]
+    names = ["rownorm_kernel", "sampler_kernel", "umma_dx_kernel", "pack_kernel", "umma_dw_kernel"]
+    bytes_score = (R * d_out + R * d_in) * 2                      # every input byte read once
+    flops_dx = 2.0 * kept_A * d_in * d_out
+    flops_dw = 2.0 * kept_W * d_in * d_out
+    stages = {
+        "rownorm_kernel": dict(ms=per[0], bound="hbm", achieved=bytes_score / per[0] / 1e6 if per[0] else None),
+        "sampler_kernel": dict(ms=per[1], bound="latency"),
+        "umma_dx_kernel": dict(ms=per[2], bound="tensor", achieved=flops_dx / per[2] / 1e9 if per[2] else None),
+        "pack_kernel": dict(ms=per[3], bound="hbm"),
+        "umma_dw_kernel": dict(ms=per[4], bound="tensor", achieved=flops_dw / per[4] / 1e9 if per[4] else None),
+    }
+    dom = max(range(5), key=lambda i: per[i])
+    dname = names[dom]
+    if stages[dname]["bound"] == "tensor":
+        roof = dict(bound="tensor", kernel=dname, achieved=stages[dname]["achieved"], peak=pk["tc_burst"],
+                    unit="TFLOP/s", traffic=None, peak_source=pk["source"] + " bf16 burst")
+    else:
+        if dname != "rownorm_kernel":   # the small latency-bound stages are reported under the scoring pass
+            dname = "rownorm_kernel"
+        roof = dict(bound="hbm", kernel=dname, achieved=stages[dname]["achieved"], peak=pk["hbm"], unit="GB/s",
+                    traffic=None, peak_source=pk["source"] + " copy bandwidth")
+    roof["frac"] = roof["achieved"] / roof["peak"] if roof["achieved"] else None
+    roof["kernel_ms"] = stages[dname]["ms"]
+
+    flops_ratio = 2.0 * R / max(1, kept_A + kept_W)
+    line = {
+        "metric": METRIC, "value": value, "unit": "ms", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "N": N, "T": T, "d_in": d_in, "d_out": d_out, "rho": rho, "nu": nu,
+                   "step": f"1 variance probe (M={PROBE_M}) + 1 ratio update + {F_CALLS} sampled backward calls",
+                   "l2": f"inputs rotate over {N_BATCHES} batches (252 MB > 126 MB L2)",
+                   "parallelism": f"{world} data-parallel replica(s), no exchange"},
+        "clocks": clock_info,
+        "e2e": {"value": e2e_ms, "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "note": "one vcas_linear_bwd per step with X, dY copied from pinned host memory and dX, dW copied back"},
+        "gpu_launches": int(launches),
+        "roofline": roof,
+        "stages": stages,
+        "sampled_ms_per_layer": ms_sampled, "dense_ms_per_layer": ms_dense,
+        "speedup_vs_dense": ms_dense / ms_sampled if ms_sampled else None,
+        "flops_reduction_ratio": flops_ratio,
+        "speedup_over_flops_ratio": (ms_dense / ms_sampled) / flops_ratio if ms_sampled else None,
+        "dense_tflops": 4.0 * R * d_in * d_out / ms_dense / 1e9,
+        "kept_rows": {"kept_A": int(kept_A), "kept_W": int(kept_W), "R": R},
+        "adaptation_state": state,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        ts = [oracle_call(case, batch=k % N_BATCHES, seed=k) for k in range(30)]
+        line["cpu_baseline"] = {"value": 1e3 * sum(ts) / len(ts), "unit": "ms", "cores": blas_threads(),
+                                "kind": "oracle", "sample": "30 full-size sampled backward calls of the workload"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -174,6 +174,17 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
  * (VCAS_OK or VCAS_ERR_TIMEOUT / VCAS_ERR_INTERNAL); the word is then cleared. */
 int vcas_last_device_status(vcas_handle h, int32_t* status);
 
+/* Stage timing for benchmarks (the paper has no counterpart; Sec. 6 only reports end-to-end
+ * hours).  While enabled, vcas_linear_bwd(_ex) and vcas_dense_bwd record CUDA events on the
+ * caller's stream at their stage boundaries, for up to 2048 calls of each kind.  Enabling
+ * allocates the events once (host objects); it also clears what was recorded. */
+int vcas_set_profiling(vcas_handle h, int32_t enable);
+/* Synchronises the device, then writes the summed milliseconds of the recorded calls to
+ * ms[0..7] (host): 0 row norms, 1 keep probabilities + masks + compaction, 2 dX product,
+ * 3 pack of the kept rows, 4 dW product, 5 dense dX, 6 dense dW, 7 unused; calls[0..1] (host)
+ * = recorded sampled / dense calls.  Clears the record. */
+int vcas_stage_times(vcas_handle h, float* ms, int32_t* calls);
+
 /* Number of this library's kernel launches enqueued through the handle so far (host out). */
 int vcas_launch_count(vcas_handle h, uint64_t* launches);
 

@@ -24,6 +24,7 @@ GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
 EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
            "vcas_linear_bwd_ex", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
+           "vcas_set_profiling", "vcas_stage_times",
            "vcas_version"]
 
 
@@ -208,6 +209,16 @@ class Layer:
         st = C.c_int32(0)
         _check(lib().vcas_last_device_status(self._h, C.byref(st)), "vcas_last_device_status")
         return st.value
+
+    def set_profiling(self, enable: bool) -> None:
+        _check(lib().vcas_set_profiling(self._h, C.c_int32(1 if enable else 0)), "vcas_set_profiling")
+
+    def stage_times(self):
+        """(ms[8], calls[2]) summed over the calls recorded since profiling was enabled or last read."""
+        ms = (C.c_float * 8)()
+        calls = (C.c_int32 * 2)()
+        _check(lib().vcas_stage_times(self._h, ms, calls), "vcas_stage_times")
+        return list(ms), list(calls)
 
     def launch_count(self) -> int:
         n = C.c_uint64(0)

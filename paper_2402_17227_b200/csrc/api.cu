@@ -91,6 +91,14 @@ int sampled_dw(Handle* h, const void* X, const void* dY, float* out, cudaStream_
   return VCAS_OK;
 }
 
+// stage boundary k of the current sampled call (no-op unless profiling is on)
+inline void mark(Handle* h, int k, cudaStream_t st) {
+  if (h->prof_enabled && h->prof_calls < PROF_RING) cudaEventRecord(h->ev[h->prof_calls * 6 + k], st);
+}
+inline void mark_dense(Handle* h, int k, cudaStream_t st) {
+  if (h->prof_enabled && h->prof_dense_calls < PROF_RING) cudaEventRecord(h->ev_dense[h->prof_dense_calls * 3 + k], st);
+}
+
 int dense_dw(Handle* h, const void* X, const void* dY, float* out, cudaStream_t st) {
   if (h->tensor_path) {
     VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, out, st));
@@ -136,6 +144,10 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->tensor_path = tensor_ok && desc->gemm_path != VCAS_GEMM_FMA;
   h->R_pad = (desc->N * desc->T + 63) / 64 * 64;
   h->launches = 0;
+  h->prof_enabled = false;
+  h->ev = nullptr;
+  h->ev_dense = nullptr;
+  h->prof_calls = h->prof_dense_calls = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&h->device) != cudaSuccess || cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
     delete h;
@@ -164,6 +176,12 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
 int vcas_destroy(vcas_handle hh) {
   if (hh == nullptr) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
+  if (h->ev != nullptr) {
+    for (int i = 0; i < PROF_RING * 6; ++i) cudaEventDestroy(h->ev[i]);
+    for (int i = 0; i < PROF_RING * 3; ++i) cudaEventDestroy(h->ev_dense[i]);
+    delete[] h->ev;
+    delete[] h->ev_dense;
+  }
   const cudaError_t e = cudaFree(h->base);
   delete h;
   return e == cudaSuccess ? VCAS_OK : VCAS_ERR_CUDA;
@@ -189,16 +207,30 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
+  mark(h, 0, st);
   VCAS_CUDA(launch_rownorms(h, dY, X, st));
+  mark(h, 1, st);
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
   VCAS_CUDA(launch_sampler(h, a, st));
+  mark(h, 2, st);
   if (h->tensor_path) {
     VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, h->ws.scaleA, Hpre, dX, st));
   }
-  return sampled_dw(h, X, dY, dW, st);
+  mark(h, 3, st);
+  if (h->tensor_path) {
+    VCAS_CUDA(launch_pack(h, dY, X, st));
+    mark(h, 4, st);
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, dW, st));
+  } else {
+    mark(h, 4, st);
+    VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, dW, st));
+  }
+  mark(h, 5, st);
+  if (h->prof_enabled && h->prof_calls < PROF_RING) h->prof_calls += 1;
+  return VCAS_OK;
 }
 
 int vcas_linear_bwd(vcas_handle hh, const void* X, const void* dY, const void* W, float rho, float nu,
@@ -212,12 +244,17 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
     return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
+  mark_dense(h, 0, st);
   if (h->tensor_path) {
     VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }
-  return dense_dw(h, X, dY, dW, st);
+  mark_dense(h, 1, st);
+  const int rc = dense_dw(h, X, dY, dW, st);
+  mark_dense(h, 2, st);
+  if (h->prof_enabled && h->prof_dense_calls < PROF_RING) h->prof_dense_calls += 1;
+  return rc;
 }
 
 int vcas_score(vcas_handle hh, const void* X, const void* dY, float rho, float nu, uint64_t seed, float* g,
@@ -313,6 +350,45 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
     if (nu < (double)cfg->nu_min) nu = (double)cfg->nu_min;
     state->nu[l] = (float)nu;
   }
+  return VCAS_OK;
+}
+
+int vcas_set_profiling(vcas_handle hh, int32_t enable) {
+  if (hh == nullptr) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  if (enable && h->ev == nullptr) {
+    h->ev = new (std::nothrow) cudaEvent_t[PROF_RING * 6];
+    h->ev_dense = new (std::nothrow) cudaEvent_t[PROF_RING * 3];
+    if (h->ev == nullptr || h->ev_dense == nullptr) return VCAS_ERR_WORKSPACE;
+    for (int i = 0; i < PROF_RING * 6; ++i) VCAS_CUDA(cudaEventCreate(&h->ev[i]));
+    for (int i = 0; i < PROF_RING * 3; ++i) VCAS_CUDA(cudaEventCreate(&h->ev_dense[i]));
+  }
+  h->prof_enabled = enable != 0;
+  h->prof_calls = h->prof_dense_calls = 0;
+  return VCAS_OK;
+}
+
+int vcas_stage_times(vcas_handle hh, float* ms, int32_t* calls) {
+  if (hh == nullptr || ms == nullptr || calls == nullptr) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  for (int k = 0; k < 8; ++k) ms[k] = 0.f;
+  calls[0] = h->prof_calls;
+  calls[1] = h->prof_dense_calls;
+  if (h->ev == nullptr) return VCAS_OK;
+  VCAS_CUDA(cudaDeviceSynchronize());
+  for (int c = 0; c < h->prof_calls; ++c)
+    for (int k = 0; k < 5; ++k) {
+      float t = 0.f;
+      VCAS_CUDA(cudaEventElapsedTime(&t, h->ev[c * 6 + k], h->ev[c * 6 + k + 1]));
+      ms[k] += t;
+    }
+  for (int c = 0; c < h->prof_dense_calls; ++c)
+    for (int k = 0; k < 2; ++k) {
+      float t = 0.f;
+      VCAS_CUDA(cudaEventElapsedTime(&t, h->ev_dense[c * 3 + k], h->ev_dense[c * 3 + k + 1]));
+      ms[5 + k] += t;
+    }
+  h->prof_calls = h->prof_dense_calls = 0;
   return VCAS_OK;
 }
 

@@ -53,7 +53,13 @@ struct Handle {
   size_t bytes;
   Workspace ws;
   uint64_t launches;
+  // optional stage timing (vcas_set_profiling): rings of CUDA events around the stages
+  bool prof_enabled;
+  cudaEvent_t* ev;        // [PROF_RING][6]: boundaries of row norms | sampler | dX | pack | dW
+  cudaEvent_t* ev_dense;  // [PROF_RING][3]: boundaries of dense dX | dense dW
+  int prof_calls, prof_dense_calls;
 };
+constexpr int PROF_RING = 2048;
 
 // ---------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies.
