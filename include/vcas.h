@@ -129,6 +129,29 @@ int vcas_score(vcas_handle h, const void* X, const void* dY, float rho, float nu
                float* g, float* p, float* w, float* q,
                int32_t* idxA, int32_t* cntA, int32_t* idxW, int32_t* cntW, vcas_stream stream);
 
+/*
+ * vcas_score without a handle and without any allocation (the paper has no counterpart; this
+ * exists for the library's users).  Some callers may not allocate device memory at the point
+ * where they need the scores: code running inside a framework's memory-pool region or a
+ * real-time loop where cudaMalloc's implicit synchronisation and possible failure are not
+ * acceptable, or plug-ins that are handed a fixed memory budget.  vcas_create / vcas_score need a
+ * workspace from cudaMalloc; this entry point instead keeps its intermediates (row norms,
+ * scores, rescale factors, index lists) in a fixed array inside the library image, about
+ * 0.5 MB that every GPU loading the library holds until the process exits.
+ *   Limits: N <= 4096 and N*T <= 16384, otherwise VCAS_ERR_SHAPE.  d_in, d_out multiples of 8.
+ *   Inputs and outputs are the caller's, as for vcas_score (any output may be NULL).
+ *   The first call on each device looks up the array's device address (with that device
+ *   current); make that first call before starting any stream capture.
+ *   All calls on a device share the one array, which keeps the previous call's contents (the
+ *   call itself clears what has to start at zero): two calls whose GPU work overlaps, e.g. on
+ *   different streams, race.  Calls on one stream are safe.
+ * It calls no cudaMalloc, cudaFree or allocating library routine.
+ */
+int vcas_score_static(int32_t N, int32_t T, int32_t d_in, int32_t d_out, int32_t dtype,
+                      const void* X, const void* dY, float rho, float nu, uint64_t seed,
+                      float* g, float* p, float* w, float* q,
+                      int32_t* idxA, int32_t* cntA, int32_t* idxW, int32_t* cntW, vcas_stream stream);
+
 /* Copies what the last vcas_linear_bwd(_ex) or vcas_score on this handle computed (same
  * outputs as vcas_score); enqueue on the same stream. */
 int vcas_last_sampling(vcas_handle h, float* g, float* p, float* w, float* q,

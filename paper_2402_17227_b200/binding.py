@@ -24,7 +24,7 @@ GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
 EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
            "vcas_linear_bwd_ex", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
-           "vcas_set_profiling", "vcas_stage_times",
+           "vcas_set_profiling", "vcas_stage_times", "vcas_score_static",
            "vcas_version"]
 
 
@@ -241,6 +241,23 @@ def update_ratios(s: float, rho, nu, V_s, V_act, V_w, p_lo, p_hi, config: Config
                                   C.byref(config))
     _check(rc, "vcas_update_ratios")
     return st.s, list(rho_a), list(nu_a)
+
+
+def score_static(X, dY, N: int, T: int, rho: float, nu: float, seed: int) -> Sampling:
+    """vcas_score_static: scores, probabilities and index lists without a handle or any device
+    allocation by the library (the output tensors below are the caller's, made by torch).
+    Limits: N <= 4096, N*T <= 16384.  Calls sharing a device must not overlap on the GPU."""
+    R, dev = N * T, X.device
+    f = dict(dtype=torch.float32, device=dev)
+    i = dict(dtype=torch.int32, device=dev)
+    b = (torch.empty(N, **f), torch.empty(N, **f), torch.empty(R, **f), torch.empty(R, **f),
+         torch.empty(N, **i), torch.zeros(1, **i), torch.empty(R, **i), torch.zeros(1, **i))
+    dt = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[X.dtype]
+    rc = lib().vcas_score_static(C.c_int32(N), C.c_int32(T), C.c_int32(X.shape[1]), C.c_int32(dY.shape[1]),
+                                 C.c_int32(dt), _ptr(X), _ptr(dY), C.c_float(rho), C.c_float(nu), C.c_uint64(seed),
+                                 *[_ptr(t) for t in b], _stream())
+    _check(rc, "vcas_score_static")
+    return Layer._pack_sampling(b)
 
 
 def version() -> int:
