@@ -185,18 +185,44 @@ def main():
     state = dict(s=1.0, rho=[1.0], nu=[1.0])
     call_no = [0]
 
+    def calls_only():
+        for _ in range(F_CALLS):
+            b = call_no[0] % N_BATCHES
+            layer.linear_bwd_plain(Xs[b], dYs[b], W, rho, nu, call_no[0], dX, dW)
+            call_no[0] += 1
+
+    def dense_only():
+        for _ in range(F_CALLS):
+            b = call_no[0] % N_BATCHES
+            layer.dense_bwd(Xs[b], dYs[b], W, dX=dX, dW=dW)
+            call_no[0] += 1
+
+    # The F backward calls of a period are captured once into a CUDA graph (the library neither
+    # synchronises nor allocates, so its calls can be captured) and replayed every step: a training
+    # loop would capture its step the same way, and replay removes the host's launch cost.
+    calls_only(); dense_only()
+    torch.cuda.synchronize()
+    l_before = layer.launch_count()
+    graph_calls = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph_calls):
+        calls_only()
+    launches_per_period = layer.launch_count() - l_before
+    graph_dense = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph_dense):
+        dense_only()
+    probe_launches = [0]
+
     def step():
         # Alg. 1: every F calls probe the variances on M batches and update (s, rho_l, nu_l) ...
+        l0 = layer.launch_count()
         layer.variance_probe(Xs[:PROBE_M], dYs[:PROBE_M], W, rho, nu, state["s"], 7777 + call_no[0], out=probe_out)
+        probe_launches[0] = layer.launch_count() - l0
         v = probe_out.cpu().numpy()
         s_new, rho_new, nu_new = vb.update_ratios(state["s"], state["rho"], state["nu"], [v[0]], [v[1]], [v[2]],
                                                   [v[3]], [v[4]], cfg)
         state.update(s=s_new, rho=rho_new, nu=nu_new)
         # ... then F sampled backward calls (at the workload's fixed ratios, so that every step does the same work)
-        for _ in range(F_CALLS):
-            b = call_no[0] % N_BATCHES
-            layer.linear_bwd_plain(Xs[b], dYs[b], W, rho, nu, call_no[0], dX, dW)
-            call_no[0] += 1
+        graph_calls.replay()
 
     def barrier():
         if world > 1:
@@ -223,34 +249,37 @@ def main():
     clocks = ClockSampler(local)
     if rank == 0:
         clocks.start()
-    l0 = layer.launch_count()
     total_ms = timed(step, args.steps)
-    launches = layer.launch_count() - l0
+    launches = args.steps * (launches_per_period + probe_launches[0])
     clock_info = clocks.stop() if rank == 0 else None
     ms_per_step = total_ms / args.steps
     value = ms_per_step / (F_CALLS * world)      # whole-job: all ranks' calls per unit time
 
-    # -- the same period without the probe, the dense backward, and per-stage times (second passes)
-    def calls_only():
-        for _ in range(F_CALLS):
-            b = call_no[0] % N_BATCHES
-            layer.linear_bwd_plain(Xs[b], dYs[b], W, rho, nu, call_no[0], dX, dW)
-            call_no[0] += 1
-
-    def dense_only():
-        for _ in range(F_CALLS):
-            b = call_no[0] % N_BATCHES
-            layer.dense_bwd(Xs[b], dYs[b], W, dX=dX, dW=dW)
-            call_no[0] += 1
-
-    dense_only()
-    reps = max(1, min(args.steps, 5))
-    ms_sampled = timed(calls_only, reps) / (reps * F_CALLS)
-    ms_dense = timed(dense_only, reps) / (reps * F_CALLS)
+    # -- the same period without the probe, the dense backward (graph replays), and per-stage times
+    reps = max(3, min(args.steps, 10))
+    ms_sampled = timed(graph_calls.replay, reps) / (reps * F_CALLS)
+    ms_dense = timed(graph_dense.replay, reps) / (reps * F_CALLS)
+    ms_sampled_eager = timed(calls_only, 3) / (3 * F_CALLS)
+    # Stage times with CUDA events at the stage boundaries.  The calls are enqueued behind a few ms of
+    # other GPU work, so that all their launches are already queued when the GPU reaches them and the
+    # events bracket GPU time, not the host's launch cost.
+    blocker = torch.empty(8192, 8192, dtype=torch.bfloat16, device=dev).normal_()
     layer.set_profiling(True)
-    calls_only(); dense_only()
+    torch.cuda.synchronize()
+    for _ in range(6):
+        torch.mm(blocker, blocker)
+    for k in range(40):
+        b = k % N_BATCHES
+        layer.linear_bwd_plain(Xs[b], dYs[b], W, rho, nu, 99000 + k, dX, dW)
     stage_ms, stage_calls = layer.stage_times()
+    for _ in range(6):
+        torch.mm(blocker, blocker)
+    for k in range(40):
+        b = k % N_BATCHES
+        layer.dense_bwd(Xs[b], dYs[b], W, dX=dX, dW=dW)
+    dense_stage_ms, dense_calls = layer.stage_times()
     layer.set_profiling(False)
+    del blocker
     smp = layer.last_sampling()
     kept_A, kept_W = smp.cntA * T, smp.cntW
     assert layer.device_status() == 0, "device-side wait timed out"
@@ -314,7 +343,8 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "N": N, "T": T, "d_in": d_in, "d_out": d_out, "rho": rho, "nu": nu,
-                   "step": f"1 variance probe (M={PROBE_M}) + 1 ratio update + {F_CALLS} sampled backward calls",
+                   "step": f"1 variance probe (M={PROBE_M}) + 1 ratio update + {F_CALLS} sampled backward calls "
+                           "(the calls replayed from one CUDA graph)",
                    "l2": f"inputs rotate over {N_BATCHES} batches (252 MB > 126 MB L2)",
                    "parallelism": f"{world} data-parallel replica(s), no exchange"},
         "clocks": clock_info,
@@ -324,6 +354,9 @@ def main():
         "roofline": roof,
         "stages": stages,
         "sampled_ms_per_layer": ms_sampled, "dense_ms_per_layer": ms_dense,
+        "sampled_ms_per_layer_eager_launch": ms_sampled_eager,
+        "dense_stages_ms": {"umma_dx_kernel": dense_stage_ms[5] / max(1, dense_calls[1]),
+                            "umma_dw_kernel": dense_stage_ms[6] / max(1, dense_calls[1])},
         "speedup_vs_dense": ms_dense / ms_sampled if ms_sampled else None,
         "flops_reduction_ratio": flops_ratio,
         "speedup_over_flops_ratio": (ms_dense / ms_sampled) / flops_ratio if ms_sampled else None,

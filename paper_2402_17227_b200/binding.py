@@ -24,7 +24,7 @@ GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
 EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
            "vcas_linear_bwd_ex", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
-           "vcas_set_profiling", "vcas_stage_times", "vcas_score_static",
+           "vcas_set_profiling", "vcas_stage_times", "vcas_score_static", "vcas_set_tuning",
            "vcas_version"]
 
 
@@ -209,6 +209,10 @@ class Layer:
         st = C.c_int32(0)
         _check(lib().vcas_last_device_status(self._h, C.byref(st)), "vcas_last_device_status")
         return st.value
+
+    def set_tuning(self, dx_tile_n: int = 0, dw_tile_n: int = 0, dx_split_k: int = 0) -> None:
+        _check(lib().vcas_set_tuning(self._h, C.c_int32(dx_tile_n), C.c_int32(dw_tile_n), C.c_int32(dx_split_k)),
+               "vcas_set_tuning")
 
     def set_profiling(self, enable: bool) -> None:
         _check(lib().vcas_set_profiling(self._h, C.c_int32(1 if enable else 0)), "vcas_set_profiling")

@@ -58,6 +58,8 @@ struct Handle {
   cudaEvent_t* ev;        // [PROF_RING][6]: boundaries of row norms | sampler | dX | pack | dW
   cudaEvent_t* ev_dense;  // [PROF_RING][3]: boundaries of dense dX | dense dW
   int prof_calls, prof_dense_calls;
+  // tuning overrides (vcas_set_tuning); 0 = choose automatically
+  int tune_dx_tile_n, tune_dw_tile_n, tune_dx_split_k;
 };
 constexpr int PROF_RING = 2048;
 

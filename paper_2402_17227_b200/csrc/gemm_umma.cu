@@ -602,7 +602,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   double kept = dense ? (double)d.N : (double)rho_hint * d.N;
   if (kept < 1.0) kept = 1.0;
   const long row_tiles = (long)(kept + 0.5) * ((d.T + BM - 1) / BM);
-  switch (pick_bn(row_tiles, d.d_in, h->num_sms)) {
+  switch (h->tune_dx_tile_n != 0 ? h->tune_dx_tile_n : pick_bn(row_tiles, d.d_in, h->num_sms)) {
     case 256: return run_dx<256>(h, tmA, tmB, P, st);
     case 128: return run_dx<128>(h, tmA, tmB, P, st);
     default: return run_dx<64>(h, tmA, tmB, P, st);
@@ -637,7 +637,7 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
   }
   DwParams P;
   P.cnt = cnt; P.dW = dW; P.status = h->ws.status; P.d_in = d.d_in; P.d_out = d.d_out;
-  switch (pick_bn((d.d_out + BM - 1) / BM, d.d_in, h->num_sms)) {
+  switch (h->tune_dw_tile_n != 0 ? h->tune_dw_tile_n : pick_bn((d.d_out + BM - 1) / BM, d.d_in, h->num_sms)) {
     case 256: return run_dw<256>(h, tmA, tmB, P, st);
     case 128: return run_dw<128>(h, tmA, tmB, P, st);
     default: return run_dw<64>(h, tmA, tmB, P, st);
