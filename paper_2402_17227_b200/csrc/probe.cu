@@ -60,12 +60,21 @@ __global__ void __launch_bounds__(256) reduce_kernel(const float4* __restrict__ 
     last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
   }
   __syncthreads();
-  if (last && threadIdx.x == 0) {
+  if (last) {
+    // the last block adds the block partials: each thread a fixed strided subset, then a fixed tree
     __threadfence();
     double tot = 0.0;
-    for (unsigned i = 0; i < gridDim.x; ++i) tot += ((volatile double*)partial)[i];
-    *acc += tot;
-    *ticket = 0;
+    for (unsigned i = threadIdx.x; i < gridDim.x; i += blockDim.x) tot += __ldcg(partial + i);
+    tot = warp_sum(tot);
+    __syncthreads();
+    if (lane == 0) sh[warp] = tot;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double b = 0.0;
+      for (int i = 0; i < 8; ++i) b += sh[i];
+      *acc += b;
+      *ticket = 0;
+    }
   }
 }
 

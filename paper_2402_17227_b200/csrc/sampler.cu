@@ -200,6 +200,285 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_kernel(SamplerParams 
   if (tid == 0) { P.counts[0] = cntA; P.counts[1] = cntW; }
 }
 
+// ---------------------------------------------------------------------------------------
+// Fast path for R <= 16 * 1024 rows and N <= 1024 data: every thread keeps its E consecutive
+// rows in registers, SampleA runs inside warp 0 with shuffles only, and each water-filling
+// iteration over the rows costs two block barriers.
+// ---------------------------------------------------------------------------------------
+struct FastShared {
+  float part_f[2][32];
+  int part_i[2][32];
+  float tot_f[2];
+  int tot_i[2];
+  int warp_tot[32];
+  float scaleA[1024];
+  float pA[1024];
+  int cntA;
+};
+
+// Block-wide sum of one float and one int in a fixed order (lanes by shuffle tree, then the 32
+// warp totals by a shuffle tree in warp 0).  fp32 on purpose: this is a single-CTA kernel, and
+// double-precision arithmetic concentrated on one SM was measured to dominate its run time; a
+// tree sum of <= 16384 non-negative fp32 terms is accurate to about 1e-6, inside the 1e-5 the
+// probabilities are specified to.
+__device__ __forceinline__ void fast_sum(float& s, int& c, FastShared* sh, int parity) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  s = warp_sum(s);
+  c = warp_sum(c);
+  if (lane == 0) { sh->part_f[parity][warp] = s; sh->part_i[parity][warp] = c; }
+  __syncthreads();
+  if (warp == 0) {
+    const float ts = warp_sum(sh->part_f[parity][lane]);
+    const int tc = warp_sum(sh->part_i[parity][lane]);
+    if (lane == 0) { sh->tot_f[parity] = ts; sh->tot_i[parity] = tc; }
+  }
+  __syncthreads();
+  s = sh->tot_f[parity];
+  c = sh->tot_i[parity];
+}
+
+// capped_prop over at most 32 values per lane of ONE warp (value i of the array sits in lane i % 32,
+// slot i / 32); p is returned in place of v.
+template <int SLOTS>
+__device__ void capped_prop_warp(float (&v)[SLOTS], float budget) {
+  float S = 0.f;
+  int nz = 0;
+#pragma unroll
+  for (int j = 0; j < SLOTS; ++j)
+    if (v[j] > 0.f) { S += v[j]; ++nz; }
+  S = warp_sum(S);
+  nz = warp_sum(nz);
+  if (nz == 0 || budget <= 0.f) {
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j) v[j] = 0.f;
+    return;
+  }
+  if ((float)nz <= budget) {
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j) v[j] = v[j] > 0.f ? 1.f : 0.f;
+    return;
+  }
+  float c = budget / S;
+  int k = 0;
+  for (int iter = 0; iter < 128; ++iter) {
+    float Su = 0.f;
+    int ks = 0;
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j)
+      if (v[j] > 0.f) {
+        if (c * v[j] >= 1.0f) ++ks; else Su += v[j];
+      }
+    Su = warp_sum(Su);
+    ks = warp_sum(ks);
+    if (ks == k) break;
+    k = ks;
+    if (Su > 0.f) {
+      const float cn = (budget - (float)k) / Su;
+      c = cn > c ? cn : c;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < SLOTS; ++j) {
+    float r = 0.f;
+    if (v[j] > 0.f) {
+      const float cx = c * v[j];
+      r = cx >= 1.0f ? 1.f : cx;
+    }
+    v[j] = r;
+  }
+}
+
+template <int E, int SLOTS>
+__global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerParams P) {
+  __shared__ FastShared sh;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int N = P.N, T = P.T, R = N * T;
+  const int r0 = tid * E;
+
+  // this thread's rows: ||dY_r|| ||X_r|| (the unscaled leverage score)
+  float ab[E];
+#pragma unroll
+  for (int e = 0; e < E; e += 4) {
+    float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
+    if (r0 + e + 3 < R) {
+      va = *reinterpret_cast<const float4*>(P.a + r0 + e);
+      vb = *reinterpret_cast<const float4*>(P.b + r0 + e);
+    } else {
+      float ta[4] = {0.f, 0.f, 0.f, 0.f}, tb[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int i = 0; i < 4; ++i)
+        if (r0 + e + i < R) { ta[i] = P.a[r0 + e + i]; tb[i] = P.b[r0 + e + i]; }
+      va = make_float4(ta[0], ta[1], ta[2], ta[3]);
+      vb = make_float4(tb[0], tb[1], tb[2], tb[3]);
+    }
+    ab[e] = sqrtf(va.x) * sqrtf(vb.x); ab[e + 1] = sqrtf(va.y) * sqrtf(vb.y);
+    ab[e + 2] = sqrtf(va.z) * sqrtf(vb.z); ab[e + 3] = sqrtf(va.w) * sqrtf(vb.w);
+  }
+
+  // ---- ||G_n||_F: one warp per datum, fixed order
+  for (int n = warp; n < N; n += 32) {
+    float s = 0.f;
+    for (int t = lane; t < T; t += 32) s += P.a[(size_t)n * T + t];
+    s = warp_sum(s);
+    if (lane == 0) { const float g = sqrtf(s); P.g[n] = g; sh.pA[n] = g; }
+  }
+  __syncthreads();
+
+  // ---- SampleA inside warp 0 (Sec. 4.1): p_n, mask, kept / dropped lists
+  if (warp == 0) {
+    float v[SLOTS];
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j) { const int n = lane + 32 * j; v[j] = n < N ? sh.pA[n] : 0.f; }
+    if (P.p_in != nullptr) {
+#pragma unroll
+      for (int j = 0; j < SLOTS; ++j) { const int n = lane + 32 * j; v[j] = n < N ? P.p_in[n] : 0.f; }
+    } else {
+      capped_prop_warp<SLOTS>(v, (float)N * P.rho);
+    }
+    int kept_before = 0, drop_before = 0;
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j) {
+      const int n = lane + 32 * j;
+      const bool in = n < N;
+      const bool keep = in && bernoulli_keep(v[j], P.seed, 0u, (uint64_t)n);
+      const unsigned bk = __ballot_sync(0xffffffffu, keep);
+      const unsigned bd = __ballot_sync(0xffffffffu, in && !keep);
+      const unsigned lower = (1u << lane) - 1u;
+      if (in) {
+        P.p[n] = v[j];
+        const float sc = keep ? 1.0f / v[j] : 0.f;
+        P.scaleA[n] = sc;
+        sh.scaleA[n] = sc;
+        sh.pA[n] = v[j];
+        if (keep) P.idxA[kept_before + __popc(bk & lower)] = n;
+        else P.dropA[drop_before + __popc(bd & lower)] = n;
+      }
+      kept_before += __popc(bk);
+      drop_before += __popc(bd);
+    }
+    if (lane == 0) sh.cntA = kept_before;
+  }
+  __syncthreads();
+  const int cntA = sh.cntA;
+
+  // ---- SampleW (Sec. 4.2, Eq. 3): leverage scores of G_hat in registers
+  float w[E];
+#pragma unroll
+  for (int e = 0; e < E; ++e) {
+    const int r = r0 + e;
+    float wr = 0.f;
+    if (r < R) {
+      const int n = r / T;
+      if (sh.scaleA[n] > 0.f) wr = ab[e] / sh.pA[n];
+      P.w[r] = wr;
+    }
+    w[e] = wr;
+  }
+  float q[E];
+  if (P.q_in != nullptr) {
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      const int r = r0 + e;
+      q[e] = (r < R && sh.scaleA[r / T] > 0.f) ? P.q_in[r] : 0.f;
+    }
+  } else {
+    const float budget = P.nu * (float)T * (float)cntA;
+    float S = 0.f;
+    int nz = 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+      if (w[e] > 0.f) { S += w[e]; ++nz; }
+    int parity = 0;
+    fast_sum(S, nz, &sh, parity); parity ^= 1;
+    if (nz == 0 || budget <= 0.f) {
+#pragma unroll
+      for (int e = 0; e < E; ++e) q[e] = 0.f;
+    } else if ((float)nz <= budget) {
+#pragma unroll
+      for (int e = 0; e < E; ++e) q[e] = w[e] > 0.f ? 1.f : 0.f;
+    } else {
+      float c = budget / S;
+      int k = 0;
+      for (int iter = 0; iter < 128; ++iter) {
+        float Su = 0.f;
+        int ks = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e)
+          if (w[e] > 0.f) {
+            if (c * w[e] >= 1.0f) ++ks; else Su += w[e];
+          }
+        fast_sum(Su, ks, &sh, parity); parity ^= 1;
+        if (ks == k) break;
+        k = ks;
+        if (Su > 0.f) {
+          const float cn = (budget - (float)k) / Su;
+          c = cn > c ? cn : c;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        float r = 0.f;
+        if (w[e] > 0.f) {
+          const float cx = c * w[e];
+          r = cx >= 1.0f ? 1.f : cx;
+        }
+        q[e] = r;
+      }
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < E; ++e)
+    if (r0 + e < R) P.q[r0 + e] = q[e];
+
+  if (P.accumulate_vw) {      // Eq. 3 at these probabilities (probe only)
+    float vw = 0.f;
+    int dummy = 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+      if (q[e] > 0.f) vw += (1.0f - q[e]) / q[e] * w[e] * w[e];
+    fast_sum(vw, dummy, &sh, 0);
+    if (tid == 0) P.acc[1] += (double)vw;
+  }
+
+  // ---- mask and ordered compaction: per-thread count, block exclusive scan, scatter
+  unsigned keepbits = 0;
+#pragma unroll
+  for (int e = 0; e < E; ++e) {
+    const int r = r0 + e;
+    bool k = false;
+    if (r < R) {
+      if (P.sample_w) k = q[e] > 0.f && bernoulli_keep(q[e], P.seed, 1u, (uint64_t)r);
+      else k = sh.scaleA[r / T] > 0.f;
+    }
+    keepbits |= (k ? 1u : 0u) << e;
+  }
+  const int mine = __popc(keepbits);
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) sh.warp_tot[warp] = incl;
+  __syncthreads();
+  int base = incl - mine;
+  int total = 0;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const int t = sh.warp_tot[i];
+    if (i < warp) base += t;
+    total += t;
+  }
+#pragma unroll
+  for (int e = 0; e < E; ++e)
+    if (keepbits & (1u << e)) {
+      const int r = r0 + e;
+      P.idxW[base] = r;
+      P.scaleW[base] = P.sample_w ? sh.scaleA[r / T] / q[e] : sh.scaleA[r / T];
+      ++base;
+    }
+  if (tid == 0) { P.counts[0] = cntA; P.counts[1] = total; }
+}
+
 __global__ void __launch_bounds__(SAMPLER_THREADS)
 mask_kernel(const float* __restrict__ p, int n, uint64_t seed, int sampler, uint8_t* keep, int32_t* idx,
             int32_t* cnt) {
@@ -227,7 +506,22 @@ cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st) {
   P.N = h->desc.N; P.T = h->desc.T;
   P.rho = a.rho; P.nu = a.nu; P.seed = a.seed;
   P.sample_w = a.sample_w; P.accumulate_vw = a.accumulate_vw;
-  sampler_kernel<<<1, SAMPLER_THREADS, 0, st>>>(P);
+  const int R = P.N * P.T;
+  if (P.N <= 1024 && R <= 16 * SAMPLER_THREADS) {
+    const bool wide = P.N > 32;       // SampleA slots per lane of warp 0
+    if (R <= 4 * SAMPLER_THREADS) {
+      if (wide) sampler_fast_kernel<4, 32><<<1, SAMPLER_THREADS, 0, st>>>(P);
+      else sampler_fast_kernel<4, 1><<<1, SAMPLER_THREADS, 0, st>>>(P);
+    } else if (R <= 8 * SAMPLER_THREADS) {
+      if (wide) sampler_fast_kernel<8, 32><<<1, SAMPLER_THREADS, 0, st>>>(P);
+      else sampler_fast_kernel<8, 1><<<1, SAMPLER_THREADS, 0, st>>>(P);
+    } else {
+      if (wide) sampler_fast_kernel<16, 32><<<1, SAMPLER_THREADS, 0, st>>>(P);
+      else sampler_fast_kernel<16, 1><<<1, SAMPLER_THREADS, 0, st>>>(P);
+    }
+  } else {
+    sampler_kernel<<<1, SAMPLER_THREADS, 0, st>>>(P);
+  }
   h->launches += 1;
   return cudaGetLastError();
 }

@@ -79,6 +79,23 @@ def test_score_matches_oracle(dtype, shape):
     layer.close()
 
 
+@pytest.mark.parametrize("N,T", [(40, 250), (64, 100), (33, 31), (20, 1000), (1100, 3)])
+def test_score_kernel_variants(N, T):
+    """Row counts that select each variant of the sampling kernel (4, 8, 16 rows per thread, more than
+    32 data, and the general kernel beyond 16384 rows or 1024 data)."""
+    d_in = d_out = 64
+    X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.5, sigma_B=1.0, zero_fraction=0.1)
+    layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_FMA)
+    Xc, dYc = cuda(X, dY)
+    for seed, rho, nu in [(1, 0.3, 0.4), (5, 0.6, 0.2)]:
+        s = layer.score(Xc, dYc, rho, nu, seed)
+        ref = o.linear_bwd(np64(X), np64(dY), np64(W), N, T, f32(rho), f32(nu), seed)
+        ref["seed"] = seed
+        check_sampling(s, ref, N, T)
+    assert layer.device_status() == 0
+    layer.close()
+
+
 @pytest.mark.parametrize("n", [1, 31, 1024, 5000, 16384 + 17])
 def test_masks_bit_exact_given_oracle_probabilities(n):
     r = np.random.default_rng(n)
