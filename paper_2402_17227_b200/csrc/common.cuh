@@ -66,12 +66,9 @@ constexpr int PROF_RING = 2048;
 // ---------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies.
 // ---------------------------------------------------------------------------------------
-// Deliberately a real function with a rolled loop: the sampling kernels run once per call on a
-// single SM with a cold instruction cache, where the number of distinct instructions fetched,
-// not the number executed, sets the run time.
-static __device__ __noinline__ uint32_t philox_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                                     uint32_t k0, uint32_t k1) {
-#pragma unroll 1
+__device__ __forceinline__ uint32_t philox_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t k0, uint32_t k1) {
+#pragma unroll
   for (int r = 0; r < 10; ++r) {
     const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
     const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;

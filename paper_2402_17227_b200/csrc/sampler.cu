@@ -221,7 +221,7 @@ struct FastShared {
 // double-precision arithmetic concentrated on one SM was measured to dominate its run time; a
 // tree sum of <= 16384 non-negative fp32 terms is accurate to about 1e-6, inside the 1e-5 the
 // probabilities are specified to.
-static __device__ __noinline__ void fast_sum(float& s, int& c, FastShared* sh, int parity) {
+__device__ __forceinline__ void fast_sum(float& s, int& c, FastShared* sh, int parity) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   s = warp_sum(s);
   c = warp_sum(c);
@@ -288,9 +288,6 @@ __device__ void capped_prop_warp(float (&v)[SLOTS], float budget) {
   }
 }
 
-// ||dY_r|| ||X_r|| from the two square-norms (a real function: see philox_word0 on code size)
-static __device__ __noinline__ float leverage(float a, float b) { return sqrtf(a) * sqrtf(b); }
-
 template <int E, int SLOTS>
 __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerParams P) {
   __shared__ FastShared sh;
@@ -313,8 +310,8 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
       va = make_float4(ta[0], ta[1], ta[2], ta[3]);
       vb = make_float4(tb[0], tb[1], tb[2], tb[3]);
     }
-    ab[e] = leverage(va.x, vb.x); ab[e + 1] = leverage(va.y, vb.y);
-    ab[e + 2] = leverage(va.z, vb.z); ab[e + 3] = leverage(va.w, vb.w);
+    ab[e] = sqrtf(va.x) * sqrtf(vb.x); ab[e + 1] = sqrtf(va.y) * sqrtf(vb.y);
+    ab[e + 2] = sqrtf(va.z) * sqrtf(vb.z); ab[e + 3] = sqrtf(va.w) * sqrtf(vb.w);
   }
 
   // ---- ||G_n||_F: one warp per datum, fixed order
