@@ -53,9 +53,13 @@ size_t layout(Handle* h, uint8_t* base) {
   if (h->tensor_path) {
     w.packG = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_out);
     w.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
+    w.partial_tiles = carve<float>(cur, (size_t)h->max_units * 128 * 256);
+    w.tickets = carve<int32_t>(cur, 2 * (size_t)h->max_units);
   } else {
     w.packG = nullptr;
     w.packX = nullptr;
+    w.partial_tiles = nullptr;
+    w.tickets = nullptr;
   }
   w.Gs = carve<float>(cur, DW);
   w.Gact = carve<float>(cur, DW);
@@ -81,10 +85,11 @@ int copy_out(Handle* h, float* g, float* p, float* w, float* q, int32_t* idxA, i
 }
 
 // dW over the rows the sampler kept (idxW / scaleW / counts[1]) into `out`
-int sampled_dw(Handle* h, const void* X, const void* dY, float* out, cudaStream_t st) {
+int sampled_dw(Handle* h, const void* X, const void* dY, float keep_hint, float* out, cudaStream_t st) {
   if (h->tensor_path) {
     VCAS_CUDA(launch_pack(h, dY, X, st));
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, out, st));
+    const int hint = (int)(keep_hint * (float)(h->desc.N * h->desc.T)) + 1;
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, out, st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, out, st));
   }
@@ -101,7 +106,7 @@ inline void mark_dense(Handle* h, int k, cudaStream_t st) {
 
 int dense_dw(Handle* h, const void* X, const void* dY, float* out, cudaStream_t st) {
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, out, st));
+    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, h->desc.N * h->desc.T, out, st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, nullptr, nullptr, h->ws.counts + 2, out, st));
   }
@@ -148,13 +153,14 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->ev = nullptr;
   h->ev_dense = nullptr;
   h->prof_calls = h->prof_dense_calls = 0;
-  h->tune_dx_tile_n = h->tune_dw_tile_n = h->tune_dx_split_k = 0;
+  h->tune_dx_tile_n = h->tune_dw_tile_n = h->tune_dx_split_k = h->tune_dw_split_k = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&h->device) != cudaSuccess || cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
     delete h;
     return VCAS_ERR_CUDA;
   }
   h->num_sms = prop.multiProcessorCount;
+  h->max_units = 2 * h->num_sms;
   if (h->tensor_path && prop.major != 10) { delete h; return VCAS_ERR_CUDA; }
   h->bytes = layout(h, nullptr);
   if (cudaMalloc(&h->base, h->bytes) != cudaSuccess) {
@@ -224,7 +230,8 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   if (h->tensor_path) {
     VCAS_CUDA(launch_pack(h, dY, X, st));
     mark(h, 4, st);
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, dW, st));
+    const int hint = (int)(rho * nu * (float)(h->desc.N * h->desc.T)) + 1;
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, st));
   } else {
     mark(h, 4, st);
     VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, dW, st));
@@ -311,7 +318,7 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
       a.seed = seed + (uint64_t)(i * M + j + 1) * 0x9E3779B97F4A7C15ull;
       VCAS_CUDA(launch_sampler(h, a, st));
       if (j == 0) VCAS_CUDA(launch_probe_sparsity(h, s_lo, s_hi, st));
-      rc = sampled_dw(h, X_i[i], dY_i[i], h->ws.Gact, st);          // G_act,ij (SampleA only)
+      rc = sampled_dw(h, X_i[i], dY_i[i], rho, h->ws.Gact, st);          // G_act,ij (SampleA only)
       if (rc != VCAS_OK) return rc;
       VCAS_CUDA(launch_probe_sqdiff(h, st));
     }
@@ -354,14 +361,16 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
   return VCAS_OK;
 }
 
-int vcas_set_tuning(vcas_handle hh, int32_t dx_tile_n, int32_t dw_tile_n, int32_t dx_split_k) {
+int vcas_set_tuning(vcas_handle hh, int32_t dx_tile_n, int32_t dw_tile_n, int32_t dx_split_k, int32_t dw_split_k) {
   if (hh == nullptr) return VCAS_ERR_BAD_ARG;
   auto tile_ok = [](int32_t t) { return t == 0 || t == 64 || t == 128 || t == 256; };
-  if (!tile_ok(dx_tile_n) || !tile_ok(dw_tile_n) || dx_split_k < 0 || dx_split_k > 16) return VCAS_ERR_BAD_ARG;
+  if (!tile_ok(dx_tile_n) || !tile_ok(dw_tile_n) || dx_split_k < 0 || dx_split_k > 16 ||
+      dw_split_k < 0 || dw_split_k > 16) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   h->tune_dx_tile_n = dx_tile_n;
   h->tune_dw_tile_n = dw_tile_n;
   h->tune_dx_split_k = dx_split_k;
+  h->tune_dw_split_k = dw_split_k;
   return VCAS_OK;
 }
 

@@ -33,6 +33,8 @@ struct Workspace {
   // compact operands of the weight-gradient product (tensor path)
   __nv_bfloat16* packG;  // [R_pad, d_out]
   __nv_bfloat16* packX;  // [R_pad, d_in]
+  float* partial_tiles;  // [max_units][128 * 256] fp32 partial tiles of a split contraction
+  int32_t* tickets;      // [2 * max_units]: slices stored, slices finished, per tile
   // probe buffers (App. D: the exact gradient, its running mean and running squared deviation)
   float* Gs;       // [d_out, d_in]
   float* Gact;     // [d_out, d_in]
@@ -49,6 +51,7 @@ struct Handle {
   int num_sms;
   bool tensor_path;
   int R_pad;
+  int max_units;   // capacity of the split-contraction workspace, in (tile, slice) units
   void* base;
   size_t bytes;
   Workspace ws;
@@ -59,7 +62,7 @@ struct Handle {
   cudaEvent_t* ev_dense;  // [PROF_RING][3]: boundaries of dense dX | dense dW
   int prof_calls, prof_dense_calls;
   // tuning overrides (vcas_set_tuning); 0 = choose automatically
-  int tune_dx_tile_n, tune_dw_tile_n, tune_dx_split_k;
+  int tune_dx_tile_n, tune_dw_tile_n, tune_dx_split_k, tune_dw_split_k;
 };
 constexpr int PROF_RING = 2048;
 
@@ -131,8 +134,9 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
                            const void* H, void* dX, cudaStream_t st);
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
+// cnt_hint: the expected *cnt, used on the host to pick the tiling
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity,
-                           const int32_t* cnt, float* dW, cudaStream_t st);
+                           const int32_t* cnt, int cnt_hint, float* dW, cudaStream_t st);
 
 // probe reductions
 cudaError_t launch_probe_reset(Handle* h, cudaStream_t st);

@@ -5,8 +5,10 @@
 // are read from device memory.  Per CTA: warps 0-3 are the epilogue (TMEM -> registers ->
 // global), warp 4 issues TMA loads into a ring of shared-memory stages, warp 5 issues
 // tcgen05.mma into one of two TMEM accumulators, so the epilogue of a tile overlaps the main
-// loop of the next one.  bf16 operands, fp32 accumulation.  Every mbarrier wait is bounded:
-// when it runs out the CTA records VCAS_ERR_TIMEOUT in the status word and leaves.
+// loop of the next one.  bf16 operands, fp32 accumulation.  Outputs leave through 128-byte-swizzled
+// shared-memory staging and TMA / bulk stores.  A contraction can be cut into slices worked on by
+// neighbouring CTAs; the slices are added in a fixed order.  Every wait (mbarrier or sibling
+// CTA) is bounded: when it runs out the CTA records VCAS_ERR_TIMEOUT in the status word and leaves.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -22,12 +24,14 @@ constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN chunk of an MN-majo
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+constexpr int EPI_WARP_BYTES = 32 * 128;                // one staging buffer: 32 rows of 128 bytes, 128B-swizzled
+constexpr int EPI_BYTES = 4 * 2 * EPI_WARP_BYTES;       // two buffers for each of the four epilogue warps
 
 template <int BN> struct TileCfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + EPI_BYTES + 256 /*barriers*/;
 };
 
 // --------------------------------------------------------------------------- PTX wrappers
@@ -87,6 +91,25 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, i
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
 }
+
+// ---- asynchronous bulk stores (shared -> global), tracked in per-thread bulk groups
+__device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(ssrc)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* ssrc, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(smem_u32(ssrc)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* ssrc, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(smem_u32(ssrc)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// at most one group of this thread may still be READING its shared-memory source
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// all groups of this thread are complete (their global writes are performed)
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -153,6 +176,8 @@ struct SmemLayout {
   uint64_t* tmem_empty;
   uint32_t* tmem_holder;
   int* abort_flag;
+  int* flag;          // epilogue broadcast slot
+  uint8_t* epi;       // [4 warps][2][32 rows][128 B] staging for bulk / TMA stores
 };
 
 template <int BN>
@@ -161,13 +186,15 @@ __device__ __forceinline__ SmemLayout carve(uint8_t* raw) {
   SmemLayout s;
   uint8_t* base = (uint8_t*)(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
   s.stages = base;
-  uint64_t* bars = (uint64_t*)(base + C::STAGES * C::STAGE_BYTES);
+  s.epi = base + C::STAGES * C::STAGE_BYTES;                       // 1024-byte aligned (swizzle atom)
+  uint64_t* bars = (uint64_t*)(s.epi + EPI_BYTES);
   s.full = bars;
   s.empty = bars + C::STAGES;
   s.tmem_full = bars + 2 * C::STAGES;
   s.tmem_empty = bars + 2 * C::STAGES + 2;
   s.tmem_holder = (uint32_t*)(bars + 2 * C::STAGES + 4);
   s.abort_flag = (int*)(s.tmem_holder + 1);
+  s.flag = s.abort_flag + 1;
   return s;
 }
 
@@ -198,223 +225,152 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// ------------------------------------------------------------------------------ dX kernel
-struct DxParams {
+// ----------------------------------------------------------------------- the two products
+// One kernel template serves both products; MODE selects operand staging and the epilogue.
+//
+// Work decomposition (all derived on the device from the kept counts): `gemm_tiles` output
+// tiles, each cut along the contraction into S slices of kb_per k-blocks -> units; a unit is
+// (tile, slice).  With S > 1 every unit stores its fp32 partial tile to the workspace and takes a
+// ticket on its tile; when all S tickets are in, each of the S units adds the S partials of its
+// share of the tile's rows in slice order (a fixed order: results do not depend on timing) and
+// writes that share of the output.
+constexpr int MODE_DX = 0, MODE_DW = 1;
+
+struct GemmParams {
+  int32_t* status;
+  float* partial;          // [max_units][128 * BN] fp32 partial tiles (split contraction)
+  int32_t* tickets;        // [2 * max_units]: slices stored / slices finished per tile; zero between launches
+  int split_k;             // slices requested by the host
+  int max_units;
+  int d_in, d_out;
+  // dX: A = dY viewed [N][T][d_out] (K-major, one TMA box = 128 tokens x 64 k of one datum),
+  //     B = W [d_out][d_in] (MN-major: n contiguous)
   const int32_t* idxA;     // kept data
   const int32_t* dropA;    // dropped data
   const int32_t* counts;   // counts[0] = number of kept data
   const float* scaleA;     // 1/p_n per datum
   const __nv_bfloat16* H;  // optional GELU pre-activation [R, d_in]
   __nv_bfloat16* dX;       // [R, d_in]
-  int32_t* status;
-  int N, T, d_in, d_out;
+  int N, T;
   int dense;               // 1: every datum kept with scale 1
   int a_tx_bytes;          // bytes one A box delivers (min(T, 128) token rows of 128 B)
+  // dW: A = rows x d_out, B = rows x d_in (both MN-major, gathered along k by the pack step)
+  const int32_t* cnt;      // number of valid rows (the contraction length)
+  float* dW;               // [d_out, d_in]
 };
 
-// A = dY viewed [N][T][d_out] (K-major, one TMA box = 128 tokens x 64 k of one datum),
-// B = W [d_out][d_in] (MN-major: n contiguous), D = 128 x BN fp32 in TMEM.
-template <int BN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
-umma_dx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, DxParams P) {
-  using C = TileCfg<BN>;
-  extern __shared__ uint8_t smem_raw[];
-  const SmemLayout s = carve<BN>(smem_raw);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t tmem_base = setup<BN>(s, warp, tid);
-  volatile int* abort_flag = s.abort_flag;
+struct Decomp {
+  int gemm_tiles, zero_tiles, kblocks, S, kb_per, units;
+  int upi;                 // units taken per pass of the grid: a multiple of S, so that the S slices of a tile
+                           // are always worked on at the same time by S neighbouring CTAs
+  int per_datum, ntiles;   // dX: tiles per datum; both: column tiles
+};
 
-  const int cntA = P.dense ? P.N : P.counts[0];
-  const int chunks = (P.T + BM - 1) / BM;
-  const int ntiles = (P.d_in + BN - 1) / BN;
-  const int per_datum = chunks * ntiles;
-  const int gemm_tiles = cntA * per_datum;
-  const int total_tiles = P.N * per_datum;
-  const int kblocks = (P.d_out + BK - 1) / BK;
-
-  if (warp == 4) {
-    if (lane == 0) {
-      int stage = 0; uint32_t phase = 0;
-      for (int tile = blockIdx.x; tile < gemm_tiles; tile += gridDim.x) {
-        const int k = tile / per_datum, rem = tile % per_datum;
-        const int c = rem / ntiles, nt = rem % ntiles;
-        const int n = P.dense ? k : P.idxA[k];
-        bool ok = true;
-        for (int kb = 0; kb < kblocks && ok; ++kb) {
-          ok = mbar_wait(&s.empty[stage], phase ^ 1u, abort_flag, P.status);
-          if (!ok) break;
-          uint8_t* sa = s.stages + stage * C::STAGE_BYTES;
-          mbar_expect_tx(&s.full[stage], (uint32_t)(P.a_tx_bytes + C::B_BYTES));
-          tma_load_3d(sa, &tmA, kb * BK, c * BM, n, &s.full[stage]);
-#pragma unroll
-          for (int j = 0; j < BN / 64; ++j)
-            tma_load_2d(sa + A_BYTES + j * CHUNK_BYTES, &tmB, nt * BN + j * 64, kb * BK, &s.full[stage]);
-          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
-        }
-        if (!ok) break;
-      }
-    }
-  } else if (warp == 5) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(BN, false, true);
-      int stage = 0; uint32_t phase = 0; int lt = 0;
-      for (int tile = blockIdx.x; tile < gemm_tiles; tile += gridDim.x, ++lt) {
-        const int buf = lt & 1; const uint32_t use = (uint32_t)(lt >> 1) & 1u;
-        bool ok = mbar_wait(&s.tmem_empty[buf], use ^ 1u, abort_flag, P.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-        for (int kb = 0; kb < kblocks; ++kb) {
-          ok = mbar_wait(&s.full[stage], phase, abort_flag, P.status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t sa = smem_u32(s.stages + stage * C::STAGE_BYTES);
-          const uint64_t da = desc_kmajor(sa), db = desc_mnmajor(sa + A_BYTES);
-#pragma unroll
-          for (int k4 = 0; k4 < BK / UMMA_K; ++k4)
-            umma_bf16(d_tmem, da + (uint64_t)(k4 * (UMMA_K * 2 >> 4)), db + (uint64_t)(k4 * (UMMA_K * 128 >> 4)), idesc,
-                      (kb | k4) != 0 ? 1u : 0u);
-          umma_commit(&s.empty[stage]);
-          if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
-        }
-        if (!ok) break;
-        umma_commit(&s.tmem_full[buf]);
-      }
-    }
+template <int MODE, int BN>
+__device__ __forceinline__ Decomp decompose(const GemmParams& P) {
+  Decomp d;
+  d.ntiles = (P.d_in + BN - 1) / BN;
+  if (MODE == MODE_DX) {
+    const int cntA = P.dense ? P.N : P.counts[0];
+    d.per_datum = ((P.T + BM - 1) / BM) * d.ntiles;
+    d.gemm_tiles = cntA * d.per_datum;
+    d.zero_tiles = (P.N - cntA) * d.per_datum;
+    d.kblocks = (P.d_out + BK - 1) / BK;
   } else {
-    // epilogue: thread (warp, lane) owns accumulator lane warp*32 + lane = tile row
-    int lt = 0;
-    const int row = warp * 32 + lane;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const bool is_gemm = tile < gemm_tiles;
-      const int t2 = is_gemm ? tile : tile - gemm_tiles;
-      const int k = t2 / per_datum, rem = t2 % per_datum;
-      const int c = rem / ntiles, nt = rem % ntiles;
-      const int n = is_gemm ? (P.dense ? k : P.idxA[k]) : P.dropA[k];
-      const int t = c * BM + row;
-      const bool valid = t < P.T;
-      const size_t off = ((size_t)n * P.T + (valid ? t : 0)) * P.d_in + (size_t)nt * BN;
-      __nv_bfloat16* out = P.dX + off;
-      if (!is_gemm) {
-        if (valid) {
-#pragma unroll
-          for (int j = 0; j < BN / 8; ++j)
-            if (nt * BN + j * 8 < P.d_in) *reinterpret_cast<uint4*>(out + j * 8) = make_uint4(0u, 0u, 0u, 0u);
-        }
-        continue;
-      }
-      const int buf = lt & 1; const uint32_t use = (uint32_t)(lt >> 1) & 1u;
-      ++lt;
-      if (!mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status)) break;
-      tc_fence_after();
-      const float sc = P.dense ? 1.0f : P.scaleA[n];
-      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * BN);
-#pragma unroll 1
-      for (int j = 0; j < BN / 32; ++j) {
-        uint32_t v[32];
-        tmem_ld32(taddr + (uint32_t)(j * 32), v);
-        if (valid) {
-#pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            const int col = nt * BN + j * 32 + g8 * 8;
-            if (col < P.d_in) {
-              float f[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) f[e] = sc * __uint_as_float(v[g8 * 8 + e]);
-              if (P.H != nullptr) {
-                const uint4 hv = *reinterpret_cast<const uint4*>(P.H + off + j * 32 + g8 * 8);
-                const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  f[2 * e] *= gelu_prime(__uint_as_float(hu[e] << 16));
-                  f[2 * e + 1] *= gelu_prime(__uint_as_float(hu[e] & 0xffff0000u));
-                }
-              }
-              uint4 o;
-              o.x = pack_bf16(f[0], f[1]); o.y = pack_bf16(f[2], f[3]);
-              o.z = pack_bf16(f[4], f[5]); o.w = pack_bf16(f[6], f[7]);
-              *reinterpret_cast<uint4*>(out + j * 32 + g8 * 8) = o;
-            }
-          }
-        }
-      }
-      tc_fence_before();
-      mbar_arrive(&s.tmem_empty[buf]);
-    }
+    d.per_datum = 0;
+    const int tiles = ((P.d_out + BM - 1) / BM) * d.ntiles;
+    d.kblocks = (*P.cnt + BK - 1) / BK;
+    d.gemm_tiles = d.kblocks > 0 ? tiles : 0;   // nothing kept: every tile is a zero tile
+    d.zero_tiles = d.kblocks > 0 ? 0 : tiles;
   }
-  __syncwarp();
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
+  int S = P.split_k < 1 ? 1 : P.split_k;
+  if (S > d.kblocks) S = d.kblocks > 0 ? d.kblocks : 1;
+  if (d.gemm_tiles > 0 && (long)d.gemm_tiles * S > P.max_units) S = P.max_units / d.gemm_tiles;
+  if (S > (int)gridDim.x) S = (int)gridDim.x;
+  if (S < 1) S = 1;
+  d.kb_per = d.kblocks > 0 ? (d.kblocks + S - 1) / S : 0;
+  d.S = d.kb_per > 0 ? (d.kblocks + d.kb_per - 1) / d.kb_per : 1;   // every slice non-empty
+  d.units = d.gemm_tiles * d.S;
+  d.upi = ((int)gridDim.x / d.S) * d.S;
+  return d;
 }
 
-// ------------------------------------------------------------------------------ dW kernel
-struct DwParams {
-  const int32_t* cnt;   // number of valid rows (the contraction length)
-  float* dW;            // [d_out, d_in]
-  int32_t* status;
-  int d_in, d_out;
-};
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// A = rows x d_out (MN-major: m contiguous), B = rows x d_in (MN-major), both gathered along k
-// by the pack step (or the original tensors for the dense product).
-template <int BN>
+template <int MODE, int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-umma_dw_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, DwParams P) {
+umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmC, GemmParams P) {
   using C = TileCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const SmemLayout s = carve<BN>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t tmem_base = setup<BN>(s, warp, tid);
   volatile int* abort_flag = s.abort_flag;
-
-  const int cnt = *P.cnt;
-  const int kblocks = (cnt + BK - 1) / BK;
-  const int mtiles = (P.d_out + BM - 1) / BM;
-  const int ntiles = (P.d_in + BN - 1) / BN;
-  const int total_tiles = mtiles * ntiles;
+  const Decomp D = decompose<MODE, BN>(P);
 
   if (warp == 4) {
-    if (lane == 0 && kblocks > 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int mt = tile / ntiles, nt = tile % ntiles;
-        bool ok = true;
-        for (int kb = 0; kb < kblocks; ++kb) {
+      bool ok = true;
+      for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi) {
+        const int tile = u / D.S, slice = u % D.S;
+        const int kb0 = slice * D.kb_per;
+        const int kb1 = min(D.kblocks, kb0 + D.kb_per);
+        int c0 = 0, c1 = 0, n = 0;   // dX: token chunk, column tile, datum; dW: row tile, column tile
+        if (MODE == MODE_DX) {
+          const int k = tile / D.per_datum, rem = tile % D.per_datum;
+          c0 = rem / D.ntiles; c1 = rem % D.ntiles;
+          n = P.dense ? k : P.idxA[k];
+        } else {
+          c0 = tile / D.ntiles; c1 = tile % D.ntiles;
+        }
+        for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(&s.empty[stage], phase ^ 1u, abort_flag, P.status);
           if (!ok) break;
           uint8_t* sa = s.stages + stage * C::STAGE_BYTES;
-          mbar_expect_tx(&s.full[stage], C::STAGE_BYTES);
+          if (MODE == MODE_DX) {
+            mbar_expect_tx(&s.full[stage], (uint32_t)(P.a_tx_bytes + C::B_BYTES));
+            tma_load_3d(sa, &tmA, kb * BK, c0 * BM, n, &s.full[stage]);
+          } else {
+            mbar_expect_tx(&s.full[stage], C::STAGE_BYTES);
 #pragma unroll
-          for (int j = 0; j < BM / 64; ++j)
-            tma_load_2d(sa + j * CHUNK_BYTES, &tmA, mt * BM + j * 64, kb * BK, &s.full[stage]);
+            for (int j = 0; j < BM / 64; ++j)
+              tma_load_2d(sa + j * CHUNK_BYTES, &tmA, c0 * BM + j * 64, kb * BK, &s.full[stage]);
+          }
 #pragma unroll
           for (int j = 0; j < BN / 64; ++j)
-            tma_load_2d(sa + A_BYTES + j * CHUNK_BYTES, &tmB, nt * BN + j * 64, kb * BK, &s.full[stage]);
+            tma_load_2d(sa + A_BYTES + j * CHUNK_BYTES, &tmB, c1 * BN + j * 64, kb * BK, &s.full[stage]);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (!ok) break;
       }
     }
   } else if (warp == 5) {
-    if (lane == 0 && kblocks > 0) {
-      constexpr uint32_t idesc = make_idesc(BN, true, true);
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BN, MODE == MODE_DW, true);
+      constexpr uint32_t a_step = MODE == MODE_DW ? (UMMA_K * 128 >> 4) : (UMMA_K * 2 >> 4);
       int stage = 0; uint32_t phase = 0; int lt = 0;
-      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
+      bool ok = true;
+      for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi, ++lt) {
+        const int slice = u % D.S;
+        const int nkb = min(D.kblocks, (slice + 1) * D.kb_per) - slice * D.kb_per;
         const int buf = lt & 1; const uint32_t use = (uint32_t)(lt >> 1) & 1u;
-        bool ok = mbar_wait(&s.tmem_empty[buf], use ^ 1u, abort_flag, P.status);
+        ok = mbar_wait(&s.tmem_empty[buf], use ^ 1u, abort_flag, P.status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-        for (int kb = 0; kb < kblocks; ++kb) {
+        for (int kb = 0; kb < nkb; ++kb) {
           ok = mbar_wait(&s.full[stage], phase, abort_flag, P.status);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(s.stages + stage * C::STAGE_BYTES);
-          const uint64_t da = desc_mnmajor(sa), db = desc_mnmajor(sa + A_BYTES);
+          const uint64_t da = MODE == MODE_DW ? desc_mnmajor(sa) : desc_kmajor(sa);
+          const uint64_t db = desc_mnmajor(sa + A_BYTES);
 #pragma unroll
           for (int k4 = 0; k4 < BK / UMMA_K; ++k4)
-            umma_bf16(d_tmem, da + (uint64_t)(k4 * (UMMA_K * 128 >> 4)), db + (uint64_t)(k4 * (UMMA_K * 128 >> 4)), idesc,
+            umma_bf16(d_tmem, da + (uint64_t)(k4 * a_step), db + (uint64_t)(k4 * (UMMA_K * 128 >> 4)), idesc,
                       (kb | k4) != 0 ? 1u : 0u);
           umma_commit(&s.empty[stage]);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -424,40 +380,247 @@ umma_dw_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
-    int lt = 0;
+    // -------------------------------------------------------------------- epilogue
+    // thread (warp, lane) owns accumulator lane warp*32 + lane = tile row
     const int row = warp * 32 + lane;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
-      const int mt = tile / ntiles, nt = tile % ntiles;
-      const int o = mt * BM + row;
-      const bool valid = o < P.d_out;
-      float* out = P.dW + (size_t)(valid ? o : 0) * P.d_in + (size_t)nt * BN;
-      if (kblocks == 0) {
-        if (valid) {
-#pragma unroll
-          for (int j = 0; j < BN / 4; ++j)
-            if (nt * BN + j * 4 < P.d_in) *reinterpret_cast<float4*>(out + j * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        continue;
+    const size_t ld = (size_t)P.d_in;
+    // output rows [row0, row0 + rows_valid) x columns [col0, col0 + BN) of the tile; sc = 1/p_n
+    auto geometry = [&](int tile, bool is_gemm, size_t& row0, int& rows_valid, int& col0, float& sc, int& n_out,
+                        int& t_out) {
+      sc = 1.0f; n_out = 0; t_out = 0;
+      if (MODE == MODE_DX) {
+        const int k = tile / D.per_datum, rem = tile % D.per_datum;
+        const int c = rem / D.ntiles, nt = rem % D.ntiles;
+        const int n = is_gemm ? (P.dense ? k : P.idxA[k]) : P.dropA[k];
+        row0 = (size_t)n * P.T + (size_t)c * BM;
+        rows_valid = min(BM, P.T - c * BM);
+        col0 = nt * BN;
+        n_out = n; t_out = c * BM;
+        if (is_gemm && !P.dense) sc = P.scaleA[n];
+      } else {
+        const int mt = tile / D.ntiles, nt = tile % D.ntiles;
+        row0 = (size_t)mt * BM;
+        rows_valid = min(BM, P.d_out - mt * BM);
+        col0 = nt * BN;
       }
+    };
+    // finishes 8 consecutive columns of one output row: rescale, optional GELU', convert, store
+    auto store8 = [&](size_t off, float sc, const float* f) {
+      if (MODE == MODE_DX) {
+        float r[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) r[e] = sc * f[e];
+        if (P.H != nullptr) {
+          const uint4 hv = *reinterpret_cast<const uint4*>(P.H + off);
+          const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            r[2 * e] *= gelu_prime(__uint_as_float(hu[e] << 16));
+            r[2 * e + 1] *= gelu_prime(__uint_as_float(hu[e] & 0xffff0000u));
+          }
+        }
+        uint4 o;
+        o.x = pack_bf16(r[0], r[1]); o.y = pack_bf16(r[2], r[3]);
+        o.z = pack_bf16(r[4], r[5]); o.w = pack_bf16(r[6], r[7]);
+        *reinterpret_cast<uint4*>(P.dX + off) = o;
+      } else {
+        *reinterpret_cast<float4*>(P.dW + off) = make_float4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<float4*>(P.dW + off + 4) = make_float4(f[4], f[5], f[6], f[7]);
+      }
+    };
+
+    uint8_t* stage0 = s.epi + warp * (2 * EPI_WARP_BYTES);       // this warp's two staging buffers
+    const uint32_t swz = (uint32_t)(lane & 7);                   // 128-byte swizzle: 16-byte slot ^= row & 7
+    int lt = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi, ++lt) {
+      const int tile = u / D.S, slice = u % D.S;
+      size_t row0; int rows_valid, col0, n_out, t_out; float sc;
+      geometry(tile, true, row0, rows_valid, col0, sc, n_out, t_out);
       const int buf = lt & 1; const uint32_t use = (uint32_t)(lt >> 1) & 1u;
       if (!mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * BN);
+      if (D.S == 1) {
+        // ---- whole contraction in this unit: accumulator -> (rescale, GELU', convert) -> swizzled
+        // shared memory -> TMA store of 32 rows x 128 bytes per warp (rows / columns outside the
+        // tensor are clipped by the tensor map, so rows of the next datum are never touched)
+        const bool valid = row < rows_valid;
+        constexpr int COLS = MODE == MODE_DX ? 64 : 32;             // columns per 128-byte staged row
+        int nbuf = 0;
+#pragma unroll 1
+        for (int j = 0; j < BN / COLS; ++j, ++nbuf) {
+          if (col0 + j * COLS >= P.d_in) break;                     // warp-uniform
+          uint8_t* buf8 = stage0 + (nbuf & 1) * EPI_WARP_BYTES;
+          if (nbuf >= 2) { if (lane == 0) bulk_wait_read_1(); __syncwarp(); }
+          uint4* myrow = reinterpret_cast<uint4*>(buf8 + lane * 128);
+          if (MODE == MODE_DX) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              uint32_t v[32];
+              tmem_ld32(taddr + (uint32_t)(j * 64 + half * 32), v);
+#pragma unroll
+              for (int g8 = 0; g8 < 4; ++g8) {
+                float r[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) r[e] = sc * __uint_as_float(v[g8 * 8 + e]);
+                if (P.H != nullptr && valid) {
+                  const size_t off = (row0 + row) * ld + col0 + j * 64 + half * 32 + g8 * 8;
+                  const uint4 hv = *reinterpret_cast<const uint4*>(P.H + off);
+                  const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    r[2 * e] *= gelu_prime(__uint_as_float(hu[e] << 16));
+                    r[2 * e + 1] *= gelu_prime(__uint_as_float(hu[e] & 0xffff0000u));
+                  }
+                }
+                uint4 o;
+                o.x = pack_bf16(r[0], r[1]); o.y = pack_bf16(r[2], r[3]);
+                o.z = pack_bf16(r[4], r[5]); o.w = pack_bf16(r[6], r[7]);
+                myrow[(uint32_t)(half * 4 + g8) ^ swz] = o;
+              }
+            }
+          } else {
+            uint32_t v[32];
+            tmem_ld32(taddr + (uint32_t)(j * 32), v);
+#pragma unroll
+            for (int g4 = 0; g4 < 8; ++g4)
+              myrow[(uint32_t)g4 ^ swz] = make_uint4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (MODE == MODE_DX) tma_store_3d(&tmC, buf8, col0 + j * 64, t_out + warp * 32, n_out);
+            else tma_store_2d(&tmC, buf8, col0 + j * 32, (int)row0 + warp * 32);
+            bulk_commit();
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(&s.tmem_empty[buf]);
+        if (lane == 0) bulk_wait_all();        // staging buffers are reused by the next unit
+        __syncwarp();
+        continue;
+      }
+      // ---- one slice of the contraction: store the fp32 partial tile.  Layout in the workspace:
+      // [32-column chunk][row][32 floats], the eight 16-byte slots of a row swizzled by (row & 7) as
+      // staged in shared memory, so each warp moves its 32 rows of a chunk with one 4 KB bulk copy.
+      float* part = P.partial + (size_t)u * (BM * BN);
 #pragma unroll 1
       for (int j = 0; j < BN / 32; ++j) {
+        if (col0 + j * 32 >= P.d_in) break;                         // warp-uniform
+        uint8_t* buf8 = stage0 + (j & 1) * EPI_WARP_BYTES;
+        if (j >= 2) { if (lane == 0) bulk_wait_read_1(); __syncwarp(); }
         uint32_t v[32];
         tmem_ld32(taddr + (uint32_t)(j * 32), v);
-        if (valid) {
+        uint4* myrow = reinterpret_cast<uint4*>(buf8 + lane * 128);
 #pragma unroll
-          for (int g4 = 0; g4 < 8; ++g4) {
-            const int col = nt * BN + j * 32 + g4 * 4;
-            if (col < P.d_in)
-              *reinterpret_cast<uint4*>(out + j * 32 + g4 * 4) = make_uint4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
-          }
+        for (int g4 = 0; g4 < 8; ++g4)
+          myrow[(uint32_t)g4 ^ swz] = make_uint4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          bulk_store(part + (size_t)j * (BM * 32) + (size_t)(warp * 32) * 32, buf8, EPI_WARP_BYTES);
+          bulk_commit();
         }
       }
       tc_fence_before();
-      mbar_arrive(&s.tmem_empty[buf]);
+      mbar_arrive(&s.tmem_empty[buf]);          // the accumulator is free again
+      if (lane == 0) bulk_wait_all();           // this warp's part of the partial tile is in global memory
+      __syncwarp();
+      // ... announce it, wait (bounded) until all S slices of the tile are stored ...
+      __threadfence();
+      epi_bar();
+      if (tid == 0) {
+        atomicAdd(&P.tickets[tile], 1);
+        unsigned long long t0 = 0; uint32_t spins = 0; int good = 1;
+        while (*(volatile int32_t*)&P.tickets[tile] < D.S) {
+          if ((++spins & 0xffu) == 0) {
+            if (*abort_flag) { good = 0; break; }
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; atomicExch(P.status, (int32_t)VCAS_ERR_TIMEOUT); good = 0; break; }
+          }
+        }
+        *s.flag = good;
+      }
+      epi_bar();
+      ok = *(volatile int*)s.flag != 0;
+      if (!ok) break;
+      __threadfence();
+      // ... then add the S partials of this unit's share of the rows, in slice order, and write the output.
+      {
+        const int rows_per = (BM + D.S - 1) / D.S;
+        const int r_begin = slice * rows_per;
+        const int r_end = min(min(BM, r_begin + rows_per), rows_valid);
+        const int c8n = min(BN, P.d_in - col0) / 8;               // 8-column groups per row inside the tensor
+        const int n_items = max(0, r_end - r_begin) * c8n;
+        const float* tile_part = P.partial + (size_t)(tile * D.S) * (BM * BN);
+        // element offset of the 8 columns (r, c8*8 ..) inside a partial tile: chunk, row, swizzled slots
+        auto slot_off = [&](int r, int c8, int half) {
+          const int slot = ((c8 & 3) * 2 + half) ^ (r & 7);
+          return (size_t)(c8 >> 2) * (BM * 32) + (size_t)r * 32 + (size_t)slot * 4;
+        };
+        for (int it0 = tid; it0 < n_items; it0 += 256) {
+          // two items per thread in flight
+          const int it1 = it0 + 128;
+          const bool has1 = it1 < n_items;
+          const int ra = r_begin + it0 / c8n, ca = it0 % c8n;
+          const int rb = has1 ? r_begin + it1 / c8n : ra, cb = has1 ? it1 % c8n : ca;
+          const size_t oa0 = slot_off(ra, ca, 0), oa1 = slot_off(ra, ca, 1);
+          const size_t ob0 = slot_off(rb, cb, 0), ob1 = slot_off(rb, cb, 1);
+          float fa[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          float fb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          for (int sl0 = 0; sl0 < D.S; sl0 += 2) {               // slices in order, two at a time in flight
+            float4 x[2][4];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const int sl = min(sl0 + q, D.S - 1);
+              const float* base = tile_part + (size_t)sl * (BM * BN);
+              x[q][0] = __ldcg(reinterpret_cast<const float4*>(base + oa0));
+              x[q][1] = __ldcg(reinterpret_cast<const float4*>(base + oa1));
+              x[q][2] = __ldcg(reinterpret_cast<const float4*>(base + ob0));
+              x[q][3] = __ldcg(reinterpret_cast<const float4*>(base + ob1));
+            }
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              if (sl0 + q < D.S) {
+                fa[0] += x[q][0].x; fa[1] += x[q][0].y; fa[2] += x[q][0].z; fa[3] += x[q][0].w;
+                fa[4] += x[q][1].x; fa[5] += x[q][1].y; fa[6] += x[q][1].z; fa[7] += x[q][1].w;
+                fb[0] += x[q][2].x; fb[1] += x[q][2].y; fb[2] += x[q][2].z; fb[3] += x[q][2].w;
+                fb[4] += x[q][3].x; fb[5] += x[q][3].y; fb[6] += x[q][3].z; fb[7] += x[q][3].w;
+              }
+            }
+          }
+          store8((row0 + ra) * ld + col0 + ca * 8, sc, fa);
+          if (has1) store8((row0 + rb) * ld + col0 + cb * 8, sc, fb);
+        }
+      }
+      epi_bar();
+      if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(&P.tickets[P.max_units + tile], 1) == D.S - 1) {   // last slice done: reset for the next launch
+          P.tickets[tile] = 0;
+          P.tickets[P.max_units + tile] = 0;
+        }
+      }
+    }
+    // zero tiles (rows of dropped data; nothing kept at all): taken from the far end of the grid first,
+    // where CTAs have no product units
+    for (int z = (int)gridDim.x - 1 - (int)blockIdx.x; z < D.zero_tiles && ok; z += gridDim.x) {
+      size_t row0; int rows_valid, col0, n_out, t_out; float sc;
+      geometry(z, false, row0, rows_valid, col0, sc, n_out, t_out);
+      if (row < rows_valid) {
+        const size_t off = (row0 + row) * ld + col0;
+        if (MODE == MODE_DX) {
+#pragma unroll
+          for (int j = 0; j < BN / 8; ++j)
+            if (col0 + j * 8 < P.d_in) *reinterpret_cast<uint4*>(P.dX + off + j * 8) = make_uint4(0u, 0u, 0u, 0u);
+        } else {
+#pragma unroll
+          for (int j = 0; j < BN / 4; ++j)
+            if (col0 + j * 4 < P.d_in) *reinterpret_cast<uint4*>(P.dW + off + j * 4) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
     }
   }
   __syncwarp();
@@ -519,61 +682,84 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 tensor of `rank` dims (innermost first), 128-byte swizzle, out-of-bounds reads give 0
+// tensor of `rank` dims (innermost first), 128-byte swizzle; out-of-bounds reads give 0, out-of-bounds
+// parts of a store are dropped
 bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-              const uint32_t* box) {
+              const uint32_t* box, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t gd[3]; cuuint64_t gs[2]; cuuint32_t bx[3]; cuuint32_t es[3] = {1, 1, 1};
   for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; }
   for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
+  return fn(m, dtype, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tile width: fewest waves of the persistent grid, weighted by the per-tile cost of each width
-// (narrow tiles reuse the A stage less and run the tensor pipe below its peak rate).
-int pick_bn(long row_tiles, int n_extent, int num_sms) {
+// Tile width and number of contraction slices from a small cost model: waves of the persistent
+// grid x (k-blocks per unit x time per k-block + fixed cost per unit) + the cost of combining
+// slices.  Times per k-block were measured on B200 (about 0.5 / 0.45 / 0.43 us for 256 / 128 / 64
+// wide tiles: the shared-memory fill rate of one SM bounds them, so narrow tiles only pay off
+// when they fill more SMs).
+struct Plan { int bn, split; };
+Plan plan_tiles(long row_tiles, int n_extent, int kblocks, int num_sms, int max_units, int force_bn, int force_split) {
   const int widths[3] = {256, 128, 64};
-  const double cost[3] = {1.0, 0.56, 0.36};
-  int best = 256; double best_t = 1e30;
+  const double c_kb[3] = {0.50, 0.45, 0.43};
+  Plan best = {256, 1};
+  double best_t = 1e30;
+  if (kblocks < 1) kblocks = 1;
   for (int i = 0; i < 3; ++i) {
+    if (force_bn != 0 && widths[i] != force_bn) continue;
+    if (force_bn == 0 && widths[i] > 64 && n_extent <= widths[i] / 2) continue;   // mostly padding
     const long tiles = row_tiles * ((n_extent + widths[i] - 1) / widths[i]);
-    const double t = (double)((tiles + num_sms - 1) / num_sms) * cost[i];
-    if (t < best_t - 1e-9) { best_t = t; best = widths[i]; }
+    for (int sp = 1; sp <= 16; ++sp) {
+      if (force_split != 0 && sp != force_split) continue;
+      if (sp > 1 && tiles * sp > max_units) continue;
+      if (sp > 1 && force_split == 0 && kblocks / sp < 4) continue;   // slices too short to pay off
+      const long units = tiles * sp;
+      const double waves = (double)((units + num_sms - 1) / num_sms);
+      double t = waves * ((double)((kblocks + sp - 1) / sp) * c_kb[i] + 4.0);
+      if (sp > 1) t += 3.0 + 0.25 * sp;
+      if (t < best_t - 1e-9) { best_t = t; best = {widths[i], sp}; }
+    }
   }
   return best;
 }
 
-template <int BN>
-cudaError_t run_dx(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const DxParams& P, cudaStream_t st) {
+template <int MODE, int BN>
+cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P,
+                     long max_items, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(umma_dx_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<BN>::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         TileCfg<BN>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const long total = (long)P.N * ((P.T + BM - 1) / BM) * ((P.d_in + BN - 1) / BN);
-  const int grid = (int)(total < h->num_sms ? total : h->num_sms);
-  umma_dx_kernel<BN><<<grid, NUM_THREADS, TileCfg<BN>::SMEM_BYTES, st>>>(a, b, P);
+  const int grid = (int)(max_items < h->num_sms ? max_items : h->num_sms);
+  umma_kernel<MODE, BN><<<grid, NUM_THREADS, TileCfg<BN>::SMEM_BYTES, st>>>(a, b, c, P);
   h->launches += 1;
   return cudaGetLastError();
 }
 
-template <int BN>
-cudaError_t run_dw(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const DwParams& P, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(umma_dw_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<BN>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
+template <int MODE>
+cudaError_t run_gemm_bn(Handle* h, int bn, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
+                        const GemmParams& P, long max_items, cudaStream_t st) {
+  switch (bn) {
+    case 256: return run_gemm<MODE, 256>(h, a, b, c, P, max_items, st);
+    case 128: return run_gemm<MODE, 128>(h, a, b, c, P, max_items, st);
+    default: return run_gemm<MODE, 64>(h, a, b, c, P, max_items, st);
   }
-  const long total = (long)((P.d_out + BM - 1) / BM) * ((P.d_in + BN - 1) / BN);
-  const int grid = (int)(total < h->num_sms ? total : h->num_sms);
-  umma_dw_kernel<BN><<<grid, NUM_THREADS, TileCfg<BN>::SMEM_BYTES, st>>>(a, b, P);
-  h->launches += 1;
-  return cudaGetLastError();
+}
+
+void common_params(Handle* h, GemmParams& P) {
+  P = GemmParams();
+  P.status = h->ws.status;
+  P.partial = h->ws.partial_tiles;
+  P.tickets = h->ws.tickets;
+  P.max_units = h->max_units;
+  P.d_in = h->desc.d_in;
+  P.d_out = h->desc.d_out;
 }
 
 }  // namespace
@@ -581,7 +767,7 @@ cudaError_t run_dw(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const 
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint, const void* H,
                            void* dX, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmC;
   {
     const uint64_t dims[3] = {(uint64_t)d.d_out, (uint64_t)d.T, (uint64_t)d.N};
     const uint64_t strides[2] = {(uint64_t)d.d_out * 2, (uint64_t)d.T * d.d_out * 2};
@@ -594,19 +780,28 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
     const uint32_t box[2] = {64, BK};
     if (!make_map(&tmB, W, 2, dims, strides, box)) return cudaErrorInvalidValue;
   }
-  DxParams P;
+  {
+    const uint64_t dims[3] = {(uint64_t)d.d_in, (uint64_t)d.T, (uint64_t)d.N};
+    const uint64_t strides[2] = {(uint64_t)d.d_in * 2, (uint64_t)d.T * d.d_in * 2};
+    const uint32_t box[3] = {64, (uint32_t)(d.T < 32 ? d.T : 32), 1};
+    if (!make_map(&tmC, dX, 3, dims, strides, box)) return cudaErrorInvalidValue;
+  }
+  GemmParams P;
+  common_params(h, P);
   P.idxA = h->ws.idxA; P.dropA = h->ws.dropA; P.counts = h->ws.counts; P.scaleA = h->ws.scaleA;
-  P.H = (const __nv_bfloat16*)H; P.dX = (__nv_bfloat16*)dX; P.status = h->ws.status;
-  P.N = d.N; P.T = d.T; P.d_in = d.d_in; P.d_out = d.d_out; P.dense = dense ? 1 : 0;
+  P.H = (const __nv_bfloat16*)H; P.dX = (__nv_bfloat16*)dX;
+  P.N = d.N; P.T = d.T; P.dense = dense ? 1 : 0;
   P.a_tx_bytes = (d.T < BM ? d.T : BM) * BK * 2;
   double kept = dense ? (double)d.N : (double)rho_hint * d.N;
   if (kept < 1.0) kept = 1.0;
-  const long row_tiles = (long)(kept + 0.5) * ((d.T + BM - 1) / BM);
-  switch (h->tune_dx_tile_n != 0 ? h->tune_dx_tile_n : pick_bn(row_tiles, d.d_in, h->num_sms)) {
-    case 256: return run_dx<256>(h, tmA, tmB, P, st);
-    case 128: return run_dx<128>(h, tmA, tmB, P, st);
-    default: return run_dx<64>(h, tmA, tmB, P, st);
-  }
+  const int chunks = (d.T + BM - 1) / BM;
+  const long row_tiles = (long)(kept + 0.5) * chunks;
+  const Plan plan = plan_tiles(row_tiles, d.d_in, (d.d_out + BK - 1) / BK, h->num_sms, h->max_units,
+                               h->tune_dx_tile_n, h->tune_dx_split_k);
+  P.split_k = plan.split;
+  // upper bound of work items: every datum kept and split, or every datum a zero tile
+  const long max_items = (long)d.N * chunks * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
+  return run_gemm_bn<MODE_DX>(h, plan.bn, tmA, tmB, tmC, P, max_items, st);
 }
 
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st) {
@@ -620,9 +815,9 @@ cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t s
 }
 
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity, const int32_t* cnt,
-                           float* dW, cudaStream_t st) {
+                           int cnt_hint, float* dW, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmC;
   {
     const uint64_t dims[2] = {(uint64_t)d.d_out, (uint64_t)rows_capacity};
     const uint64_t strides[1] = {(uint64_t)d.d_out * 2};
@@ -635,13 +830,21 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
     const uint32_t box[2] = {64, BK};
     if (!make_map(&tmB, B_rows, 2, dims, strides, box)) return cudaErrorInvalidValue;
   }
-  DwParams P;
-  P.cnt = cnt; P.dW = dW; P.status = h->ws.status; P.d_in = d.d_in; P.d_out = d.d_out;
-  switch (h->tune_dw_tile_n != 0 ? h->tune_dw_tile_n : pick_bn((d.d_out + BM - 1) / BM, d.d_in, h->num_sms)) {
-    case 256: return run_dw<256>(h, tmA, tmB, P, st);
-    case 128: return run_dw<128>(h, tmA, tmB, P, st);
-    default: return run_dw<64>(h, tmA, tmB, P, st);
+  {
+    const uint64_t dims[2] = {(uint64_t)d.d_in, (uint64_t)d.d_out};
+    const uint64_t strides[1] = {(uint64_t)d.d_in * 4};
+    const uint32_t box[2] = {32, 32};
+    if (!make_map(&tmC, dW, 2, dims, strides, box, CU_TENSOR_MAP_DATA_TYPE_FLOAT32)) return cudaErrorInvalidValue;
   }
+  GemmParams P;
+  common_params(h, P);
+  P.cnt = cnt; P.dW = dW;
+  const long mtiles = (d.d_out + BM - 1) / BM;
+  const Plan plan = plan_tiles(mtiles, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
+                               h->tune_dw_tile_n, h->tune_dw_split_k);
+  P.split_k = plan.split;
+  const long max_items = mtiles * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
+  return run_gemm_bn<MODE_DW>(h, plan.bn, tmA, tmB, tmC, P, max_items, st);
 }
 
 }  // namespace vcas

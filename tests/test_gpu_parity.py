@@ -137,6 +137,29 @@ def test_linear_bwd_given_oracle_probabilities(name, dtype, path, shape):
     layer.close()
 
 
+@pytest.mark.parametrize("tile_n,split", [(256, 3), (128, 2), (64, 5), (256, 16), (256, 1), (64, 1)])
+def test_tensor_path_split_contraction_and_tile_widths(tile_n, split):
+    """Every tile width and a contraction cut into slices (combined in a fixed order) give the same
+    results within tolerance, for the sampled and the dense products; repeated runs are bit-identical."""
+    N, T, d_in, d_out = 5, 197, 320, 448
+    X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.5, sigma_B=1.0)
+    layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
+    layer.set_tuning(tile_n, tile_n, split, split)
+    Xc, dYc, Wc = cuda(X, dY, W)
+    ref = o.linear_bwd(np64(X), np64(dY), np64(W), N, T, 0.5, 0.5, 4)
+    p_in, q_in = torch.from_numpy(ref["p32"]).cuda(), torch.from_numpy(ref["q32"]).cuda()
+    dX, dW = layer.linear_bwd(Xc, dYc, Wc, 0.5, 0.5, 4, p_in=p_in, q_in=q_in)
+    assert rel_fro(np64(dX), ref["dX"]) <= tol_for(BF16) and rel_fro(np64(dW), ref["dW"]) <= tol_for(BF16)
+    assert not np64(dX)[np.repeat(~ref["keepA"], T)].any()
+    dX2, dW2 = layer.linear_bwd(Xc, dYc, Wc, 0.5, 0.5, 4, p_in=p_in, q_in=q_in)
+    assert torch.equal(dX, dX2) and torch.equal(dW, dW2)
+    dXd, dWd = o.dense_bwd(np64(X), np64(dY), np64(W))
+    dX3, dW3 = layer.dense_bwd(Xc, dYc, Wc)
+    assert rel_fro(np64(dX3), dXd) <= tol_for(BF16) and rel_fro(np64(dW3), dWd) <= tol_for(BF16)
+    assert layer.device_status() == 0
+    layer.close()
+
+
 @pytest.mark.parametrize("name,dtype,path", PATHS)
 def test_linear_bwd_end_to_end(name, dtype, path):
     """No overrides: the library's own probabilities, masks and products against the oracle's."""
