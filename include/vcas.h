@@ -15,7 +15,9 @@
  *  - "host" in an argument comment means a host pointer;
  *  - work is enqueued on the caller's stream and is asynchronous; no entry point except
  *    vcas_create, vcas_destroy and vcas_last_device_status synchronises or allocates;
- *  - a handle owns one workspace and must not be used from two streams at the same time;
+ *  - a handle owns one workspace and must not be used from two streams at the same time; inside a
+ *    call the library may fork part of the work onto a stream of its own and join it back before the
+ *    call's work on the caller's stream ends (stream capture records both branches);
  *  - device-side failures (a bounded wait that ran out) are recorded in a status word that
  *    vcas_last_device_status reads back.
  *

@@ -53,8 +53,8 @@ size_t layout(Handle* h, uint8_t* base) {
   if (h->tensor_path) {
     w.packG = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_out);
     w.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
-    w.partial_tiles = carve<float>(cur, (size_t)h->max_units * 128 * 256);
-    w.tickets = carve<int32_t>(cur, 2 * (size_t)h->max_units);
+    w.partial_tiles = carve<float>(cur, 2 * (size_t)h->max_units * 128 * 256);
+    w.tickets = carve<int32_t>(cur, 4 * (size_t)h->max_units);
   } else {
     w.packG = nullptr;
     w.packX = nullptr;
@@ -98,10 +98,10 @@ int sampled_dw(Handle* h, const void* X, const void* dY, float keep_hint, float*
 
 // stage boundary k of the current sampled call (no-op unless profiling is on)
 inline void mark(Handle* h, int k, cudaStream_t st) {
-  if (h->prof_enabled && h->prof_calls < PROF_RING) cudaEventRecord(h->ev[h->prof_calls * 6 + k], st);
+  if (h->prof_enabled && h->prof_calls < PROF_RING) cudaEventRecord(h->ev[h->prof_calls * 8 + k], st);
 }
 inline void mark_dense(Handle* h, int k, cudaStream_t st) {
-  if (h->prof_enabled && h->prof_dense_calls < PROF_RING) cudaEventRecord(h->ev_dense[h->prof_dense_calls * 3 + k], st);
+  if (h->prof_enabled && h->prof_dense_calls < PROF_RING) cudaEventRecord(h->ev_dense[h->prof_dense_calls * 4 + k], st);
 }
 
 int dense_dw(Handle* h, const void* X, const void* dY, float* out, cudaStream_t st) {
@@ -176,6 +176,13 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
     delete h;
     return VCAS_ERR_CUDA;
   }
+  if (cudaStreamCreateWithFlags(&h->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    cudaFree(h->base);
+    delete h;
+    return VCAS_ERR_CUDA;
+  }
   *out = reinterpret_cast<vcas_handle>(h);
   return VCAS_OK;
 }
@@ -184,11 +191,14 @@ int vcas_destroy(vcas_handle hh) {
   if (hh == nullptr) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   if (h->ev != nullptr) {
-    for (int i = 0; i < PROF_RING * 6; ++i) cudaEventDestroy(h->ev[i]);
-    for (int i = 0; i < PROF_RING * 3; ++i) cudaEventDestroy(h->ev_dense[i]);
+    for (int i = 0; i < PROF_RING * 8; ++i) cudaEventDestroy(h->ev[i]);
+    for (int i = 0; i < PROF_RING * 4; ++i) cudaEventDestroy(h->ev_dense[i]);
     delete[] h->ev;
     delete[] h->ev_dense;
   }
+  cudaStreamDestroy(h->side_stream);
+  cudaEventDestroy(h->ev_fork);
+  cudaEventDestroy(h->ev_join);
   const cudaError_t e = cudaFree(h->base);
   delete h;
   return e == cudaSuccess ? VCAS_OK : VCAS_ERR_CUDA;
@@ -220,6 +230,14 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
   VCAS_CUDA(launch_sampler(h, a, st));
+  // The two products are independent once the sampler has run: the dW branch (pack + product) is
+  // forked onto the handle's side stream and joined back before the call's work ends on `st`.
+  cudaStream_t sw = st;
+  if (h->tensor_path) {
+    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
+    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+    sw = h->side_stream;
+  }
   mark(h, 2, st);
   if (h->tensor_path) {
     VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, st));
@@ -228,15 +246,20 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   }
   mark(h, 3, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_pack(h, dY, X, st));
-    mark(h, 4, st);
+    mark(h, 6, sw);
+    VCAS_CUDA(launch_pack(h, dY, X, sw));
+    mark(h, 4, sw);
     const int hint = (int)(rho * nu * (float)(h->desc.N * h->desc.T)) + 1;
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, sw));
+    mark(h, 5, sw);
+    VCAS_CUDA(cudaEventRecord(h->ev_join, sw));
+    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   } else {
+    mark(h, 6, st);
     mark(h, 4, st);
     VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, dW, st));
+    mark(h, 5, st);
   }
-  mark(h, 5, st);
   if (h->prof_enabled && h->prof_calls < PROF_RING) h->prof_calls += 1;
   return VCAS_OK;
 }
@@ -252,6 +275,12 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
     return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
+  cudaStream_t sw = st;
+  if (h->tensor_path) {
+    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
+    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+    sw = h->side_stream;
+  }
   mark_dense(h, 0, st);
   if (h->tensor_path) {
     VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, st));
@@ -259,8 +288,13 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }
   mark_dense(h, 1, st);
-  const int rc = dense_dw(h, X, dY, dW, st);
-  mark_dense(h, 2, st);
+  mark_dense(h, 3, sw);
+  const int rc = dense_dw(h, X, dY, dW, sw);
+  mark_dense(h, 2, sw);
+  if (h->tensor_path) {
+    VCAS_CUDA(cudaEventRecord(h->ev_join, sw));
+    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
+  }
   if (h->prof_enabled && h->prof_dense_calls < PROF_RING) h->prof_dense_calls += 1;
   return rc;
 }
@@ -378,11 +412,11 @@ int vcas_set_profiling(vcas_handle hh, int32_t enable) {
   if (hh == nullptr) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   if (enable && h->ev == nullptr) {
-    h->ev = new (std::nothrow) cudaEvent_t[PROF_RING * 6];
-    h->ev_dense = new (std::nothrow) cudaEvent_t[PROF_RING * 3];
+    h->ev = new (std::nothrow) cudaEvent_t[PROF_RING * 8];
+    h->ev_dense = new (std::nothrow) cudaEvent_t[PROF_RING * 4];
     if (h->ev == nullptr || h->ev_dense == nullptr) return VCAS_ERR_WORKSPACE;
-    for (int i = 0; i < PROF_RING * 6; ++i) VCAS_CUDA(cudaEventCreate(&h->ev[i]));
-    for (int i = 0; i < PROF_RING * 3; ++i) VCAS_CUDA(cudaEventCreate(&h->ev_dense[i]));
+    for (int i = 0; i < PROF_RING * 8; ++i) VCAS_CUDA(cudaEventCreate(&h->ev[i]));
+    for (int i = 0; i < PROF_RING * 4; ++i) VCAS_CUDA(cudaEventCreate(&h->ev_dense[i]));
   }
   h->prof_enabled = enable != 0;
   h->prof_calls = h->prof_dense_calls = 0;
@@ -397,18 +431,21 @@ int vcas_stage_times(vcas_handle hh, float* ms, int32_t* calls) {
   calls[1] = h->prof_dense_calls;
   if (h->ev == nullptr) return VCAS_OK;
   VCAS_CUDA(cudaDeviceSynchronize());
+  // stage k lies between events (from, to): row norms 0-1, sampler 1-2, dX 2-3, pack 6-4, dW 4-5
+  const int from[5] = {0, 1, 2, 6, 4}, to[5] = {1, 2, 3, 4, 5};
   for (int c = 0; c < h->prof_calls; ++c)
     for (int k = 0; k < 5; ++k) {
       float t = 0.f;
-      VCAS_CUDA(cudaEventElapsedTime(&t, h->ev[c * 6 + k], h->ev[c * 6 + k + 1]));
+      VCAS_CUDA(cudaEventElapsedTime(&t, h->ev[c * 8 + from[k]], h->ev[c * 8 + to[k]]));
       ms[k] += t;
     }
-  for (int c = 0; c < h->prof_dense_calls; ++c)
-    for (int k = 0; k < 2; ++k) {
-      float t = 0.f;
-      VCAS_CUDA(cudaEventElapsedTime(&t, h->ev_dense[c * 3 + k], h->ev_dense[c * 3 + k + 1]));
-      ms[5 + k] += t;
-    }
+  for (int c = 0; c < h->prof_dense_calls; ++c) {      // dense dX between events 0-1, dense dW between 3-2
+    float t = 0.f;
+    VCAS_CUDA(cudaEventElapsedTime(&t, h->ev_dense[c * 4 + 0], h->ev_dense[c * 4 + 1]));
+    ms[5] += t;
+    VCAS_CUDA(cudaEventElapsedTime(&t, h->ev_dense[c * 4 + 3], h->ev_dense[c * 4 + 2]));
+    ms[6] += t;
+  }
   h->prof_calls = h->prof_dense_calls = 0;
   return VCAS_OK;
 }

@@ -33,8 +33,8 @@ struct Workspace {
   // compact operands of the weight-gradient product (tensor path)
   __nv_bfloat16* packG;  // [R_pad, d_out]
   __nv_bfloat16* packX;  // [R_pad, d_in]
-  float* partial_tiles;  // [max_units][128 * 256] fp32 partial tiles of a split contraction
-  int32_t* tickets;      // [2 * max_units]: slices stored, slices finished, per tile
+  float* partial_tiles;  // [2 products][max_units][128 * 256] fp32 partial tiles of a split contraction
+  int32_t* tickets;      // [2 products][2 * max_units]: slices stored, slices finished, per tile
   // probe buffers (App. D: the exact gradient, its running mean and running squared deviation)
   float* Gs;       // [d_out, d_in]
   float* Gact;     // [d_out, d_in]
@@ -56,10 +56,13 @@ struct Handle {
   size_t bytes;
   Workspace ws;
   uint64_t launches;
+  // second stream and fork/join events: the dW branch (pack + product) runs beside the dX product
+  cudaStream_t side_stream;
+  cudaEvent_t ev_fork, ev_join;
   // optional stage timing (vcas_set_profiling): rings of CUDA events around the stages
   bool prof_enabled;
-  cudaEvent_t* ev;        // [PROF_RING][6]: boundaries of row norms | sampler | dX | pack | dW
-  cudaEvent_t* ev_dense;  // [PROF_RING][3]: boundaries of dense dX | dense dW
+  cudaEvent_t* ev;        // [PROF_RING][8]: stage boundaries of a sampled call (see vcas_stage_times)
+  cudaEvent_t* ev_dense;  // [PROF_RING][4]: stage boundaries of a dense call
   int prof_calls, prof_dense_calls;
   // tuning overrides (vcas_set_tuning); 0 = choose automatically
   int tune_dx_tile_n, tune_dw_tile_n, tune_dx_split_k, tune_dw_split_k;

@@ -570,10 +570,10 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const size_t ob0 = slot_off(rb, cb, 0), ob1 = slot_off(rb, cb, 1);
           float fa[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
           float fb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          for (int sl0 = 0; sl0 < D.S; sl0 += 2) {               // slices in order, two at a time in flight
-            float4 x[2][4];
+          for (int sl0 = 0; sl0 < D.S; sl0 += 4) {               // slices in order, four at a time in flight
+            float4 x[4][4];
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
+            for (int q = 0; q < 4; ++q) {
               const int sl = min(sl0 + q, D.S - 1);
               const float* base = tile_part + (size_t)sl * (BM * BN);
               x[q][0] = __ldcg(reinterpret_cast<const float4*>(base + oa0));
@@ -582,7 +582,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               x[q][3] = __ldcg(reinterpret_cast<const float4*>(base + ob1));
             }
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
+            for (int q = 0; q < 4; ++q) {
               if (sl0 + q < D.S) {
                 fa[0] += x[q][0].x; fa[1] += x[q][0].y; fa[2] += x[q][0].z; fa[3] += x[q][0].w;
                 fa[4] += x[q][1].x; fa[5] += x[q][1].y; fa[6] += x[q][1].z; fa[7] += x[q][1].w;
@@ -752,11 +752,13 @@ cudaError_t run_gemm_bn(Handle* h, int bn, const CUtensorMap& a, const CUtensorM
   }
 }
 
-void common_params(Handle* h, GemmParams& P) {
+// which = 0: the dX product, 1: the dW product (they may run at the same time on two streams, so
+// each has its own split-contraction workspace)
+void common_params(Handle* h, GemmParams& P, int which) {
   P = GemmParams();
   P.status = h->ws.status;
-  P.partial = h->ws.partial_tiles;
-  P.tickets = h->ws.tickets;
+  P.partial = h->ws.partial_tiles + (size_t)which * h->max_units * (BM * 256);
+  P.tickets = h->ws.tickets + (size_t)which * 2 * h->max_units;
   P.max_units = h->max_units;
   P.d_in = h->desc.d_in;
   P.d_out = h->desc.d_out;
@@ -787,7 +789,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
     if (!make_map(&tmC, dX, 3, dims, strides, box)) return cudaErrorInvalidValue;
   }
   GemmParams P;
-  common_params(h, P);
+  common_params(h, P, 0);
   P.idxA = h->ws.idxA; P.dropA = h->ws.dropA; P.counts = h->ws.counts; P.scaleA = h->ws.scaleA;
   P.H = (const __nv_bfloat16*)H; P.dX = (__nv_bfloat16*)dX;
   P.N = d.N; P.T = d.T; P.dense = dense ? 1 : 0;
@@ -837,7 +839,7 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
     if (!make_map(&tmC, dW, 2, dims, strides, box, CU_TENSOR_MAP_DATA_TYPE_FLOAT32)) return cudaErrorInvalidValue;
   }
   GemmParams P;
-  common_params(h, P);
+  common_params(h, P, 1);
   P.cnt = cnt; P.dW = dW;
   const long mtiles = (d.d_out + BM - 1) / BM;
   const Plan plan = plan_tiles(mtiles, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
