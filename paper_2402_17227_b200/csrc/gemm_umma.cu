@@ -696,11 +696,11 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tile width and number of contraction slices from a small cost model: waves of the persistent
-// grid x (k-blocks per unit x time per k-block + fixed cost per unit) + the cost of combining
-// slices.  Times per k-block were measured on B200 (about 0.5 / 0.45 / 0.43 us for 256 / 128 / 64
-// wide tiles: the shared-memory fill rate of one SM bounds them, so narrow tiles only pay off
-// when they fill more SMs).
+// Tile width and number of contraction slices from a small cost model, calibrated on B200 with
+// in-kernel timestamps: a k-block costs about 0.5 / 0.45 / 0.43 us for 256 / 128 / 64 wide tiles
+// (the shared-memory fill rate of one SM bounds it, so narrow tiles only pay off when they fill
+// more SMs); a unit costs about 4 us of set-up, pipeline fill and output store; a sliced unit
+// about 7 us more (partial store, wait for its siblings, reduction).
 struct Plan { int bn, split; };
 Plan plan_tiles(long row_tiles, int n_extent, int kblocks, int num_sms, int max_units, int force_bn, int force_split) {
   const int widths[3] = {256, 128, 64};
@@ -718,8 +718,8 @@ Plan plan_tiles(long row_tiles, int n_extent, int kblocks, int num_sms, int max_
       if (sp > 1 && force_split == 0 && kblocks / sp < 4) continue;   // slices too short to pay off
       const long units = tiles * sp;
       const double waves = (double)((units + num_sms - 1) / num_sms);
-      double t = waves * ((double)((kblocks + sp - 1) / sp) * c_kb[i] + 4.0);
-      if (sp > 1) t += 3.0 + 0.25 * sp;
+      const double unit_fixed = sp > 1 ? 11.0 + 0.25 * sp : 4.0;
+      const double t = waves * ((double)((kblocks + sp - 1) / sp) * c_kb[i] + unit_fixed);
       if (t < best_t - 1e-9) { best_t = t; best = {widths[i], sp}; }
     }
   }
