@@ -207,7 +207,9 @@ int vcas_set_tuning(vcas_handle h, int32_t dx_tile_n, int32_t dw_tile_n, int32_t
 
 /* Stage timing for benchmarks (the paper has no counterpart; Sec. 6 only reports end-to-end
  * hours).  While enabled, vcas_linear_bwd(_ex) and vcas_dense_bwd record CUDA events on the
- * caller's stream at their stage boundaries, for up to 2048 calls of each kind.  Enabling
+ * caller's stream at their stage boundaries, for up to 2048 calls of each kind, and run their
+ * kernels one after the other on that stream (no internal fork) so that each pair of events
+ * brackets one kernel.  Enabling
  * allocates the events once (host objects); it also clears what was recorded. */
 int vcas_set_profiling(vcas_handle h, int32_t enable);
 /* Synchronises the device, then writes the summed milliseconds of the recorded calls to

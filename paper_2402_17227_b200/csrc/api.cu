@@ -232,8 +232,11 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   VCAS_CUDA(launch_sampler(h, a, st));
   // The two products are independent once the sampler has run: the dW branch (pack + product) is
   // forked onto the handle's side stream and joined back before the call's work ends on `st`.
+  // (While stage profiling is on, everything stays on `st` so that each pair of events brackets
+  // one kernel.)
   cudaStream_t sw = st;
-  if (h->tensor_path) {
+  const bool fork = h->tensor_path && !h->prof_enabled;
+  if (fork) {
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
     sw = h->side_stream;
@@ -252,8 +255,10 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     const int hint = (int)(rho * nu * (float)(h->desc.N * h->desc.T)) + 1;
     VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, sw));
     mark(h, 5, sw);
-    VCAS_CUDA(cudaEventRecord(h->ev_join, sw));
-    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
+    if (fork) {
+      VCAS_CUDA(cudaEventRecord(h->ev_join, sw));
+      VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
+    }
   } else {
     mark(h, 6, st);
     mark(h, 4, st);
@@ -276,7 +281,8 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
   cudaStream_t sw = st;
-  if (h->tensor_path) {
+  const bool fork = h->tensor_path && !h->prof_enabled;
+  if (fork) {
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
     sw = h->side_stream;
@@ -291,7 +297,7 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
   mark_dense(h, 3, sw);
   const int rc = dense_dw(h, X, dY, dW, sw);
   mark_dense(h, 2, sw);
-  if (h->tensor_path) {
+  if (fork) {
     VCAS_CUDA(cudaEventRecord(h->ev_join, sw));
     VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   }

@@ -314,11 +314,15 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     ab[e + 2] = sqrtf(va.z) * sqrtf(vb.z); ab[e + 3] = sqrtf(va.w) * sqrtf(vb.w);
   }
 
-  // ---- ||G_n||_F: one warp per datum, fixed order
+  // ---- ||G_n||_F: one warp per datum, fixed order; four independent partial sums per lane keep
+  // several loads in flight (a dependent chain of T/32 loads would cost a memory latency each)
   for (int n = warp; n < N; n += 32) {
-    float s = 0.f;
-    for (int t = lane; t < T; t += 32) s += P.a[(size_t)n * T + t];
-    s = warp_sum(s);
+    const float* an = P.a + (size_t)n * T;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    int t = lane;
+    for (; t + 96 < T; t += 128) { s0 += an[t]; s1 += an[t + 32]; s2 += an[t + 64]; s3 += an[t + 96]; }
+    for (; t < T; t += 32) s0 += an[t];
+    const float s = warp_sum((s0 + s1) + (s2 + s3));
     if (lane == 0) { const float g = sqrtf(s); P.g[n] = g; sh.pA[n] = g; }
   }
   __syncthreads();
