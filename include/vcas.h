@@ -139,7 +139,7 @@ int vcas_score(vcas_handle h, const void* X, const void* dY, float rho, float nu
  * acceptable, or plug-ins that are handed a fixed memory budget.  vcas_create / vcas_score need a
  * workspace from cudaMalloc; this entry point instead keeps its intermediates (row norms,
  * scores, rescale factors, index lists) in a fixed array inside the library image, about
- * 0.5 MB that every GPU loading the library holds until the process exits.
+ * 0.6 MB that every GPU loading the library holds until the process exits.
  *   Limits: N <= 4096 and N*T <= 16384, otherwise VCAS_ERR_SHAPE.  d_in, d_out multiples of 8.
  *   Inputs and outputs are the caller's, as for vcas_score (any output may be NULL).
  *   The first call on each device looks up the array's device address (with that device

@@ -36,6 +36,8 @@ size_t layout(Handle* h, uint8_t* base) {
   Workspace& w = h->ws;
   w.a = carve<float>(cur, R);
   w.b = carve<float>(cur, R);
+  w.lev = carve<float>(cur, R);
+  w.u24 = carve<uint32_t>(cur, R);
   w.g = carve<float>(cur, N);
   w.p = carve<float>(cur, N);
   w.w = carve<float>(cur, R);
@@ -225,7 +227,7 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
   mark(h, 0, st);
-  VCAS_CUDA(launch_rownorms(h, dY, X, st));
+  VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
   mark(h, 1, st);
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
@@ -312,7 +314,7 @@ int vcas_score(vcas_handle hh, const void* X, const void* dY, float rho, float n
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
-  VCAS_CUDA(launch_rownorms(h, dY, X, st));
+  VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 1; a.accumulate_vw = 0;
   VCAS_CUDA(launch_sampler(h, a, st));
@@ -351,7 +353,7 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
     int rc = dense_dw(h, X_i[i], dY_i[i], h->ws.Gs, st);            // G_s,i
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(launch_probe_welford(h, i, st));
-    VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], st));
+    VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, st));   // the probe draws no SampleW mask
     for (int j = 0; j < M; ++j) {
       SamplerArgs a;
       a.rho = rho; a.nu = nu; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 0; a.accumulate_vw = 1;

@@ -16,6 +16,8 @@ struct Workspace {
   // scores (Sec. 4.1, 4.2)
   float* a;        // [R]  ||dY_r||^2
   float* b;        // [R]  ||X_r||^2
+  float* lev;      // [R]  ||dY_r|| ||X_r||
+  uint32_t* u24;   // [R]  SampleW's 24-bit uniform of each row
   float* g;        // [N]  ||G_n||_F
   float* p;        // [N]  SampleA keep probabilities
   float* w;        // [R]  leverage scores of G_hat
@@ -112,7 +114,8 @@ __device__ __forceinline__ int warp_sum(int v) {
 // ---------------------------------------------------------------------------------------
 // Launchers (one per .cu file).  All enqueue on `st` and return a cudaError_t.
 // ---------------------------------------------------------------------------------------
-cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, cudaStream_t st);
+// seed: the call's seed (the SampleW uniforms are drawn here, one per row)
+cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, cudaStream_t st);
 
 struct SamplerArgs {
   float rho, nu;

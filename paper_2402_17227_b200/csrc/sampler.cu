@@ -121,6 +121,7 @@ __device__ int block_compact(int n, KeepFn keep, EmitFn emit, Scratch* sc) {
 
 struct SamplerParams {
   const float* a; const float* b;
+  const float* lev; const uint32_t* u24;   // per-row leverage ||dY_r|| ||X_r|| and SampleW uniform (row-norm kernel)
   float* g; float* p; float* w; float* q;
   float* scaleA; float* scaleW;
   int32_t* idxA; int32_t* dropA; int32_t* idxW; int32_t* counts;
@@ -295,23 +296,35 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
   const int N = P.N, T = P.T, R = N * T;
   const int r0 = tid * E;
 
-  // this thread's rows: ||dY_r|| ||X_r|| (the unscaled leverage score)
+  // this thread's rows: the unscaled leverage score and the SampleW uniform, both made per row by
+  // the row-norm kernel
   float ab[E];
+  uint32_t ur[E];
 #pragma unroll
   for (int e = 0; e < E; e += 4) {
-    float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
     if (r0 + e + 3 < R) {
-      va = *reinterpret_cast<const float4*>(P.a + r0 + e);
-      vb = *reinterpret_cast<const float4*>(P.b + r0 + e);
+      const float4 v = *reinterpret_cast<const float4*>(P.lev + r0 + e);
+      const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + r0 + e);
+      ab[e] = v.x; ab[e + 1] = v.y; ab[e + 2] = v.z; ab[e + 3] = v.w;
+      ur[e] = u.x; ur[e + 1] = u.y; ur[e + 2] = u.z; ur[e + 3] = u.w;
     } else {
-      float ta[4] = {0.f, 0.f, 0.f, 0.f}, tb[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int i = 0; i < 4; ++i)
-        if (r0 + e + i < R) { ta[i] = P.a[r0 + e + i]; tb[i] = P.b[r0 + e + i]; }
-      va = make_float4(ta[0], ta[1], ta[2], ta[3]);
-      vb = make_float4(tb[0], tb[1], tb[2], tb[3]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const bool in = r0 + e + i < R;
+        ab[e + i] = in ? P.lev[r0 + e + i] : 0.f;
+        ur[e + i] = in ? P.u24[r0 + e + i] : 0xffffffffu;
+      }
     }
-    ab[e] = sqrtf(va.x) * sqrtf(vb.x); ab[e + 1] = sqrtf(va.y) * sqrtf(vb.y);
-    ab[e + 2] = sqrtf(va.z) * sqrtf(vb.z); ab[e + 3] = sqrtf(va.w) * sqrtf(vb.w);
+  }
+  // datum of each of this thread's rows without a division per row
+  int nrow[E];
+  {
+    int n = r0 / T, rem = r0 - n * T;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+      nrow[e] = n < N ? n : N - 1;
+      if (++rem == T) { rem = 0; ++n; }
+    }
   }
 
   // ---- ||G_n||_F: one warp per datum, fixed order; four independent partial sums per lane keep
@@ -371,7 +384,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     const int r = r0 + e;
     float wr = 0.f;
     if (r < R) {
-      const int n = r / T;
+      const int n = nrow[e];
       if (sh.scaleA[n] > 0.f) wr = ab[e] / sh.pA[n];
       P.w[r] = wr;
     }
@@ -382,7 +395,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
 #pragma unroll
     for (int e = 0; e < E; ++e) {
       const int r = r0 + e;
-      q[e] = (r < R && sh.scaleA[r / T] > 0.f) ? P.q_in[r] : 0.f;
+      q[e] = (r < R && sh.scaleA[nrow[e]] > 0.f) ? P.q_in[r] : 0.f;
     }
   } else {
     const float budget = P.nu * (float)T * (float)cntA;
@@ -450,8 +463,8 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     const int r = r0 + e;
     bool k = false;
     if (r < R) {
-      if (P.sample_w) k = q[e] > 0.f && bernoulli_keep(q[e], P.seed, 1u, (uint64_t)r);
-      else k = sh.scaleA[r / T] > 0.f;
+      if (P.sample_w) k = q[e] > 0.f && ur[e] < (uint32_t)floorf(q[e] * 16777216.0f);
+      else k = sh.scaleA[nrow[e]] > 0.f;
     }
     keepbits |= (k ? 1u : 0u) << e;
   }
@@ -477,7 +490,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     if (keepbits & (1u << e)) {
       const int r = r0 + e;
       P.idxW[base] = r;
-      P.scaleW[base] = P.sample_w ? sh.scaleA[r / T] / q[e] : sh.scaleA[r / T];
+      P.scaleW[base] = P.sample_w ? sh.scaleA[nrow[e]] / q[e] : sh.scaleA[nrow[e]];
       ++base;
     }
   if (tid == 0) { P.counts[0] = cntA; P.counts[1] = total; }
@@ -502,7 +515,7 @@ mask_kernel(const float* __restrict__ p, int n, uint64_t seed, int sampler, uint
 cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st) {
   const Workspace& ws = h->ws;
   SamplerParams P;
-  P.a = ws.a; P.b = ws.b; P.g = ws.g; P.p = ws.p; P.w = ws.w; P.q = ws.q;
+  P.a = ws.a; P.b = ws.b; P.lev = ws.lev; P.u24 = ws.u24; P.g = ws.g; P.p = ws.p; P.w = ws.w; P.q = ws.q;
   P.scaleA = ws.scaleA; P.scaleW = ws.scaleW;
   P.idxA = ws.idxA; P.dropA = ws.dropA; P.idxW = ws.idxW; P.counts = ws.counts;
   P.acc = ws.acc;

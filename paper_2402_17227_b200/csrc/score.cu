@@ -41,20 +41,11 @@ template <> struct Vec<float> {
   static __device__ __forceinline__ float one(float x) { return x * x; }
 };
 
-// task t < R: row t of dY -> a[t];  task t >= R: row t-R of X -> b[t-R]
+// sum of squares of one row of d elements, accumulated by the 32 lanes of a warp (not yet reduced)
 template <typename T>
-__global__ void __launch_bounds__(256) rownorm_kernel(const T* __restrict__ dY, const T* __restrict__ X,
-                                                      int R, int d_out, int d_in,
-                                                      float* __restrict__ a, float* __restrict__ b) {
+__device__ __forceinline__ float row_partial(const T* __restrict__ src, int d, int lane) {
   using V = typename Vec<T>::type;
   constexpr int VN = Vec<T>::N;
-  const int lane = threadIdx.x & 31;
-  const int task = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (task >= 2 * R) return;
-  const bool is_x = task >= R;
-  const int row = is_x ? task - R : task;
-  const int d = is_x ? d_in : d_out;
-  const T* src = (is_x ? X : dY) + (size_t)row * d;
   float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
   if ((d % VN) == 0) {
     const V* v = reinterpret_cast<const V*>(src);
@@ -68,23 +59,45 @@ __global__ void __launch_bounds__(256) rownorm_kernel(const T* __restrict__ dY, 
   } else {
     for (int i = lane; i < d; i += 32) acc0 += Vec<T>::one(src[i]);
   }
-  const float s = warp_sum((acc0 + acc1) + (acc2 + acc3));
-  if (lane == 0) (is_x ? b : a)[row] = s;
+  return (acc0 + acc1) + (acc2 + acc3);
+}
+
+// One warp per row r: a[r] = ||dY_r||^2, b[r] = ||X_r||^2, and two per-row values the sampling
+// stage would otherwise compute on its single SM: lev[r] = ||dY_r|| ||X_r|| (the leverage score of
+// Sec. 4.2 before the 1/p_n rescale) and u24[r], the 24-bit Philox uniform of SampleW for this row.
+template <typename T>
+__global__ void __launch_bounds__(256) rownorm_kernel(const T* __restrict__ dY, const T* __restrict__ X,
+                                                      int R, int d_out, int d_in, uint64_t seed,
+                                                      float* __restrict__ a, float* __restrict__ b,
+                                                      float* __restrict__ lev, uint32_t* __restrict__ u24) {
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= R) return;
+  const float pa = row_partial<T>(dY + (size_t)row * d_out, d_out, lane);
+  const float pb = row_partial<T>(X + (size_t)row * d_in, d_in, lane);
+  const float sa = warp_sum(pa), sb = warp_sum(pb);
+  if (lane == 0) {
+    a[row] = sa;
+    b[row] = sb;
+    lev[row] = sqrtf(sa) * sqrtf(sb);
+    u24[row] = philox_word0((uint32_t)row, 0u, 1u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32)) >> 8;
+  }
 }
 
 }  // namespace
 
-cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, cudaStream_t st) {
+cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   const int R = d.N * d.T;
   const int warps_per_block = 8;
-  const int blocks = (2 * R + warps_per_block - 1) / warps_per_block;
+  const int blocks = (R + warps_per_block - 1) / warps_per_block;
   if (d.dtype == VCAS_DTYPE_BF16) {
-    rownorm_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dY, (const __nv_bfloat16*)X,
-                                                          R, d.d_out, d.d_in, h->ws.a, h->ws.b);
+    rownorm_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dY, (const __nv_bfloat16*)X, R,
+                                                          d.d_out, d.d_in, seed, h->ws.a, h->ws.b, h->ws.lev,
+                                                          h->ws.u24);
   } else {
-    rownorm_kernel<float><<<blocks, 256, 0, st>>>((const float*)dY, (const float*)X, R, d.d_out, d.d_in,
-                                                  h->ws.a, h->ws.b);
+    rownorm_kernel<float><<<blocks, 256, 0, st>>>((const float*)dY, (const float*)X, R, d.d_out, d.d_in, seed,
+                                                  h->ws.a, h->ws.b, h->ws.lev, h->ws.u24);
   }
   h->launches += 1;
   return cudaGetLastError();

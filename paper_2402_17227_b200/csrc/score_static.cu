@@ -11,12 +11,12 @@ namespace {
 
 constexpr int STATIC_MAX_R = 16384;   // rows (N*T) the fixed scratch can serve
 constexpr int STATIC_MAX_N = 4096;    // data
-constexpr size_t kRowArrays = 6;      // a, b, w, q, scaleW (float) and idxW (int32), each [STATIC_MAX_R]
+constexpr size_t kRowArrays = 8;      // a, b, w, q, scaleW, lev (float), idxW (int32), u24 (uint32), each [STATIC_MAX_R]
 constexpr size_t kDatumArrays = 6;    // g, p, scaleA, sorted (float) and idxA, dropA (int32), each [STATIC_MAX_N]
 constexpr size_t kTailBytes = 512;    // counts [8] int32 and acc [16] double, 256-byte slots
 constexpr size_t kScratchBytes = kRowArrays * STATIC_MAX_R * 4 + kDatumArrays * STATIC_MAX_N * 4 + kTailBytes;
 
-// Lives in every GPU that loads the library until the process exits (about 0.5 MB).  In host
+// Lives in every GPU that loads the library until the process exits (about 0.6 MB).  In host
 // code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_score_scratch[kScratchBytes];
 
@@ -68,6 +68,8 @@ extern "C" int vcas_score_static(int32_t N, int32_t T, int32_t d_in, int32_t d_o
   ws.q = fr + 3 * STATIC_MAX_R;
   ws.scaleW = fr + 4 * STATIC_MAX_R;
   ws.idxW = reinterpret_cast<int32_t*>(fr + 5 * STATIC_MAX_R);
+  ws.lev = fr + 6 * STATIC_MAX_R;
+  ws.u24 = reinterpret_cast<uint32_t*>(fr + 7 * STATIC_MAX_R);
   float* fn = fr + kRowArrays * STATIC_MAX_R;
   ws.g = fn + 0 * STATIC_MAX_N;
   ws.p = fn + 1 * STATIC_MAX_N;
@@ -81,7 +83,7 @@ extern "C" int vcas_score_static(int32_t N, int32_t T, int32_t d_in, int32_t d_o
 
   // The array keeps the previous call's contents: the counters and accumulators start at zero.
   if (cudaMemsetAsync(tail, 0, kTailBytes, st) != cudaSuccess) return VCAS_ERR_CUDA;
-  if (launch_rownorms(&h, dY, X, st) != cudaSuccess) return VCAS_ERR_CUDA;
+  if (launch_rownorms(&h, dY, X, seed, st) != cudaSuccess) return VCAS_ERR_CUDA;
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 1; a.accumulate_vw = 0;
   if (launch_sampler(&h, a, st) != cudaSuccess) return VCAS_ERR_CUDA;
