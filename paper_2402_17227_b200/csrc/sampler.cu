@@ -294,7 +294,9 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
   __shared__ FastShared sh;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = P.N, T = P.T, R = N * T;
-  const int r0 = tid * E;
+  // Element e of this thread is row (e / 4) * 4096 + tid * 4 + (e % 4): four consecutive rows per
+  // thread and group, so that every 16-byte load or store of a warp covers 512 contiguous bytes.
+  auto row_of = [&](int e) { return (e >> 2) * (4 * SAMPLER_THREADS) + tid * 4 + (e & 3); };
 
   // this thread's rows: the unscaled leverage score and the SampleW uniform, both made per row by
   // the row-norm kernel
@@ -302,27 +304,30 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
   uint32_t ur[E];
 #pragma unroll
   for (int e = 0; e < E; e += 4) {
-    if (r0 + e + 3 < R) {
-      const float4 v = *reinterpret_cast<const float4*>(P.lev + r0 + e);
-      const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + r0 + e);
+    const int rb = row_of(e);
+    if (rb + 3 < R) {
+      const float4 v = *reinterpret_cast<const float4*>(P.lev + rb);
+      const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + rb);
       ab[e] = v.x; ab[e + 1] = v.y; ab[e + 2] = v.z; ab[e + 3] = v.w;
       ur[e] = u.x; ur[e + 1] = u.y; ur[e + 2] = u.z; ur[e + 3] = u.w;
     } else {
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const bool in = r0 + e + i < R;
-        ab[e + i] = in ? P.lev[r0 + e + i] : 0.f;
-        ur[e + i] = in ? P.u24[r0 + e + i] : 0xffffffffu;
+        const bool in = rb + i < R;
+        ab[e + i] = in ? P.lev[rb + i] : 0.f;
+        ur[e + i] = in ? P.u24[rb + i] : 0xffffffffu;
       }
     }
   }
-  // datum of each of this thread's rows without a division per row
+  // datum of each of this thread's rows: one division per group of four rows
   int nrow[E];
-  {
-    int n = r0 / T, rem = r0 - n * T;
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-      nrow[e] = n < N ? n : N - 1;
+  for (int e = 0; e < E; e += 4) {
+    const int rb = row_of(e);
+    int n = rb / T, rem = rb - n * T;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      nrow[e + i] = n < N ? n : N - 1;
       if (++rem == T) { rem = 0; ++n; }
     }
   }
@@ -381,20 +386,25 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
   float w[E];
 #pragma unroll
   for (int e = 0; e < E; ++e) {
-    const int r = r0 + e;
-    float wr = 0.f;
-    if (r < R) {
-      const int n = nrow[e];
-      if (sh.scaleA[n] > 0.f) wr = ab[e] / sh.pA[n];
-      P.w[r] = wr;
+    const int n = nrow[e];
+    w[e] = (row_of(e) < R && sh.scaleA[n] > 0.f) ? ab[e] / sh.pA[n] : 0.f;
+  }
+#pragma unroll
+  for (int e = 0; e < E; e += 4) {
+    const int rb = row_of(e);
+    if (rb + 3 < R) {
+      *reinterpret_cast<float4*>(P.w + rb) = make_float4(w[e], w[e + 1], w[e + 2], w[e + 3]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (rb + i < R) P.w[rb + i] = w[e + i];
     }
-    w[e] = wr;
   }
   float q[E];
   if (P.q_in != nullptr) {
 #pragma unroll
     for (int e = 0; e < E; ++e) {
-      const int r = r0 + e;
+      const int r = row_of(e);
       q[e] = (r < R && sh.scaleA[nrow[e]] > 0.f) ? P.q_in[r] : 0.f;
     }
   } else {
@@ -443,8 +453,16 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     }
   }
 #pragma unroll
-  for (int e = 0; e < E; ++e)
-    if (r0 + e < R) P.q[r0 + e] = q[e];
+  for (int e = 0; e < E; e += 4) {
+    const int rb = row_of(e);
+    if (rb + 3 < R) {
+      *reinterpret_cast<float4*>(P.q + rb) = make_float4(q[e], q[e + 1], q[e + 2], q[e + 3]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (rb + i < R) P.q[rb + i] = q[e + i];
+    }
+  }
 
   if (P.accumulate_vw) {      // Eq. 3 at these probabilities (probe only)
     float vw = 0.f;
@@ -456,43 +474,48 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     if (tid == 0) P.acc[1] += (double)vw;
   }
 
-  // ---- mask and ordered compaction: per-thread count, block exclusive scan, scatter
+  // ---- mask and ordered compaction: rows ascend with (group, thread, k), so each group of 4096 rows
+  // gets its own block-wide exclusive scan of the per-thread counts, on top of the groups before it
   unsigned keepbits = 0;
 #pragma unroll
   for (int e = 0; e < E; ++e) {
-    const int r = r0 + e;
     bool k = false;
-    if (r < R) {
+    if (row_of(e) < R) {
       if (P.sample_w) k = q[e] > 0.f && ur[e] < (uint32_t)floorf(q[e] * 16777216.0f);
       else k = sh.scaleA[nrow[e]] > 0.f;
     }
     keepbits |= (k ? 1u : 0u) << e;
   }
-  const int mine = __popc(keepbits);
-  int incl = mine;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += t;
-  }
-  if (lane == 31) sh.warp_tot[warp] = incl;
-  __syncthreads();
-  int base = incl - mine;
   int total = 0;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const int t = sh.warp_tot[i];
-    if (i < warp) base += t;
-    total += t;
-  }
+  for (int g4 = 0; g4 < E / 4; ++g4) {
+    const unsigned bits = (keepbits >> (g4 * 4)) & 0xfu;
+    const int mine = __popc(bits);
+    int incl = mine;
 #pragma unroll
-  for (int e = 0; e < E; ++e)
-    if (keepbits & (1u << e)) {
-      const int r = r0 + e;
-      P.idxW[base] = r;
-      P.scaleW[base] = P.sample_w ? sh.scaleA[nrow[e]] / q[e] : sh.scaleA[nrow[e]];
-      ++base;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
     }
+    __syncthreads();                       // warp_tot of the previous group has been read by everyone
+    if (lane == 31) sh.warp_tot[warp] = incl;
+    __syncthreads();
+    int base = total + incl - mine;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int t = sh.warp_tot[i];
+      if (i < warp) base += t;
+      total += t;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (bits & (1u << i)) {
+        const int e = g4 * 4 + i;
+        P.idxW[base] = row_of(e);
+        P.scaleW[base] = P.sample_w ? sh.scaleA[nrow[e]] / q[e] : sh.scaleA[nrow[e]];
+        ++base;
+      }
+  }
   if (tid == 0) { P.counts[0] = cntA; P.counts[1] = total; }
 }
 
