@@ -333,3 +333,34 @@ def gelu_prime(h):
     Phi = 0.5 * (1.0 + np.vectorize(erf)(h / sqrt(2.0)))
     phi = np.exp(-0.5 * h * h) / sqrt(2.0 * pi)
     return Phi + h * phi
+
+
+# --------------------------------------------------------------------------------------
+# Entry-by-entry forms for inputs too large for the whole-matrix functions above
+# --------------------------------------------------------------------------------------
+def row_sqnorms_chunked(M, chunk: int = 2048):
+    """row_sqnorms on slices of rows (same sums; avoids a float64 copy of a very large matrix)."""
+    return np.concatenate([row_sqnorms(np.asarray(M[i:i + chunk], dtype=np.float64))
+                           for i in range(0, M.shape[0], chunk)])
+
+
+def dX_rows(dY, W, p32, keepA, T: int, rows):
+    """Rows `rows` of dX = G_hat W (App. E): (1/p_n) dY_r W for rows of kept data, 0 otherwise."""
+    W = np.asarray(W, dtype=np.float64)
+    out = np.zeros((len(rows), W.shape[1]))
+    for i, r in enumerate(rows):
+        n = r // T
+        if keepA[n]:
+            out[i] = (np.asarray(dY[r], dtype=np.float64) / float(p32[n])) @ W
+    return out
+
+
+def dW_rows(dY, X, p32, q32, keepW, T: int, outs):
+    """Rows `outs` of dW = G_tilde^T X (Sec. 4.2): sum over kept rows r of dY[r, o] / (p_n q_r) * X_r."""
+    kept = np.flatnonzero(keepW)
+    scale = 1.0 / (np.asarray(p32, dtype=np.float64)[kept // T] * np.asarray(q32, dtype=np.float64)[kept])
+    Xk = np.asarray(X[kept], dtype=np.float64)
+    out = np.zeros((len(outs), Xk.shape[1]))
+    for i, oo in enumerate(outs):
+        out[i] = (np.asarray(dY[kept, oo], dtype=np.float64) * scale) @ Xk
+    return out

@@ -395,3 +395,16 @@ def test_gelu_prime_is_the_derivative_of_gelu():
     t = torch.tensor(h, dtype=torch.float64, requires_grad=True)
     torch.nn.functional.gelu(t).sum().backward()          # library erf-GELU
     assert np.allclose(o.gelu_prime(h), t.grad.numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_entrywise_forms_agree_with_whole_matrix_forms():
+    # the per-row forms used on very large inputs are the same numbers as linear_bwd's matrices
+    N, T, di, do = 6, 5, 7, 9
+    X, dY, W = _tiny(21, N, T, di, do)
+    out = o.linear_bwd(X, dY, W, N, T, 0.6, 0.5, seed=4)
+    rows = [0, 7, 13, 29]
+    assert np.allclose(o.dX_rows(dY, W, out["p32"], out["keepA"], T, rows), out["dX"][rows], rtol=1e-12, atol=1e-12)
+    outs = [0, 3, 8]
+    assert np.allclose(o.dW_rows(dY, X, out["p32"], out["q32"], out["keepW"], T, outs), out["dW"][outs],
+                       rtol=1e-12, atol=1e-12)
+    assert np.allclose(o.row_sqnorms_chunked(dY, chunk=4), o.row_sqnorms(dY), rtol=1e-15)
