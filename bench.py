@@ -212,6 +212,7 @@ def main():
 
     from paper_2402_17227_b200 import binding as vb
     from paper_2402_17227_b200 import build as vbuild
+    from paper_2402_17227_b200 import dist_util
     from paper_2402_17227_b200 import inputs
 
     rank = int(os.environ.get("RANK", "0"))
@@ -235,7 +236,7 @@ def main():
     layer = vb.Layer(N, T, d_in, d_out, case.dtype, vb.GEMM_AUTO, cfg)
 
     # rank r draws its own batches (data-parallel replicas: per-replica sampling, no exchange here)
-    host = [inputs.make_layer(case, batch=rank * N_BATCHES + b) for b in range(N_BATCHES)]
+    host = [inputs.make_layer(case, batch=b) for b in dist_util.rank_batches(rank, N_BATCHES)]
     W = host[0][2].to(dev)
     Xs = [h[0].to(dev) for h in host]
     dYs = [h[1].to(dev) for h in host]
@@ -297,12 +298,7 @@ def main():
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return dist_util.max_over_ranks(e0.elapsed_time(e1), dev)
 
     for _ in range(args.warmup):
         step()
@@ -313,7 +309,7 @@ def main():
     launches = args.steps * (launches_per_period + probe_launches[0])
     clock_info = clocks.stop() if rank == 0 else None
     ms_per_step = total_ms / args.steps
-    value = ms_per_step / (F_CALLS * world)      # whole-job: all ranks' calls per unit time
+    value = dist_util.ms_per_layer(ms_per_step, F_CALLS, world)      # whole-job: all ranks' calls per unit time
 
     # -- the same period without the probe, the dense backward (graph replays), and per-stage times
     reps = max(3, min(args.steps, 10))
