@@ -42,6 +42,21 @@ def peaks():
     return dict(hbm=6650.0, tc_burst=1590.0, tc_sustained=1400.0, source="fallback")
 
 
+def ncu_traffic(kernel: str):
+    """DRAM bytes per launch of `kernel` from the last ncu capture (profiles/), or None when the kernel's
+    source file has changed since that capture."""
+    import hashlib
+    path = os.path.join(ROOT, "paper_2402_17227_b200", "ncu_traffic.json")
+    if not os.path.exists(path):
+        return None
+    rec = json.load(open(path)).get(kernel)
+    if rec is None:
+        return None
+    src = os.path.join(ROOT, "paper_2402_17227_b200", "csrc", rec["source"])
+    sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+    return rec["dram_bytes_per_launch"] if sha == rec["source_sha256"] else None
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -395,12 +410,12 @@ def main():
     dname = names[dom]
     if stages[dname]["bound"] == "tensor":
         roof = dict(bound="tensor", kernel=dname, achieved=stages[dname]["achieved"], peak=pk["tc_burst"],
-                    unit="TFLOP/s", traffic=None, peak_source=pk["source"] + " bf16 burst")
+                    unit="TFLOP/s", traffic=ncu_traffic(dname), peak_source=pk["source"] + " bf16 burst")
     else:
         if dname != "rownorm_kernel":   # the small latency-bound stages are reported under the scoring pass
             dname = "rownorm_kernel"
         roof = dict(bound="hbm", kernel=dname, achieved=stages[dname]["achieved"], peak=pk["hbm"], unit="GB/s",
-                    traffic=None, peak_source=pk["source"] + " copy bandwidth")
+                    traffic=ncu_traffic(dname), peak_source=pk["source"] + " copy bandwidth")
     roof["frac"] = roof["achieved"] / roof["peak"] if roof["achieved"] else None
     roof["kernel_ms"] = stages[dname]["ms"]
 

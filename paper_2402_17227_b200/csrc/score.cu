@@ -41,7 +41,7 @@ template <> struct Vec<float> {
   static __device__ __forceinline__ float one(float x) { return x * x; }
 };
 
-// sum of squares of one row of d elements, accumulated by the 32 lanes of a warp (not yet reduced)
+// Sum of squares of one row of d elements, accumulated by the 32 lanes of a warp (not yet reduced).
 template <typename T>
 __device__ __forceinline__ float row_partial(const T* __restrict__ src, int d, int lane) {
   using V = typename Vec<T>::type;
@@ -51,6 +51,12 @@ __device__ __forceinline__ float row_partial(const T* __restrict__ src, int d, i
     const V* v = reinterpret_cast<const V*>(src);
     const int nv = d / VN;
     int i = lane;
+    for (; i + 224 < nv; i += 256) {          // eight independent 16-byte loads in flight per lane
+      const V x0 = __ldg(v + i), x1 = __ldg(v + i + 32), x2 = __ldg(v + i + 64), x3 = __ldg(v + i + 96);
+      const V x4 = __ldg(v + i + 128), x5 = __ldg(v + i + 160), x6 = __ldg(v + i + 192), x7 = __ldg(v + i + 224);
+      acc0 += Vec<T>::sq(x0); acc1 += Vec<T>::sq(x1); acc2 += Vec<T>::sq(x2); acc3 += Vec<T>::sq(x3);
+      acc0 += Vec<T>::sq(x4); acc1 += Vec<T>::sq(x5); acc2 += Vec<T>::sq(x6); acc3 += Vec<T>::sq(x7);
+    }
     for (; i + 96 < nv; i += 128) {
       const V x0 = __ldg(v + i), x1 = __ldg(v + i + 32), x2 = __ldg(v + i + 64), x3 = __ldg(v + i + 96);
       acc0 += Vec<T>::sq(x0); acc1 += Vec<T>::sq(x1); acc2 += Vec<T>::sq(x2); acc3 += Vec<T>::sq(x3);
@@ -73,8 +79,26 @@ __global__ void __launch_bounds__(256) rownorm_kernel(const T* __restrict__ dY, 
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= R) return;
+  // the first four vectors per lane of the X row are requested before the dY row is touched
+  using V = typename Vec<T>::type;
+  constexpr int VN = Vec<T>::N;
+  const T* xrow = X + (size_t)row * d_in;
+  const bool xvec = (d_in % VN) == 0;
+  const int nvx = xvec ? d_in / VN : 0;
+  V xv[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    if (lane + 32 * k < nvx) xv[k] = __ldg(reinterpret_cast<const V*>(xrow) + lane + 32 * k);
   const float pa = row_partial<T>(dY + (size_t)row * d_out, d_out, lane);
-  const float pb = row_partial<T>(X + (size_t)row * d_in, d_in, lane);
+  float pb = 0.f;
+  if (xvec) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (lane + 32 * k < nvx) pb += Vec<T>::sq(xv[k]);
+    for (int i = lane + 128; i < nvx; i += 32) pb += Vec<T>::sq(__ldg(reinterpret_cast<const V*>(xrow) + i));
+  } else {
+    pb = row_partial<T>(xrow, d_in, lane);
+  }
   const float sa = warp_sum(pa), sb = warp_sum(pb);
   if (lane == 0) {
     a[row] = sa;
