@@ -307,6 +307,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t tmem_base = setup<BN>(s, warp, tid);
   volatile int* abort_flag = s.abort_flag;
+  pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
   const Decomp D = decompose<MODE, BN>(P);
 
   if (warp == 4) {
@@ -637,6 +638,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const __nv_bfloat16* __restri
                                                    const int32_t* __restrict__ idxW, const float* __restrict__ scaleW,
                                                    const int32_t* __restrict__ counts, __nv_bfloat16* __restrict__ packG,
                                                    __nv_bfloat16* __restrict__ packX, int d_out, int d_in) {
+  pdl_trigger();   // the dW product kernel may set itself up; it waits for this grid before loading
   const int cnt = counts[1];
   const int padded = (cnt + BK - 1) / BK * BK;
   const int vo = d_out / 8, vi = d_in / 8;
@@ -737,9 +739,10 @@ cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, cons
     attr_set = true;
   }
   const int grid = (int)(max_items < h->num_sms ? max_items : h->num_sms);
-  umma_kernel<MODE, BN><<<grid, NUM_THREADS, TileCfg<BN>::SMEM_BYTES, st>>>(a, b, c, P);
+  cudaError_t e = launch_after(umma_kernel<MODE, BN>, dim3(grid), dim3(NUM_THREADS), (size_t)TileCfg<BN>::SMEM_BYTES, st,
+                               a, b, c, P);
   h->launches += 1;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <int MODE>

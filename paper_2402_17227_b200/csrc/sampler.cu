@@ -135,6 +135,8 @@ struct SamplerParams {
 
 __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_kernel(SamplerParams P) {
   __shared__ Scratch sc;
+  pdl_wait();      // the row norms come from the kernel before this one
+  pdl_trigger();   // the product kernel may set itself up meanwhile
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
   const int N = P.N, T = P.T, R = N * T;
 
@@ -292,6 +294,8 @@ __device__ void capped_prop_warp(float (&v)[SLOTS], float budget) {
 template <int E, int SLOTS>
 __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerParams P) {
   __shared__ FastShared sh;
+  pdl_wait();      // the row norms come from the kernel before this one
+  pdl_trigger();   // the product kernel may set itself up meanwhile
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = P.N, T = P.T, R = N * T;
   // Element e of this thread is row (e / 4) * 4096 + tid * 4 + (e % 4): four consecutive rows per
@@ -547,23 +551,24 @@ cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st) {
   P.rho = a.rho; P.nu = a.nu; P.seed = a.seed;
   P.sample_w = a.sample_w; P.accumulate_vw = a.accumulate_vw;
   const int R = P.N * P.T;
+  cudaError_t e = cudaSuccess;
   if (P.N <= 1024 && R <= 16 * SAMPLER_THREADS) {
     const bool wide = P.N > 32;       // SampleA slots per lane of warp 0
     if (R <= 4 * SAMPLER_THREADS) {
-      if (wide) sampler_fast_kernel<4, 32><<<1, SAMPLER_THREADS, 0, st>>>(P);
-      else sampler_fast_kernel<4, 1><<<1, SAMPLER_THREADS, 0, st>>>(P);
+      if (wide) e = launch_after(sampler_fast_kernel<4, 32>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
+      else e = launch_after(sampler_fast_kernel<4, 1>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
     } else if (R <= 8 * SAMPLER_THREADS) {
-      if (wide) sampler_fast_kernel<8, 32><<<1, SAMPLER_THREADS, 0, st>>>(P);
-      else sampler_fast_kernel<8, 1><<<1, SAMPLER_THREADS, 0, st>>>(P);
+      if (wide) e = launch_after(sampler_fast_kernel<8, 32>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
+      else e = launch_after(sampler_fast_kernel<8, 1>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
     } else {
-      if (wide) sampler_fast_kernel<16, 32><<<1, SAMPLER_THREADS, 0, st>>>(P);
-      else sampler_fast_kernel<16, 1><<<1, SAMPLER_THREADS, 0, st>>>(P);
+      if (wide) e = launch_after(sampler_fast_kernel<16, 32>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
+      else e = launch_after(sampler_fast_kernel<16, 1>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
     }
   } else {
-    sampler_kernel<<<1, SAMPLER_THREADS, 0, st>>>(P);
+    e = launch_after(sampler_kernel, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
   }
   h->launches += 1;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_mask_from_probs(Handle* h, const float* p, int n, uint64_t seed, int sampler,

@@ -76,6 +76,7 @@ __global__ void __launch_bounds__(256) rownorm_kernel(const T* __restrict__ dY, 
                                                       int R, int d_out, int d_in, uint64_t seed,
                                                       float* __restrict__ a, float* __restrict__ b,
                                                       float* __restrict__ lev, uint32_t* __restrict__ u24) {
+  pdl_trigger();   // the sampling kernel may be scheduled now; it waits for this grid before reading
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= R) return;
