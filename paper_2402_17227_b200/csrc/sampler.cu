@@ -305,36 +305,37 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
   // this thread's rows: the unscaled leverage score and the SampleW uniform, both made per row by
   // the row-norm kernel
   float ab[E];
-  uint32_t ur[E];
 #pragma unroll
   for (int e = 0; e < E; e += 4) {
     const int rb = row_of(e);
     if (rb + 3 < R) {
       const float4 v = *reinterpret_cast<const float4*>(P.lev + rb);
-      const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + rb);
       ab[e] = v.x; ab[e + 1] = v.y; ab[e + 2] = v.z; ab[e + 3] = v.w;
-      ur[e] = u.x; ur[e + 1] = u.y; ur[e + 2] = u.z; ur[e + 3] = u.w;
     } else {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const bool in = rb + i < R;
-        ab[e + i] = in ? P.lev[rb + i] : 0.f;
-        ur[e + i] = in ? P.u24[rb + i] : 0xffffffffu;
-      }
+      for (int i = 0; i < 4; ++i) ab[e + i] = rb + i < R ? P.lev[rb + i] : 0.f;
     }
   }
-  // datum of each of this thread's rows: one division per group of four rows
-  int nrow[E];
+  // Datum of each of this thread's rows, one division per group of four rows, kept as one word per
+  // group (registers are scarce at 1024 threads): the first row's datum and three 2-bit increments.
+  int ncode[E / 4];
 #pragma unroll
   for (int e = 0; e < E; e += 4) {
     const int rb = row_of(e);
-    int n = rb / T, rem = rb - n * T;
+    const int n0 = rb / T;
+    int n = n0, rem = rb - n0 * T, code = n0;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      nrow[e + i] = n < N ? n : N - 1;
+    for (int i = 1; i < 4; ++i) {
       if (++rem == T) { rem = 0; ++n; }
+      code |= (n - n0) << (14 + 2 * i);
     }
+    ncode[e >> 2] = code;
   }
+  auto datum_of = [&](int e) {
+    const int code = ncode[e >> 2];
+    const int n = (code & 0xffff) + ((e & 3) ? ((code >> (14 + 2 * (e & 3))) & 3) : 0);
+    return n < N ? n : N - 1;
+  };
 
   // ---- ||G_n||_F: one warp per datum, fixed order; four independent partial sums per lane keep
   // several loads in flight (a dependent chain of T/32 loads would cost a memory latency each)
@@ -390,7 +391,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
   float w[E];
 #pragma unroll
   for (int e = 0; e < E; ++e) {
-    const int n = nrow[e];
+    const int n = datum_of(e);
     w[e] = (row_of(e) < R && sh.scaleA[n] > 0.f) ? ab[e] / sh.pA[n] : 0.f;
   }
 #pragma unroll
@@ -409,7 +410,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
 #pragma unroll
     for (int e = 0; e < E; ++e) {
       const int r = row_of(e);
-      q[e] = (r < R && sh.scaleA[nrow[e]] > 0.f) ? P.q_in[r] : 0.f;
+      q[e] = (r < R && sh.scaleA[datum_of(e)] > 0.f) ? P.q_in[r] : 0.f;
     }
   } else {
     const float budget = P.nu * (float)T * (float)cntA;
@@ -482,13 +483,28 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
   // gets its own block-wide exclusive scan of the per-thread counts, on top of the groups before it
   unsigned keepbits = 0;
 #pragma unroll
-  for (int e = 0; e < E; ++e) {
-    bool k = false;
-    if (row_of(e) < R) {
-      if (P.sample_w) k = q[e] > 0.f && ur[e] < (uint32_t)floorf(q[e] * 16777216.0f);
-      else k = sh.scaleA[nrow[e]] > 0.f;
+  for (int e = 0; e < E; e += 4) {
+    const int rb = row_of(e);
+    uint32_t ur[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};   // the rows' SampleW uniforms
+    if (P.sample_w) {
+      if (rb + 3 < R) {
+        const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + rb);
+        ur[0] = u.x; ur[1] = u.y; ur[2] = u.z; ur[3] = u.w;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (rb + i < R) ur[i] = P.u24[rb + i];
+      }
     }
-    keepbits |= (k ? 1u : 0u) << e;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      bool k = false;
+      if (rb + i < R) {
+        if (P.sample_w) k = q[e + i] > 0.f && ur[i] < (uint32_t)floorf(q[e + i] * 16777216.0f);
+        else k = sh.scaleA[datum_of(e + i)] > 0.f;
+      }
+      keepbits |= (k ? 1u : 0u) << (e + i);
+    }
   }
   int total = 0;
 #pragma unroll
@@ -516,7 +532,7 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
       if (bits & (1u << i)) {
         const int e = g4 * 4 + i;
         P.idxW[base] = row_of(e);
-        P.scaleW[base] = P.sample_w ? sh.scaleA[nrow[e]] / q[e] : sh.scaleA[nrow[e]];
+        P.scaleW[base] = P.sample_w ? sh.scaleA[datum_of(e)] / q[e] : sh.scaleA[datum_of(e)];
         ++base;
       }
   }
