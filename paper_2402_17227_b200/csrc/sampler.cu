@@ -343,6 +343,13 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     const float* an = P.a + (size_t)n * T;
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
     int t = lane;
+    for (; t + 480 < T; t += 512) {            // sixteen loads in flight per lane
+      float v[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) v[k] = an[t + 32 * k];
+#pragma unroll
+      for (int k = 0; k < 16; k += 4) { s0 += v[k]; s1 += v[k + 1]; s2 += v[k + 2]; s3 += v[k + 3]; }
+    }
     for (; t + 96 < T; t += 128) { s0 += an[t]; s1 += an[t + 32]; s2 += an[t + 64]; s3 += an[t + 96]; }
     for (; t < T; t += 32) s0 += an[t];
     const float s = warp_sum((s0 + s1) + (s2 + s3));
