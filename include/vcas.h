@@ -200,10 +200,12 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
 int vcas_last_device_status(vcas_handle h, int32_t* status);
 
 /* Tuning overrides for the tensor-core products (the paper has no counterpart): output tile
- * width of the dX and dW kernels (64, 128 or 256) and the number of slices each contraction is
- * split into (1..16; slices are combined in a fixed order, so results stay reproducible).
- * 0 = let the library choose from the shapes and ratios. */
-int vcas_set_tuning(vcas_handle h, int32_t dx_tile_n, int32_t dw_tile_n, int32_t dx_split_k, int32_t dw_split_k);
+ * width of the dX and dW kernels (64, 128 or 256), the number of slices each contraction is
+ * split into (1..16; slices are combined in a fixed order, so results stay reproducible), and
+ * the tile height (tile_m = 1: 128 rows, 2: 256 rows whenever the width is 256 and the
+ * contraction is not sliced).  0 = let the library choose from the shapes and ratios. */
+int vcas_set_tuning(vcas_handle h, int32_t dx_tile_n, int32_t dw_tile_n, int32_t dx_split_k, int32_t dw_split_k,
+                    int32_t tile_m);
 
 /* Stage timing for benchmarks (the paper has no counterpart; Sec. 6 only reports end-to-end
  * hours).  While enabled, vcas_linear_bwd(_ex) and vcas_dense_bwd record CUDA events on the

@@ -68,6 +68,7 @@ struct Handle {
   int prof_calls, prof_dense_calls;
   // tuning overrides (vcas_set_tuning); 0 = choose automatically
   int tune_dx_tile_n, tune_dw_tile_n, tune_dx_split_k, tune_dw_split_k;
+  int tune_tile_m;   // 0 auto, 1: 128-row tiles only, 2: 256-row tiles whenever the width is 256
 };
 constexpr int PROF_RING = 2048;
 

@@ -27,10 +27,15 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 constexpr int EPI_WARP_BYTES = 32 * 128;                // one staging buffer: 32 rows of 128 bytes, 128B-swizzled
 constexpr int EPI_BYTES = 4 * 2 * EPI_WARP_BYTES;       // two buffers for each of the four epilogue warps
 
-template <int BN> struct TileCfg {
+// MH = number of 128-row halves of a tile (1 or 2).  A 256-row tile reuses each B stage for two
+// accumulators, which cuts the shared-memory fill per FLOP by a third (the fill rate of one SM is
+// what bounds a 128 x 256 tile); it uses all 512 TMEM columns, so its epilogue does not overlap the
+// next main loop.  It is used for large problems only and never with a sliced contraction.
+template <int BN, int MH> struct TileCfg {
   static constexpr int B_BYTES = BN * BK * 2;
-  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int AT_BYTES = MH * A_BYTES;                       // the A part of a stage
+  static constexpr int STAGE_BYTES = AT_BYTES + B_BYTES;
+  static constexpr int STAGES = MH == 2 ? 3 : (BN == 256 ? 4 : (BN == 128 ? 6 : 8));
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + EPI_BYTES + 256 /*barriers*/;
 };
 
@@ -180,9 +185,9 @@ struct SmemLayout {
   uint8_t* epi;       // [4 warps][2][32 rows][128 B] staging for bulk / TMA stores
 };
 
-template <int BN>
+template <int BN, int MH>
 __device__ __forceinline__ SmemLayout carve(uint8_t* raw) {
-  using C = TileCfg<BN>;
+  using C = TileCfg<BN, MH>;
   SmemLayout s;
   uint8_t* base = (uint8_t*)(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
   s.stages = base;
@@ -198,9 +203,9 @@ __device__ __forceinline__ SmemLayout carve(uint8_t* raw) {
   return s;
 }
 
-template <int BN>
+template <int BN, int MH>
 __device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid) {
-  using C = TileCfg<BN>;
+  using C = TileCfg<BN, MH>;
   if (tid == 0) {
     for (int i = 0; i < C::STAGES; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&s.tmem_full[i], 1); mbar_init(&s.tmem_empty[i], 128); }
@@ -266,24 +271,25 @@ struct Decomp {
   int per_datum, ntiles;   // dX: tiles per datum; both: column tiles
 };
 
-template <int MODE, int BN>
+template <int MODE, int BN, int MH>
 __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
+  constexpr int BMT = BM * MH;
   Decomp d;
   d.ntiles = (P.d_in + BN - 1) / BN;
   if (MODE == MODE_DX) {
     const int cntA = P.dense ? P.N : P.counts[0];
-    d.per_datum = ((P.T + BM - 1) / BM) * d.ntiles;
+    d.per_datum = ((P.T + BMT - 1) / BMT) * d.ntiles;
     d.gemm_tiles = cntA * d.per_datum;
     d.zero_tiles = (P.N - cntA) * d.per_datum;
     d.kblocks = (P.d_out + BK - 1) / BK;
   } else {
     d.per_datum = 0;
-    const int tiles = ((P.d_out + BM - 1) / BM) * d.ntiles;
+    const int tiles = ((P.d_out + BMT - 1) / BMT) * d.ntiles;
     d.kblocks = (*P.cnt + BK - 1) / BK;
     d.gemm_tiles = d.kblocks > 0 ? tiles : 0;   // nothing kept: every tile is a zero tile
     d.zero_tiles = d.kblocks > 0 ? 0 : tiles;
   }
-  int S = P.split_k < 1 ? 1 : P.split_k;
+  int S = (P.split_k < 1 || MH == 2) ? 1 : P.split_k;
   if (S > d.kblocks) S = d.kblocks > 0 ? d.kblocks : 1;
   if (d.gemm_tiles > 0 && (long)d.gemm_tiles * S > P.max_units) S = P.max_units / d.gemm_tiles;
   if (S > (int)gridDim.x) S = (int)gridDim.x;
@@ -297,18 +303,20 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <int MODE, int BN>
+template <int MODE, int BN, int MH>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, GemmParams P) {
-  using C = TileCfg<BN>;
+  using C = TileCfg<BN, MH>;
+  constexpr int BMT = BM * MH;          // rows of a tile
+  constexpr int NACC = MH == 2 ? 1 : 2;  // accumulator sets in TMEM
   extern __shared__ uint8_t smem_raw[];
-  const SmemLayout s = carve<BN>(smem_raw);
+  const SmemLayout s = carve<BN, MH>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t tmem_base = setup<BN>(s, warp, tid);
+  const uint32_t tmem_base = setup<BN, MH>(s, warp, tid);
   volatile int* abort_flag = s.abort_flag;
   pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
-  const Decomp D = decompose<MODE, BN>(P);
+  const Decomp D = decompose<MODE, BN, MH>(P);
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
@@ -332,17 +340,19 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (!ok) break;
           uint8_t* sa = s.stages + stage * C::STAGE_BYTES;
           if (MODE == MODE_DX) {
-            mbar_expect_tx(&s.full[stage], (uint32_t)(P.a_tx_bytes + C::B_BYTES));
-            tma_load_3d(sa, &tmA, kb * BK, c0 * BM, n, &s.full[stage]);
+            mbar_expect_tx(&s.full[stage], (uint32_t)(MH * P.a_tx_bytes + C::B_BYTES));
+#pragma unroll
+            for (int hh = 0; hh < MH; ++hh)
+              tma_load_3d(sa + hh * A_BYTES, &tmA, kb * BK, c0 * BMT + hh * BM, n, &s.full[stage]);
           } else {
             mbar_expect_tx(&s.full[stage], C::STAGE_BYTES);
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j)
-              tma_load_2d(sa + j * CHUNK_BYTES, &tmA, c0 * BM + j * 64, kb * BK, &s.full[stage]);
+            for (int j = 0; j < BMT / 64; ++j)
+              tma_load_2d(sa + j * CHUNK_BYTES, &tmA, c0 * BMT + j * 64, kb * BK, &s.full[stage]);
           }
 #pragma unroll
           for (int j = 0; j < BN / 64; ++j)
-            tma_load_2d(sa + A_BYTES + j * CHUNK_BYTES, &tmB, c1 * BN + j * 64, kb * BK, &s.full[stage]);
+            tma_load_2d(sa + C::AT_BYTES + j * CHUNK_BYTES, &tmB, c1 * BN + j * 64, kb * BK, &s.full[stage]);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -357,22 +367,25 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi, ++lt) {
         const int slice = u % D.S;
         const int nkb = min(D.kblocks, (slice + 1) * D.kb_per) - slice * D.kb_per;
-        const int buf = lt & 1; const uint32_t use = (uint32_t)(lt >> 1) & 1u;
+        const int buf = lt % NACC; const uint32_t use = (uint32_t)(lt / NACC) & 1u;
         ok = mbar_wait(&s.tmem_empty[buf], use ^ 1u, abort_flag, P.status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);   // half hh of a 256-row tile: + hh * BN
         for (int kb = 0; kb < nkb; ++kb) {
           ok = mbar_wait(&s.full[stage], phase, abort_flag, P.status);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(s.stages + stage * C::STAGE_BYTES);
-          const uint64_t da = MODE == MODE_DW ? desc_mnmajor(sa) : desc_kmajor(sa);
-          const uint64_t db = desc_mnmajor(sa + A_BYTES);
+          const uint64_t db = desc_mnmajor(sa + C::AT_BYTES);
 #pragma unroll
-          for (int k4 = 0; k4 < BK / UMMA_K; ++k4)
-            umma_bf16(d_tmem, da + (uint64_t)(k4 * a_step), db + (uint64_t)(k4 * (UMMA_K * 128 >> 4)), idesc,
-                      (kb | k4) != 0 ? 1u : 0u);
+          for (int hh = 0; hh < MH; ++hh) {
+            const uint64_t da = MODE == MODE_DW ? desc_mnmajor(sa + hh * A_BYTES) : desc_kmajor(sa + hh * A_BYTES);
+#pragma unroll
+            for (int k4 = 0; k4 < BK / UMMA_K; ++k4)
+              umma_bf16(d_tmem + (uint32_t)(hh * BN), da + (uint64_t)(k4 * a_step),
+                        db + (uint64_t)(k4 * (UMMA_K * 128 >> 4)), idesc, (kb | k4) != 0 ? 1u : 0u);
+          }
           umma_commit(&s.empty[stage]);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -393,15 +406,15 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int k = tile / D.per_datum, rem = tile % D.per_datum;
         const int c = rem / D.ntiles, nt = rem % D.ntiles;
         const int n = is_gemm ? (P.dense ? k : P.idxA[k]) : P.dropA[k];
-        row0 = (size_t)n * P.T + (size_t)c * BM;
-        rows_valid = min(BM, P.T - c * BM);
+        row0 = (size_t)n * P.T + (size_t)c * BMT;
+        rows_valid = min(BMT, P.T - c * BMT);
         col0 = nt * BN;
-        n_out = n; t_out = c * BM;
+        n_out = n; t_out = c * BMT;
         if (is_gemm && !P.dense) sc = P.scaleA[n];
       } else {
         const int mt = tile / D.ntiles, nt = tile % D.ntiles;
-        row0 = (size_t)mt * BM;
-        rows_valid = min(BM, P.d_out - mt * BM);
+        row0 = (size_t)mt * BMT;
+        rows_valid = min(BMT, P.d_out - mt * BMT);
         col0 = nt * BN;
       }
     };
@@ -438,7 +451,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int tile = u / D.S, slice = u % D.S;
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(tile, true, row0, rows_valid, col0, sc, n_out, t_out);
-      const int buf = lt & 1; const uint32_t use = (uint32_t)(lt >> 1) & 1u;
+      const int buf = lt % NACC; const uint32_t use = (uint32_t)(lt / NACC) & 1u;
       if (!mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * BN);
@@ -446,12 +459,15 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // ---- whole contraction in this unit: accumulator -> (rescale, GELU', convert) -> swizzled
         // shared memory -> TMA store of 32 rows x 128 bytes per warp (rows / columns outside the
         // tensor are clipped by the tensor map, so rows of the next datum are never touched)
-        const bool valid = row < rows_valid;
         constexpr int COLS = MODE == MODE_DX ? 64 : 32;             // columns per 128-byte staged row
         int nbuf = 0;
 #pragma unroll 1
-        for (int j = 0; j < BN / COLS; ++j, ++nbuf) {
-          if (col0 + j * COLS >= P.d_in) break;                     // warp-uniform
+        for (int hj = 0; hj < MH * (BN / COLS); ++hj, ++nbuf) {
+          const int hh = hj / (BN / COLS), j = hj % (BN / COLS);    // 128-row half of the tile, column chunk
+          const int hrow = hh * BM + row;
+          const bool valid = hrow < rows_valid;
+          const uint32_t taddr_h = taddr + (uint32_t)(hh * BN);
+          if (col0 + j * COLS >= P.d_in) { --nbuf; continue; }      // warp-uniform
           uint8_t* buf8 = stage0 + (nbuf & 1) * EPI_WARP_BYTES;
           if (nbuf >= 2) { if (lane == 0) bulk_wait_read_1(); __syncwarp(); }
           uint4* myrow = reinterpret_cast<uint4*>(buf8 + lane * 128);
@@ -459,14 +475,14 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
               uint32_t v[32];
-              tmem_ld32(taddr + (uint32_t)(j * 64 + half * 32), v);
+              tmem_ld32(taddr_h + (uint32_t)(j * 64 + half * 32), v);
 #pragma unroll
               for (int g8 = 0; g8 < 4; ++g8) {
                 float r[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) r[e] = sc * __uint_as_float(v[g8 * 8 + e]);
                 if (P.H != nullptr && valid) {
-                  const size_t off = (row0 + row) * ld + col0 + j * 64 + half * 32 + g8 * 8;
+                  const size_t off = (row0 + hrow) * ld + col0 + j * 64 + half * 32 + g8 * 8;
                   const uint4 hv = *reinterpret_cast<const uint4*>(P.H + off);
                   const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
 #pragma unroll
@@ -483,7 +499,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
           } else {
             uint32_t v[32];
-            tmem_ld32(taddr + (uint32_t)(j * 32), v);
+            tmem_ld32(taddr_h + (uint32_t)(j * 32), v);
 #pragma unroll
             for (int g4 = 0; g4 < 8; ++g4)
               myrow[(uint32_t)g4 ^ swz] = make_uint4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
@@ -491,8 +507,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           fence_async_smem();
           __syncwarp();
           if (lane == 0) {
-            if (MODE == MODE_DX) tma_store_3d(&tmC, buf8, col0 + j * 64, t_out + warp * 32, n_out);
-            else tma_store_2d(&tmC, buf8, col0 + j * 32, (int)row0 + warp * 32);
+            if (MODE == MODE_DX) tma_store_3d(&tmC, buf8, col0 + j * 64, t_out + hh * BM + warp * 32, n_out);
+            else tma_store_2d(&tmC, buf8, col0 + j * 32, (int)row0 + hh * BM + warp * 32);
             bulk_commit();
           }
         }
@@ -610,8 +626,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     for (int z = (int)gridDim.x - 1 - (int)blockIdx.x; z < D.zero_tiles && ok; z += gridDim.x) {
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(z, false, row0, rows_valid, col0, sc, n_out, t_out);
-      if (row < rows_valid) {
-        const size_t off = (row0 + row) * ld + col0;
+#pragma unroll 1
+      for (int hh = 0; hh < MH; ++hh) {
+        const int hrow = hh * BM + row;
+        if (hrow >= rows_valid) continue;
+        const size_t off = (row0 + hrow) * ld + col0;
         if (MODE == MODE_DX) {
 #pragma unroll
           for (int j = 0; j < BN / 8; ++j)
@@ -703,17 +722,21 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
 // (the shared-memory fill rate of one SM bounds it, so narrow tiles only pay off when they fill
 // more SMs); a unit costs about 4 us of set-up, pipeline fill and output store; a sliced unit
 // about 7 us more (partial store, wait for its siblings, reduction).
-struct Plan { int bn, split; };
-Plan plan_tiles(long row_tiles, int n_extent, int kblocks, int num_sms, int max_units, int force_bn, int force_split) {
+struct Plan { int bn, split, mh; };
+// row_tiles128: number of 128-row tile rows (for dX: kept data x 128-token chunks).  A 256-row tile
+// (mh = 2) covers two of them; its k-block costs about 0.62 us for twice the work.
+Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks, int num_sms, int max_units,
+                int force_bn, int force_split) {
   const int widths[3] = {256, 128, 64};
   const double c_kb[3] = {0.50, 0.45, 0.43};
-  Plan best = {256, 1};
+  Plan best = {256, 1, 1};
   double best_t = 1e30;
   if (kblocks < 1) kblocks = 1;
   for (int i = 0; i < 3; ++i) {
     if (force_bn != 0 && widths[i] != force_bn) continue;
     if (force_bn == 0 && widths[i] > 64 && n_extent <= widths[i] / 2) continue;   // mostly padding
-    const long tiles = row_tiles * ((n_extent + widths[i] - 1) / widths[i]);
+    const long ntiles = (n_extent + widths[i] - 1) / widths[i];
+    const long tiles = row_tiles128 * ntiles;
     for (int sp = 1; sp <= 16; ++sp) {
       if (force_split != 0 && sp != force_split) continue;
       if (sp > 1 && tiles * sp > max_units) continue;
@@ -722,41 +745,46 @@ Plan plan_tiles(long row_tiles, int n_extent, int kblocks, int num_sms, int max_
       const double waves = (double)((units + num_sms - 1) / num_sms);
       const double unit_fixed = sp > 1 ? 11.0 + 0.25 * sp : 4.0;
       const double t = waves * ((double)((kblocks + sp - 1) / sp) * c_kb[i] + unit_fixed);
-      if (t < best_t - 1e-9) { best_t = t; best = {widths[i], sp}; }
+      if (t < best_t - 1e-9) { best_t = t; best = {widths[i], sp, 1}; }
+    }
+    if (widths[i] == 256 && force_split <= 1) {                        // 256 x 256 tiles, never sliced
+      const long units = row_tiles256 * ntiles;
+      const double waves = (double)((units + num_sms - 1) / num_sms);
+      const double t = waves * ((double)kblocks * 0.62 + 7.0);
+      if (t < best_t - 1e-9) { best_t = t; best = {256, 1, 2}; }
     }
   }
   return best;
 }
 
-template <int MODE, int BN>
+template <int MODE, int BN, int MH>
 cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P,
                      long max_items, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         TileCfg<BN>::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         TileCfg<BN, MH>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   const int grid = (int)(max_items < h->num_sms ? max_items : h->num_sms);
-  cudaError_t e = launch_after(umma_kernel<MODE, BN>, dim3(grid), dim3(NUM_THREADS), (size_t)TileCfg<BN>::SMEM_BYTES, st,
-                               a, b, c, P);
+  cudaError_t e = launch_after(umma_kernel<MODE, BN, MH>, dim3(grid), dim3(NUM_THREADS),
+                               (size_t)TileCfg<BN, MH>::SMEM_BYTES, st, a, b, c, P);
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <int MODE>
-cudaError_t run_gemm_bn(Handle* h, int bn, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
+cudaError_t run_gemm_bn(Handle* h, const Plan& plan, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
                         const GemmParams& P, long max_items, cudaStream_t st) {
-  switch (bn) {
-    case 256: return run_gemm<MODE, 256>(h, a, b, c, P, max_items, st);
-    case 128: return run_gemm<MODE, 128>(h, a, b, c, P, max_items, st);
-    default: return run_gemm<MODE, 64>(h, a, b, c, P, max_items, st);
+  if (plan.mh == 2) return run_gemm<MODE, 256, 2>(h, a, b, c, P, max_items, st);
+  switch (plan.bn) {
+    case 256: return run_gemm<MODE, 256, 1>(h, a, b, c, P, max_items, st);
+    case 128: return run_gemm<MODE, 128, 1>(h, a, b, c, P, max_items, st);
+    default: return run_gemm<MODE, 64, 1>(h, a, b, c, P, max_items, st);
   }
 }
 
-// which = 0: the dX product, 1: the dW product (they may run at the same time on two streams, so
-// each has its own split-contraction workspace)
 void common_params(Handle* h, GemmParams& P, int which) {
   P = GemmParams();
   P.status = h->ws.status;
@@ -799,14 +827,16 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   P.a_tx_bytes = (d.T < BM ? d.T : BM) * BK * 2;
   double kept = dense ? (double)d.N : (double)rho_hint * d.N;
   if (kept < 1.0) kept = 1.0;
-  const int chunks = (d.T + BM - 1) / BM;
-  const long row_tiles = (long)(kept + 0.5) * chunks;
-  const Plan plan = plan_tiles(row_tiles, d.d_in, (d.d_out + BK - 1) / BK, h->num_sms, h->max_units,
-                               h->tune_dx_tile_n, h->tune_dx_split_k);
+  const int chunks = (d.T + BM - 1) / BM, chunks2 = (d.T + 2 * BM - 1) / (2 * BM);
+  const long nk = (long)(kept + 0.5);
+  Plan plan = plan_tiles(nk * chunks, nk * chunks2, d.d_in, (d.d_out + BK - 1) / BK, h->num_sms, h->max_units,
+                         h->tune_dx_tile_n, h->tune_dx_split_k);
+  if (h->tune_tile_m == 1) plan.mh = 1;
+  if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
   P.split_k = plan.split;
   // upper bound of work items: every datum kept and split, or every datum a zero tile
-  const long max_items = (long)d.N * chunks * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
-  return run_gemm_bn<MODE_DX>(h, plan.bn, tmA, tmB, tmC, P, max_items, st);
+  const long max_items = (long)d.N * (plan.mh == 2 ? chunks2 : chunks) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
+  return run_gemm_bn<MODE_DX>(h, plan, tmA, tmB, tmC, P, max_items, st);
 }
 
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st) {
@@ -844,12 +874,14 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
   GemmParams P;
   common_params(h, P, 1);
   P.cnt = cnt; P.dW = dW;
-  const long mtiles = (d.d_out + BM - 1) / BM;
-  const Plan plan = plan_tiles(mtiles, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
-                               h->tune_dw_tile_n, h->tune_dw_split_k);
+  const long mtiles = (d.d_out + BM - 1) / BM, mtiles2 = (d.d_out + 2 * BM - 1) / (2 * BM);
+  Plan plan = plan_tiles(mtiles, mtiles2, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
+                         h->tune_dw_tile_n, h->tune_dw_split_k);
+  if (h->tune_tile_m == 1) plan.mh = 1;
+  if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
   P.split_k = plan.split;
-  const long max_items = mtiles * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
-  return run_gemm_bn<MODE_DW>(h, plan.bn, tmA, tmB, tmC, P, max_items, st);
+  const long max_items = (plan.mh == 2 ? mtiles2 : mtiles) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
+  return run_gemm_bn<MODE_DW>(h, plan, tmA, tmB, tmC, P, max_items, st);
 }
 
 }  // namespace vcas
