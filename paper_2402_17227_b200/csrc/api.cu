@@ -227,22 +227,32 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
-  mark(h, 0, st);
-  VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
-  mark(h, 1, st);
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
-  VCAS_CUDA(launch_sampler(h, a, st));
-  // The two products are independent once the sampler has run: the dW branch (pack + product) is
-  // forked onto the handle's side stream and joined back before the call's work ends on `st`.
+  a.a_done = fast_sampling(h->desc) ? 1 : 0;
+  // The two products are independent: the dW branch (SampleW, pack, product) is forked onto the
+  // handle's side stream and joined back before the call's work ends on `st`.  When SampleA runs in
+  // the tail of the row-norm kernel the fork comes right after that kernel, so that the dX product,
+  // which needs only the kept data, overlaps the whole of SampleW; otherwise after the sampler.
   // (While stage profiling is on, everything stays on `st` so that each pair of events brackets
   // one kernel.)
-  cudaStream_t sw = st;
   const bool fork = h->tensor_path && !h->prof_enabled;
-  if (fork) {
+  cudaStream_t sw = st;
+  mark(h, 0, st);
+  VCAS_CUDA(launch_rownorms(h, dY, X, seed, a.a_done ? &a : nullptr, st));
+  mark(h, 1, st);
+  if (fork && a.a_done) {
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
     sw = h->side_stream;
+    VCAS_CUDA(launch_sampler(h, a, sw, true));
+  } else {
+    VCAS_CUDA(launch_sampler(h, a, st));
+    if (fork) {
+      VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
+      VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+      sw = h->side_stream;
+    }
   }
   mark(h, 2, st);
   if (h->tensor_path) {
@@ -315,9 +325,10 @@ int vcas_score(vcas_handle hh, const void* X, const void* dY, float rho, float n
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
-  VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 1; a.accumulate_vw = 0;
+  a.a_done = fast_sampling(h->desc) ? 1 : 0;
+  VCAS_CUDA(launch_rownorms(h, dY, X, seed, a.a_done ? &a : nullptr, st));
   VCAS_CUDA(launch_sampler(h, a, st));
   return copy_out(h, g, p, w, q, idxA, cntA, idxW, cntW, st);
 }
@@ -354,10 +365,10 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
     int rc = dense_dw(h, X_i[i], dY_i[i], h->ws.Gs, st);            // G_s,i
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(launch_probe_welford(h, i, st));
-    VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, st));   // the probe draws no SampleW mask
+    VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, nullptr, st));   // the probe draws no SampleW mask
     for (int j = 0; j < M; ++j) {
       SamplerArgs a;
-      a.rho = rho; a.nu = nu; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 0; a.accumulate_vw = 1;
+      a.rho = rho; a.nu = nu; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 0; a.accumulate_vw = 1; a.a_done = 0;
       a.seed = seed + (uint64_t)(i * M + j + 1) * 0x9E3779B97F4A7C15ull;
       VCAS_CUDA(launch_sampler(h, a, st));
       if (j == 0) VCAS_CUDA(launch_probe_sparsity(h, s_lo, s_hi, st));

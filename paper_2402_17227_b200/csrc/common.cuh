@@ -28,7 +28,7 @@ struct Workspace {
   int32_t* idxA;   // [N]  kept data, ascending
   int32_t* dropA;  // [N]  dropped data, ascending
   int32_t* idxW;   // [R]  kept rows, ascending
-  int32_t* counts; // [8]  0: cntA, 1: cntW, 2: R (constant, for dense launches), 4: reduction ticket
+  int32_t* counts; // [8]  0: cntA, 1: cntW, 2: R (constant, for dense launches), 4: reduction ticket, 5: row-norm ticket
   int32_t* status; // [1]  device status word
   double* acc;     // [16] probe accumulators (0: V_act, 1: V_w, 2: p_lo, 3: p_hi, 4: V_s)
   double* partial; // [PARTIAL_SLOTS] block partial sums of the probe reductions
@@ -135,11 +135,136 @@ __device__ __forceinline__ int warp_sum(int v) {
 }
 
 // ---------------------------------------------------------------------------------------
+// SampleA inside one warp (Sec. 4.1), shared by the sampling kernel and the tail of the row-norm kernel.
+// ---------------------------------------------------------------------------------------
+// Sum of the T squared row norms of one datum by one warp, in a fixed order, result in every lane.  Up to
+// sixteen independent loads per lane are in flight (a dependent chain of T/32 loads would cost a memory
+// latency each).  The loads bypass L1: the values may have been written by other SMs of the same grid.
+__device__ __forceinline__ float datum_sqnorm_warp(const float* an, int T, int lane) {
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+  int t = lane;
+  for (; t + 480 < T; t += 512) {
+    float v[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) v[k] = __ldcg(an + t + 32 * k);
+#pragma unroll
+    for (int k = 0; k < 16; k += 4) { s0 += v[k]; s1 += v[k + 1]; s2 += v[k + 2]; s3 += v[k + 3]; }
+  }
+  for (; t + 96 < T; t += 128) {
+    s0 += __ldcg(an + t); s1 += __ldcg(an + t + 32); s2 += __ldcg(an + t + 64); s3 += __ldcg(an + t + 96);
+  }
+  for (; t < T; t += 32) s0 += __ldcg(an + t);
+  return warp_sum((s0 + s1) + (s2 + s3));
+}
+
+// Keep probabilities proportional to v, capped at 1, summing to `budget` (the minimiser of
+// sum (1-p)/p v^2 under that budget): p = min(1, c v).  The saturated set is grown from empty; c only
+// increases, so the iteration reaches the least fixed point, which is the unique solution.  Value i of the
+// array sits in lane i % 32, slot i / 32 of ONE warp; p is returned in place of v.
+template <int SLOTS>
+__device__ __forceinline__ void capped_prop_warp(float (&v)[SLOTS], float budget) {
+  float S = 0.f;
+  int nz = 0;
+#pragma unroll
+  for (int j = 0; j < SLOTS; ++j)
+    if (v[j] > 0.f) { S += v[j]; ++nz; }
+  S = warp_sum(S);
+  nz = warp_sum(nz);
+  if (nz == 0 || budget <= 0.f) {
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j) v[j] = 0.f;
+    return;
+  }
+  if ((float)nz <= budget) {
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j) v[j] = v[j] > 0.f ? 1.f : 0.f;
+    return;
+  }
+  float c = budget / S;
+  int k = 0;
+  for (int iter = 0; iter < 128; ++iter) {
+    float Su = 0.f;
+    int ks = 0;
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j)
+      if (v[j] > 0.f) {
+        if (c * v[j] >= 1.0f) ++ks; else Su += v[j];
+      }
+    Su = warp_sum(Su);
+    ks = warp_sum(ks);
+    if (ks == k) break;
+    k = ks;
+    if (Su > 0.f) {
+      const float cn = (budget - (float)k) / Su;
+      c = cn > c ? cn : c;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < SLOTS; ++j) {
+    float r = 0.f;
+    if (v[j] > 0.f) {
+      const float cx = c * v[j];
+      r = cx >= 1.0f ? 1.f : cx;
+    }
+    v[j] = r;
+  }
+}
+
+// Where SampleA's results go: the workspace arrays, and optionally shared-memory copies of p and 1/p.
+struct SampleAOut {
+  float* p; float* scaleA; int32_t* idxA; int32_t* dropA;
+  float* sh_p; float* sh_scaleA;
+};
+
+// SampleA over N <= 32 * SLOTS data by one full warp: keep probabilities from the data norms g (or the
+// given p_in), Philox masks (sampler 0), kept and dropped lists in ascending order.  Returns the number
+// of kept data in every lane.
+template <int SLOTS>
+__device__ __forceinline__ int sample_a_warp(const float* g, int N, float rho, const float* p_in, uint64_t seed,
+                                             const SampleAOut& o, int lane) {
+  float v[SLOTS];
+  if (p_in != nullptr) {
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j) { const int n = lane + 32 * j; v[j] = n < N ? p_in[n] : 0.f; }
+  } else {
+#pragma unroll
+    for (int j = 0; j < SLOTS; ++j) { const int n = lane + 32 * j; v[j] = n < N ? g[n] : 0.f; }
+    capped_prop_warp<SLOTS>(v, (float)N * rho);
+  }
+  int kept_before = 0, drop_before = 0;
+#pragma unroll
+  for (int j = 0; j < SLOTS; ++j) {
+    const int n = lane + 32 * j;
+    const bool in = n < N;
+    const bool keep = in && bernoulli_keep(v[j], seed, 0u, (uint64_t)n);
+    const unsigned bk = __ballot_sync(0xffffffffu, keep);
+    const unsigned bd = __ballot_sync(0xffffffffu, in && !keep);
+    const unsigned lower = (1u << lane) - 1u;
+    if (in) {
+      const float sc = keep ? 1.0f / v[j] : 0.f;
+      o.p[n] = v[j];
+      o.scaleA[n] = sc;
+      if (o.sh_p != nullptr) { o.sh_p[n] = v[j]; o.sh_scaleA[n] = sc; }
+      if (keep) o.idxA[kept_before + __popc(bk & lower)] = n;
+      else o.dropA[drop_before + __popc(bd & lower)] = n;
+    }
+    kept_before += __popc(bk);
+    drop_before += __popc(bd);
+  }
+  return kept_before;
+}
+
+// The single-CTA register-resident sampling kernel, and with it SampleA in the tail of the row-norm
+// kernel, serve layers of at most this many data and rows.
+constexpr int FAST_MAX_N = 1024;
+constexpr int FAST_MAX_R = 16 * 1024;
+inline bool fast_sampling(const vcas_layer_desc& d) {
+  return d.N <= FAST_MAX_N && (long long)d.N * d.T <= FAST_MAX_R;
+}
+
+// ---------------------------------------------------------------------------------------
 // Launchers (one per .cu file).  All enqueue on `st` and return a cudaError_t.
 // ---------------------------------------------------------------------------------------
-// seed: the call's seed (the SampleW uniforms are drawn here, one per row)
-cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, cudaStream_t st);
-
 struct SamplerArgs {
   float rho, nu;
   uint64_t seed;
@@ -147,8 +272,15 @@ struct SamplerArgs {
   const float* q_in;
   int sample_w;      // 1: SampleW mask applied; 0: all rows of kept data survive (probe)
   int accumulate_vw; // 1: add Eq. 3 at ratio nu to acc[1]
+  int a_done;        // 1: SampleA's results are already in the workspace (row-norm kernel's tail)
 };
-cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st);
+// seed: the call's seed (the SampleW uniforms are drawn here, one per row).  tail != nullptr and
+// fast_sampling(desc): the last CTA to finish also runs SampleA with tail's rho, p_in and seed, so that
+// the dX product can follow directly; the caller then passes a_done = 1 to launch_sampler.
+cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, const SamplerArgs* tail,
+                            cudaStream_t st);
+// after_event: launched plainly (its inputs come through an event from another stream)
+cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st, bool after_event = false);
 cudaError_t launch_mask_from_probs(Handle* h, const float* p, int n, uint64_t seed, int sampler,
                                    uint8_t* keep, int32_t* idx, int32_t* cnt, cudaStream_t st);
 

@@ -657,6 +657,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const __nv_bfloat16* __restri
                                                    const int32_t* __restrict__ idxW, const float* __restrict__ scaleW,
                                                    const int32_t* __restrict__ counts, __nv_bfloat16* __restrict__ packG,
                                                    __nv_bfloat16* __restrict__ packX, int d_out, int d_in) {
+  pdl_wait();      // the kept rows come from the sampling kernel before this one
   pdl_trigger();   // the dW product kernel may set itself up; it waits for this grid before loading
   const int cnt = counts[1];
   const int padded = (cnt + BK - 1) / BK * BK;
@@ -843,10 +844,11 @@ cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t s
   const vcas_layer_desc& d = h->desc;
   int blocks = h->num_sms * 8;
   if (blocks > h->R_pad) blocks = h->R_pad;
-  pack_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dY, (const __nv_bfloat16*)X, h->ws.idxW, h->ws.scaleW,
-                                      h->ws.counts, h->ws.packG, h->ws.packX, d.d_out, d.d_in);
+  const cudaError_t e = launch_after(pack_kernel, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)dY,
+                                     (const __nv_bfloat16*)X, h->ws.idxW, h->ws.scaleW, h->ws.counts, h->ws.packG,
+                                     h->ws.packX, d.d_out, d.d_in);
   h->launches += 1;
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity, const int32_t* cnt,

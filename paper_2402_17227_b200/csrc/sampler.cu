@@ -8,6 +8,7 @@ namespace vcas {
 namespace {
 
 constexpr int SAMPLER_THREADS = 1024;
+static_assert(FAST_MAX_N <= SAMPLER_THREADS && FAST_MAX_R == 16 * SAMPLER_THREADS, "fast sampling limits");
 
 struct Scratch {
   double d[32];
@@ -130,7 +131,7 @@ struct SamplerParams {
   int N, T;
   float rho, nu;
   uint64_t seed;
-  int sample_w, accumulate_vw;
+  int sample_w, accumulate_vw, a_done;
 };
 
 __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_kernel(SamplerParams P) {
@@ -240,57 +241,6 @@ __device__ __forceinline__ void fast_sum(float& s, int& c, FastShared* sh, int p
   c = sh->tot_i[parity];
 }
 
-// capped_prop over at most 32 values per lane of ONE warp (value i of the array sits in lane i % 32,
-// slot i / 32); p is returned in place of v.
-template <int SLOTS>
-__device__ void capped_prop_warp(float (&v)[SLOTS], float budget) {
-  float S = 0.f;
-  int nz = 0;
-#pragma unroll
-  for (int j = 0; j < SLOTS; ++j)
-    if (v[j] > 0.f) { S += v[j]; ++nz; }
-  S = warp_sum(S);
-  nz = warp_sum(nz);
-  if (nz == 0 || budget <= 0.f) {
-#pragma unroll
-    for (int j = 0; j < SLOTS; ++j) v[j] = 0.f;
-    return;
-  }
-  if ((float)nz <= budget) {
-#pragma unroll
-    for (int j = 0; j < SLOTS; ++j) v[j] = v[j] > 0.f ? 1.f : 0.f;
-    return;
-  }
-  float c = budget / S;
-  int k = 0;
-  for (int iter = 0; iter < 128; ++iter) {
-    float Su = 0.f;
-    int ks = 0;
-#pragma unroll
-    for (int j = 0; j < SLOTS; ++j)
-      if (v[j] > 0.f) {
-        if (c * v[j] >= 1.0f) ++ks; else Su += v[j];
-      }
-    Su = warp_sum(Su);
-    ks = warp_sum(ks);
-    if (ks == k) break;
-    k = ks;
-    if (Su > 0.f) {
-      const float cn = (budget - (float)k) / Su;
-      c = cn > c ? cn : c;
-    }
-  }
-#pragma unroll
-  for (int j = 0; j < SLOTS; ++j) {
-    float r = 0.f;
-    if (v[j] > 0.f) {
-      const float cx = c * v[j];
-      r = cx >= 1.0f ? 1.f : cx;
-    }
-    v[j] = r;
-  }
-}
-
 template <int E, int SLOTS>
 __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerParams P) {
   __shared__ FastShared sh;
@@ -337,59 +287,25 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     return n < N ? n : N - 1;
   };
 
-  // ---- ||G_n||_F: one warp per datum, fixed order; four independent partial sums per lane keep
-  // several loads in flight (a dependent chain of T/32 loads would cost a memory latency each)
-  for (int n = warp; n < N; n += 32) {
-    const float* an = P.a + (size_t)n * T;
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-    int t = lane;
-    for (; t + 480 < T; t += 512) {            // sixteen loads in flight per lane
-      float v[16];
-#pragma unroll
-      for (int k = 0; k < 16; ++k) v[k] = an[t + 32 * k];
-#pragma unroll
-      for (int k = 0; k < 16; k += 4) { s0 += v[k]; s1 += v[k + 1]; s2 += v[k + 2]; s3 += v[k + 3]; }
+  if (P.a_done) {
+    // SampleA already ran in the tail of the row-norm kernel: fetch its results
+    for (int n = tid; n < N; n += SAMPLER_THREADS) { sh.scaleA[n] = P.scaleA[n]; sh.pA[n] = P.p[n]; }
+    if (tid == 0) sh.cntA = P.counts[0];
+  } else {
+    // ---- ||G_n||_F: one warp per datum, fixed order
+    for (int n = warp; n < N; n += 32) {
+      const float s = datum_sqnorm_warp(P.a + (size_t)n * T, T, lane);
+      if (lane == 0) { const float g = sqrtf(s); P.g[n] = g; sh.pA[n] = g; }
     }
-    for (; t + 96 < T; t += 128) { s0 += an[t]; s1 += an[t + 32]; s2 += an[t + 64]; s3 += an[t + 96]; }
-    for (; t < T; t += 32) s0 += an[t];
-    const float s = warp_sum((s0 + s1) + (s2 + s3));
-    if (lane == 0) { const float g = sqrtf(s); P.g[n] = g; sh.pA[n] = g; }
-  }
-  __syncthreads();
-
-  // ---- SampleA inside warp 0 (Sec. 4.1): p_n, mask, kept / dropped lists
-  if (warp == 0) {
-    float v[SLOTS];
-#pragma unroll
-    for (int j = 0; j < SLOTS; ++j) { const int n = lane + 32 * j; v[j] = n < N ? sh.pA[n] : 0.f; }
-    if (P.p_in != nullptr) {
-#pragma unroll
-      for (int j = 0; j < SLOTS; ++j) { const int n = lane + 32 * j; v[j] = n < N ? P.p_in[n] : 0.f; }
-    } else {
-      capped_prop_warp<SLOTS>(v, (float)N * P.rho);
+    __syncthreads();
+    // ---- SampleA inside warp 0 (Sec. 4.1): p_n, mask, kept / dropped lists
+    if (warp == 0) {
+      SampleAOut o;
+      o.p = P.p; o.scaleA = P.scaleA; o.idxA = P.idxA; o.dropA = P.dropA;
+      o.sh_p = sh.pA; o.sh_scaleA = sh.scaleA;
+      const int kept = sample_a_warp<SLOTS>(sh.pA, N, P.rho, P.p_in, P.seed, o, lane);
+      if (lane == 0) sh.cntA = kept;
     }
-    int kept_before = 0, drop_before = 0;
-#pragma unroll
-    for (int j = 0; j < SLOTS; ++j) {
-      const int n = lane + 32 * j;
-      const bool in = n < N;
-      const bool keep = in && bernoulli_keep(v[j], P.seed, 0u, (uint64_t)n);
-      const unsigned bk = __ballot_sync(0xffffffffu, keep);
-      const unsigned bd = __ballot_sync(0xffffffffu, in && !keep);
-      const unsigned lower = (1u << lane) - 1u;
-      if (in) {
-        P.p[n] = v[j];
-        const float sc = keep ? 1.0f / v[j] : 0.f;
-        P.scaleA[n] = sc;
-        sh.scaleA[n] = sc;
-        sh.pA[n] = v[j];
-        if (keep) P.idxA[kept_before + __popc(bk & lower)] = n;
-        else P.dropA[drop_before + __popc(bd & lower)] = n;
-      }
-      kept_before += __popc(bk);
-      drop_before += __popc(bd);
-    }
-    if (lane == 0) sh.cntA = kept_before;
   }
   __syncthreads();
   const int cntA = sh.cntA;
@@ -543,7 +459,10 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
         ++base;
       }
   }
-  if (tid == 0) { P.counts[0] = cntA; P.counts[1] = total; }
+  if (tid == 0) {
+    if (!P.a_done) P.counts[0] = cntA;
+    P.counts[1] = total;
+  }
 }
 
 __global__ void __launch_bounds__(SAMPLER_THREADS)
@@ -562,7 +481,7 @@ mask_kernel(const float* __restrict__ p, int n, uint64_t seed, int sampler, uint
 
 }  // namespace
 
-cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st) {
+cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st, bool after_event) {
   const Workspace& ws = h->ws;
   SamplerParams P;
   P.a = ws.a; P.b = ws.b; P.lev = ws.lev; P.u24 = ws.u24; P.g = ws.g; P.p = ws.p; P.w = ws.w; P.q = ws.q;
@@ -573,22 +492,22 @@ cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st) {
   P.N = h->desc.N; P.T = h->desc.T;
   P.rho = a.rho; P.nu = a.nu; P.seed = a.seed;
   P.sample_w = a.sample_w; P.accumulate_vw = a.accumulate_vw;
+  P.a_done = a.a_done && fast_sampling(h->desc);
   const int R = P.N * P.T;
   cudaError_t e = cudaSuccess;
-  if (P.N <= 1024 && R <= 16 * SAMPLER_THREADS) {
+  // after_event: the kernel before this one in the stream is not the producer of its inputs (those
+  // arrive through an event from another stream), so it is launched without the programmatic attribute
+  auto go = [&](void (*k)(SamplerParams)) {
+    if (after_event) { k<<<1, SAMPLER_THREADS, 0, st>>>(P); return cudaSuccess; }
+    return launch_after(k, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
+  };
+  if (fast_sampling(h->desc)) {
     const bool wide = P.N > 32;       // SampleA slots per lane of warp 0
-    if (R <= 4 * SAMPLER_THREADS) {
-      if (wide) e = launch_after(sampler_fast_kernel<4, 32>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
-      else e = launch_after(sampler_fast_kernel<4, 1>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
-    } else if (R <= 8 * SAMPLER_THREADS) {
-      if (wide) e = launch_after(sampler_fast_kernel<8, 32>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
-      else e = launch_after(sampler_fast_kernel<8, 1>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
-    } else {
-      if (wide) e = launch_after(sampler_fast_kernel<16, 32>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
-      else e = launch_after(sampler_fast_kernel<16, 1>, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
-    }
+    if (R <= 4 * SAMPLER_THREADS) e = go(wide ? sampler_fast_kernel<4, 32> : sampler_fast_kernel<4, 1>);
+    else if (R <= 8 * SAMPLER_THREADS) e = go(wide ? sampler_fast_kernel<8, 32> : sampler_fast_kernel<8, 1>);
+    else e = go(wide ? sampler_fast_kernel<16, 32> : sampler_fast_kernel<16, 1>);
   } else {
-    e = launch_after(sampler_kernel, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
+    e = go(sampler_kernel);
   }
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
