@@ -256,7 +256,9 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   }
   mark(h, 2, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, st));
+    // the sampling kernel on the side stream is one CTA that needs a whole SM's registers: the
+    // persistent dX grid, which starts first, leaves it one
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, fork && a.a_done ? 1 : 0, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, h->ws.scaleA, Hpre, dX, st));
   }
@@ -302,7 +304,7 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
   }
   mark_dense(h, 0, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }

@@ -291,8 +291,9 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
                           const float* scale, const int32_t* cnt, float* dW, cudaStream_t st);
 
 // tensor-core products
+// spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it)
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, cudaStream_t st);
+                           const void* H, void* dX, int spare_sms, cudaStream_t st);
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling
