@@ -230,55 +230,59 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
   a.a_done = fast_sampling(h->desc) ? 1 : 0;
-  // The two products are independent: the dW branch (SampleW, pack, product) is forked onto the
-  // handle's side stream and joined back before the call's work ends on `st`.  When SampleA runs in
-  // the tail of the row-norm kernel the fork comes right after that kernel, so that the dX product,
-  // which needs only the kept data, overlaps the whole of SampleW; otherwise after the sampler.
-  // (While stage profiling is on, everything stays on `st` so that each pair of events brackets
-  // one kernel.)
-  const bool fork = h->tensor_path && !h->prof_enabled;
-  cudaStream_t sw = st;
-  mark(h, 0, st);
-  VCAS_CUDA(launch_rownorms(h, dY, X, seed, a.a_done ? &a : nullptr, st));
-  mark(h, 1, st);
-  if (fork && a.a_done) {
-    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
-    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-    sw = h->side_stream;
-    VCAS_CUDA(launch_sampler(h, a, sw, true));
-  } else {
+  const int hint = (int)(rho * nu * (float)(h->desc.N * h->desc.T)) + 1;
+  if (!h->tensor_path) {
+    mark(h, 0, st);
+    VCAS_CUDA(launch_rownorms(h, dY, X, seed, a.a_done ? &a : nullptr, st));
+    mark(h, 1, st);
     VCAS_CUDA(launch_sampler(h, a, st));
-    if (fork) {
-      VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
-      VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-      sw = h->side_stream;
-    }
-  }
-  mark(h, 2, st);
-  if (h->tensor_path) {
-    // the sampling kernel on the side stream is one CTA that needs a whole SM's registers: the
-    // persistent dX grid, which starts first, leaves it one
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, fork && a.a_done ? 1 : 0, st));
-  } else {
+    mark(h, 2, st);
     VCAS_CUDA(launch_fma_dx(h, dY, W, h->ws.scaleA, Hpre, dX, st));
-  }
-  mark(h, 3, st);
-  if (h->tensor_path) {
-    mark(h, 6, sw);
-    VCAS_CUDA(launch_pack(h, dY, X, sw));
-    mark(h, 4, sw);
-    const int hint = (int)(rho * nu * (float)(h->desc.N * h->desc.T)) + 1;
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, sw));
-    mark(h, 5, sw);
-    if (fork) {
-      VCAS_CUDA(cudaEventRecord(h->ev_join, sw));
-      VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
-    }
-  } else {
+    mark(h, 3, st);
     mark(h, 6, st);
     mark(h, 4, st);
     VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, dW, st));
     mark(h, 5, st);
+  } else if (h->prof_enabled) {
+    // stage profiling: everything on `st`, so that each pair of events brackets one kernel
+    mark(h, 0, st);
+    VCAS_CUDA(launch_rownorms(h, dY, X, seed, a.a_done ? &a : nullptr, st));
+    mark(h, 1, st);
+    VCAS_CUDA(launch_sampler(h, a, st));
+    mark(h, 2, st);
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, st));
+    mark(h, 3, st);
+    mark(h, 6, st);
+    VCAS_CUDA(launch_pack(h, dY, X, st));
+    mark(h, 4, st);
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, st));
+    mark(h, 5, st);
+  } else if (a.a_done) {
+    // SampleA ran in the tail of the row-norm kernel, and the dX product needs nothing else: it is
+    // forked onto the handle's side stream right after that kernel and overlaps SampleW, the pack
+    // and the dW product, which stay on `st` as a chain of programmatic dependent launches (the
+    // longer of the two branches).  The dX grid leaves one SM free: the sampling kernel is a single
+    // CTA that needs a whole SM's registers.
+    VCAS_CUDA(launch_rownorms(h, dY, X, seed, &a, st));
+    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
+    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+    VCAS_CUDA(launch_sampler(h, a, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, h->side_stream));
+    VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
+    VCAS_CUDA(launch_pack(h, dY, X, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, st));
+    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
+  } else {
+    // large layers (generic sampling kernel): the products fork once the sampler has run
+    VCAS_CUDA(launch_rownorms(h, dY, X, seed, nullptr, st));
+    VCAS_CUDA(launch_sampler(h, a, st));
+    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
+    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, st));
+    VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, h->side_stream));
+    VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
+    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   }
   if (h->prof_enabled && h->prof_calls < PROF_RING) h->prof_calls += 1;
   return VCAS_OK;
@@ -304,7 +308,7 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
   }
   mark_dense(h, 0, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, false, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }

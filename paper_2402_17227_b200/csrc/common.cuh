@@ -103,8 +103,11 @@ __device__ __forceinline__ bool bernoulli_keep(float p, uint64_t seed, uint32_t 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// programmatic = false: an ordinary launch (for a kernel whose inputs arrive through an event from
+// another stream rather than from the kernel before it in its own stream).
 template <typename... KArgs, typename... Args>
-cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+cudaError_t launch_maybe_after(bool programmatic, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                               cudaStream_t st, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -114,8 +117,12 @@ cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = programmatic ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  return launch_maybe_after(true, kernel, grid, block, smem, st, args...);
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -291,9 +298,10 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
                           const float* scale, const int32_t* cnt, float* dW, cudaStream_t st);
 
 // tensor-core products
-// spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it)
+// spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it);
+// after_event: launched plainly (its inputs come through an event from another stream)
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, int spare_sms, cudaStream_t st);
+                           const void* H, void* dX, int spare_sms, bool after_event, cudaStream_t st);
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling

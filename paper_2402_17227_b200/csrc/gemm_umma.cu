@@ -760,7 +760,7 @@ Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks,
 
 template <int MODE, int BN, int MH>
 cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P,
-                     long max_items, int ctas, cudaStream_t st) {
+                     long max_items, int ctas, bool pdl, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -769,20 +769,20 @@ cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, cons
     attr_set = true;
   }
   const int grid = (int)(max_items < ctas ? max_items : ctas);
-  cudaError_t e = launch_after(umma_kernel<MODE, BN, MH>, dim3(grid), dim3(NUM_THREADS),
-                               (size_t)TileCfg<BN, MH>::SMEM_BYTES, st, a, b, c, P);
+  cudaError_t e = launch_maybe_after(pdl, umma_kernel<MODE, BN, MH>, dim3(grid), dim3(NUM_THREADS),
+                                     (size_t)TileCfg<BN, MH>::SMEM_BYTES, st, a, b, c, P);
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <int MODE>
 cudaError_t run_gemm_bn(Handle* h, const Plan& plan, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
-                        const GemmParams& P, long max_items, int ctas, cudaStream_t st) {
-  if (plan.mh == 2) return run_gemm<MODE, 256, 2>(h, a, b, c, P, max_items, ctas, st);
+                        const GemmParams& P, long max_items, int ctas, bool pdl, cudaStream_t st) {
+  if (plan.mh == 2) return run_gemm<MODE, 256, 2>(h, a, b, c, P, max_items, ctas, pdl, st);
   switch (plan.bn) {
-    case 256: return run_gemm<MODE, 256, 1>(h, a, b, c, P, max_items, ctas, st);
-    case 128: return run_gemm<MODE, 128, 1>(h, a, b, c, P, max_items, ctas, st);
-    default: return run_gemm<MODE, 64, 1>(h, a, b, c, P, max_items, ctas, st);
+    case 256: return run_gemm<MODE, 256, 1>(h, a, b, c, P, max_items, ctas, pdl, st);
+    case 128: return run_gemm<MODE, 128, 1>(h, a, b, c, P, max_items, ctas, pdl, st);
+    default: return run_gemm<MODE, 64, 1>(h, a, b, c, P, max_items, ctas, pdl, st);
   }
 }
 
@@ -799,7 +799,7 @@ void common_params(Handle* h, GemmParams& P, int which) {
 }  // namespace
 
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint, const void* H,
-                           void* dX, int spare_sms, cudaStream_t st) {
+                           void* dX, int spare_sms, bool after_event, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -838,7 +838,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   P.split_k = plan.split;
   // upper bound of work items: every datum kept and split, or every datum a zero tile
   const long max_items = (long)d.N * (plan.mh == 2 ? chunks2 : chunks) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
-  return run_gemm_bn<MODE_DX>(h, plan, tmA, tmB, tmC, P, max_items, ctas, st);
+  return run_gemm_bn<MODE_DX>(h, plan, tmA, tmB, tmC, P, max_items, ctas, !after_event, st);
 }
 
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st) {
@@ -884,7 +884,7 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
   if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
   P.split_k = plan.split;
   const long max_items = (plan.mh == 2 ? mtiles2 : mtiles) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
-  return run_gemm_bn<MODE_DW>(h, plan, tmA, tmB, tmC, P, max_items, h->num_sms, st);
+  return run_gemm_bn<MODE_DW>(h, plan, tmA, tmB, tmC, P, max_items, h->num_sms, true, st);
 }
 
 }  // namespace vcas

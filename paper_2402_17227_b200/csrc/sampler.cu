@@ -266,6 +266,27 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
       for (int i = 0; i < 4; ++i) ab[e + i] = rb + i < R ? P.lev[rb + i] : 0.f;
     }
   }
+  // The rows' SampleW uniforms: requested now, together with the scores, when the registers allow it
+  // (E <= 8); with E = 16 they are loaded just before the masks are drawn.
+  constexpr bool EARLY_U = E <= 8;
+  uint32_t ue[EARLY_U ? E : 4];
+  if (EARLY_U) {
+#pragma unroll
+    for (int e = 0; e < (EARLY_U ? E : 4); e += 4) {
+      const int rb = row_of(e);
+      ue[e] = ue[e + 1] = ue[e + 2] = ue[e + 3] = 0xffffffffu;
+      if (P.sample_w) {
+        if (rb + 3 < R) {
+          const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + rb);
+          ue[e] = u.x; ue[e + 1] = u.y; ue[e + 2] = u.z; ue[e + 3] = u.w;
+        } else {
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            if (rb + i < R) ue[e + i] = P.u24[rb + i];
+        }
+      }
+    }
+  }
   // Datum of each of this thread's rows, one division per group of four rows, kept as one word per
   // group (registers are scarce at 1024 threads): the first row's datum and three 2-bit increments.
   int ncode[E / 4];
@@ -409,7 +430,10 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
   for (int e = 0; e < E; e += 4) {
     const int rb = row_of(e);
     uint32_t ur[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};   // the rows' SampleW uniforms
-    if (P.sample_w) {
+    if (EARLY_U) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) ur[i] = ue[(EARLY_U ? e : 0) + i];
+    } else if (P.sample_w) {
       if (rb + 3 < R) {
         const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + rb);
         ur[0] = u.x; ur[1] = u.y; ur[2] = u.z; ur[3] = u.w;
