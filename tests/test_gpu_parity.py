@@ -137,15 +137,17 @@ def test_linear_bwd_given_oracle_probabilities(name, dtype, path, shape):
     layer.close()
 
 
-@pytest.mark.parametrize("tile_n,split,tile_m", [(256, 3, 1), (128, 2, 1), (64, 5, 1), (256, 16, 1), (256, 1, 1),
-                                                 (64, 1, 1), (256, 1, 2), (256, 0, 2)])
-def test_tensor_path_split_contraction_and_tile_widths(tile_n, split, tile_m):
-    """Every tile width and a contraction cut into slices (combined in a fixed order) give the same
+@pytest.mark.parametrize("tile_n,split,tile_m,exchange", [
+    (256, 3, 1, 1), (128, 2, 1, 1), (64, 5, 1, 1), (256, 16, 1, 0), (256, 1, 1, 0), (64, 1, 1, 0), (256, 1, 2, 0),
+    (256, 0, 2, 0), (256, 2, 1, 2), (256, 3, 1, 2), (128, 4, 1, 2), (64, 5, 1, 2), (128, 8, 1, 2), (256, 4, 1, 0)])
+def test_tensor_path_split_contraction_and_tile_widths(tile_n, split, tile_m, exchange):
+    """Every tile width and a contraction cut into slices (combined in a fixed order; exchanged through the
+    workspace or inside thread-block clusters, some slices empty when the contraction is short) give the same
     results within tolerance, for the sampled and the dense products; repeated runs are bit-identical."""
     N, T, d_in, d_out = 5, 197, 320, 448
     X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.5, sigma_B=1.0)
     layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
-    layer.set_tuning(tile_n, tile_n, split, split, tile_m)
+    layer.set_tuning(tile_n, tile_n, split, split, tile_m, exchange)
     Xc, dYc, Wc = cuda(X, dY, W)
     ref = o.linear_bwd(np64(X), np64(dY), np64(W), N, T, 0.5, 0.5, 4)
     p_in, q_in = torch.from_numpy(ref["p32"]).cuda(), torch.from_numpy(ref["q32"]).cuda()
