@@ -914,11 +914,13 @@ cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, cons
   cfg.attrs = attr;
   cfg.numAttrs = 0;
   int grid = (int)(max_items < ctas ? max_items : ctas);
-  // A contraction in 2..8 slices runs as thread-block clusters of that many CTAs (one slice each, exchanged
-  // through distributed shared memory) when that many co-resident CTAs can be had; otherwise, and for
-  // more slices, the slices are exchanged through the workspace.
+  // On request (vcas_set_tuning) a contraction in 2..8 slices runs as thread-block clusters of that many
+  // CTAs, one slice each, exchanged through distributed shared memory.  The default is the exchange
+  // through the workspace: on the benchmark layer it was measured 2-4 us per product faster (33 or fewer
+  // clusters of four 226 KB CTAs fit the GPU at once, and the cluster launch and barriers cost more than
+  // the L2 round trip they replace).
   const int S = P.split_k;
-  if (MH == 1 && S >= 2 && S <= 8 && h->tune_exchange != 1) {
+  if (MH == 1 && S >= 2 && S <= 8 && h->tune_exchange == 2) {
     static int max_clusters[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};   // co-resident clusters per size, queried once
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)S;
