@@ -427,7 +427,7 @@ int vcas_set_tuning(vcas_handle hh, int32_t dx_tile_n, int32_t dw_tile_n, int32_
   if (hh == nullptr) return VCAS_ERR_BAD_ARG;
   auto tile_ok = [](int32_t t) { return t == 0 || t == 64 || t == 128 || t == 256; };
   if (!tile_ok(dx_tile_n) || !tile_ok(dw_tile_n) || dx_split_k < 0 || dx_split_k > 16 ||
-      dw_split_k < 0 || dw_split_k > 16 || tile_m < 0 || tile_m > 2 || exchange < 0 || exchange > 2)
+      dw_split_k < 0 || dw_split_k > 16 || tile_m < 0 || tile_m > 3 || exchange < 0 || exchange > 2)
     return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   h->tune_dx_tile_n = dx_tile_n;

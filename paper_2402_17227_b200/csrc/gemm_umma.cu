@@ -308,6 +308,11 @@ struct GemmParams {
   int xch;                 // > 0: launched in clusters of xch CTAs, one slice per CTA, slices exchanged through
                            // distributed shared memory; 0: slices exchanged through the workspace
   int max_units;
+  // Whole waves and remainder (256-wide tiles): part 1 is the launch with 256-row tiles, which takes only as
+  // many tiles as fill its head_ctas CTAs a whole number of times (when the rest is at most half a wave);
+  // part 2 is a second launch with 128-row tiles that covers the remaining 256-row tiles, two tiles each,
+  // the contraction cut into as many slices as fill its grid once.  0: one launch does everything.
+  int part, head_ctas;
   int d_in, d_out;
   // dX: A = dY viewed [N][T][d_out] (K-major, one TMA box = 128 tokens x 64 k of one datum),
   //     B = W [d_out][d_in] (MN-major: n contiguous)
@@ -332,6 +337,7 @@ struct Decomp {
   int upi;                 // units taken per pass of the grid: a multiple of S, so that the S slices of a tile
                            // are always worked on at the same time by S neighbouring CTAs
   int per_datum, ntiles;   // dX: tiles per datum; both: column tiles
+  int head256, per_datum256;   // parts 1 and 2: 256-row tiles left to part 1; dX: 256-row tiles per datum
 };
 
 template <int MODE, int BN, int MH>
@@ -352,6 +358,30 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
     d.gemm_tiles = d.kblocks > 0 ? tiles : 0;   // nothing kept: every tile is a zero tile
     d.zero_tiles = d.kblocks > 0 ? 0 : tiles;
   }
+  int split_req = P.split_k;
+  d.head256 = 0;
+  d.per_datum256 = 0;
+  if (P.part != 0) {
+    int total256;
+    if (MODE == MODE_DX) {
+      d.per_datum256 = ((P.T + 2 * BM - 1) / (2 * BM)) * d.ntiles;
+      total256 = (P.dense ? P.N : P.counts[0]) * d.per_datum256;
+    } else {
+      total256 = d.kblocks > 0 ? ((P.d_out + 2 * BM - 1) / (2 * BM)) * d.ntiles : 0;
+    }
+    const int frac = total256 % P.head_ctas;
+    const int tail256 = 2 * frac <= P.head_ctas ? frac : 0;
+    d.head256 = total256 - tail256;
+    if (P.part == 1) {
+      d.gemm_tiles = d.head256;
+    } else {
+      d.gemm_tiles = 2 * tail256;
+      d.zero_tiles = 0;                      // part 1 writes them
+      split_req = d.gemm_tiles > 0 ? (int)gridDim.x / d.gemm_tiles : 1;
+      if (split_req > 8) split_req = 8;
+      if (split_req > d.kblocks / 4) split_req = d.kblocks / 4;      // slices of at least four k-blocks
+    }
+  }
   if (P.xch > 0) {
     d.S = P.xch;
     d.kb_per = d.kblocks > 0 ? (d.kblocks + d.S - 1) / d.S : 0;
@@ -360,7 +390,7 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
     d.upi = (int)gridDim.x;          // a multiple of the cluster size
     return d;
   }
-  int S = (P.split_k < 1 || MH == 2) ? 1 : P.split_k;
+  int S = (split_req < 1 || MH == 2) ? 1 : split_req;
   if (S > d.kblocks) S = d.kblocks > 0 ? d.kblocks : 1;
   if (d.gemm_tiles > 0 && (long)d.gemm_tiles * S > P.max_units) S = P.max_units / d.gemm_tiles;
   if (S > (int)gridDim.x) S = (int)gridDim.x;
@@ -371,6 +401,29 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
   d.units = d.gemm_tiles * d.S;
   d.upi = ((int)gridDim.x / d.S) * d.S;
   return d;
+}
+
+// Product tile -> (kept datum k [dX], row chunk c0 in units of this kernel's tile height, column tile c1).
+// In part 2 tile j is half (j & 1) of the 256-row tile head256 + j / 2.
+template <int MODE>
+__device__ __forceinline__ void tile_coords(const GemmParams& P, const Decomp& D, int tile, int& k, int& c0, int& c1) {
+  k = 0;
+  if (P.part == 2) {
+    const int t = D.head256 + (tile >> 1), half = tile & 1;
+    if (MODE == MODE_DX) {
+      k = t / D.per_datum256;
+      const int rem = t % D.per_datum256;
+      c0 = 2 * (rem / D.ntiles) + half; c1 = rem % D.ntiles;
+    } else {
+      c0 = 2 * (t / D.ntiles) + half; c1 = t % D.ntiles;
+    }
+  } else if (MODE == MODE_DX) {
+    k = tile / D.per_datum;
+    const int rem = tile % D.per_datum;
+    c0 = rem / D.ntiles; c1 = rem % D.ntiles;
+  } else {
+    c0 = tile / D.ntiles; c1 = tile % D.ntiles;
+  }
 }
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -405,12 +458,10 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (!ok) break;
         }
         int c0 = 0, c1 = 0, n = 0;   // dX: token chunk, column tile, datum; dW: row tile, column tile
-        if (MODE == MODE_DX) {
-          const int k = tile / D.per_datum, rem = tile % D.per_datum;
-          c0 = rem / D.ntiles; c1 = rem % D.ntiles;
-          n = P.dense ? k : P.idxA[k];
-        } else {
-          c0 = tile / D.ntiles; c1 = tile % D.ntiles;
+        {
+          int k;
+          tile_coords<MODE>(P, D, tile, k, c0, c1);
+          if (MODE == MODE_DX) n = P.dense ? k : P.idxA[k];
         }
         for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(&s.empty[stage], phase ^ 1u, abort_flag, P.status);
@@ -481,8 +532,14 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         int& t_out) {
       sc = 1.0f; n_out = 0; t_out = 0;
       if (MODE == MODE_DX) {
-        const int k = tile / D.per_datum, rem = tile % D.per_datum;
-        const int c = rem / D.ntiles, nt = rem % D.ntiles;
+        int k, c, nt;
+        if (is_gemm) {
+          tile_coords<MODE>(P, D, tile, k, c, nt);
+        } else {
+          k = tile / D.per_datum;
+          const int rem = tile % D.per_datum;
+          c = rem / D.ntiles; nt = rem % D.ntiles;
+        }
         const int n = is_gemm ? (P.dense ? k : P.idxA[k]) : P.dropA[k];
         row0 = (size_t)n * P.T + (size_t)c * BMT;
         rows_valid = min(BMT, P.T - c * BMT);
@@ -490,7 +547,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         n_out = n; t_out = c * BMT;
         if (is_gemm && !P.dense) sc = P.scaleA[n];
       } else {
-        const int mt = tile / D.ntiles, nt = tile % D.ntiles;
+        int k, mt, nt;
+        if (is_gemm) { tile_coords<MODE>(P, D, tile, k, mt, nt); } else { mt = tile / D.ntiles; nt = tile % D.ntiles; }
         row0 = (size_t)mt * BMT;
         rows_valid = min(BMT, P.d_out - mt * BMT);
         col0 = nt * BN;
@@ -860,11 +918,12 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
 // (the shared-memory fill rate of one SM bounds it, so narrow tiles only pay off when they fill
 // more SMs); a unit costs about 4 us of set-up, pipeline fill and output store; a sliced unit
 // about 7 us more (partial store, wait for its siblings, reduction).
-struct Plan { int bn, split, mh; };
+struct Plan { int bn, split, mh; };   // mh: 1 = 128-row tiles, 2 = 256-row tiles, 3 = 256-row whole waves + 128-row remainder
 // row_tiles128: number of 128-row tile rows (for dX: kept data x 128-token chunks).  A 256-row tile
 // (mh = 2) covers two of them; its k-block costs about 0.62 us for twice the work.
+// remainder_ok: 256-row tiles may leave a last partial wave to a second launch with 128-row tiles (mh = 3)
 Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks, int num_sms, int max_units,
-                int force_bn, int force_split) {
+                int force_bn, int force_split, bool remainder_ok) {
   const int widths[3] = {256, 128, 64};
   const double c_kb[3] = {0.50, 0.45, 0.43};
   Plan best = {256, 1, 1};
@@ -887,9 +946,19 @@ Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks,
     }
     if (widths[i] == 256 && force_split <= 1) {                        // 256 x 256 tiles, never sliced
       const long units = row_tiles256 * ntiles;
-      const double waves = (double)((units + num_sms - 1) / num_sms);
-      const double t = waves * ((double)kblocks * 0.62 + 7.0);
+      const double wave = (double)kblocks * 0.62 + 7.0;
+      const double t = (double)((units + num_sms - 1) / num_sms) * wave;
       if (t < best_t - 1e-9) { best_t = t; best = {256, 1, 2}; }
+      const long frac = units % num_sms;
+      if (remainder_ok && frac > 0 && 2 * frac <= num_sms) {            // whole waves, then the rest as sliced 128-row tiles
+        long sp = num_sms / (2 * frac);
+        if (sp > 8) sp = 8;
+        if (sp > kblocks / 4) sp = kblocks / 4;
+        if (sp < 1) sp = 1;
+        const double tail = (double)((kblocks + sp - 1) / sp) * 0.50 + (sp > 1 ? 11.0 + 0.25 * sp : 4.0) + 4.0;
+        const double t2 = (double)(units / num_sms) * wave + tail;
+        if (t2 < best_t - 1e-9) { best_t = t2; best = {256, 1, 3}; }
+      }
     }
   }
   return best;
@@ -957,6 +1026,19 @@ cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, cons
 template <int MODE>
 cudaError_t run_gemm_bn(Handle* h, const Plan& plan, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
                         const GemmParams& P, long max_items, int ctas, bool pdl, cudaStream_t st) {
+  if (plan.mh == 3) {
+    // whole waves of 256-row tiles, then the remaining tiles as 128-row tiles with a sliced contraction
+    // (both launches derive the same division from the device-resident counts)
+    GemmParams Q = P;
+    Q.split_k = 1;
+    Q.part = 1;
+    Q.head_ctas = (int)(max_items < ctas ? max_items : ctas);
+    const cudaError_t e = run_gemm<MODE, 256, 2>(h, a, b, c, Q, max_items, ctas, pdl, st);
+    if (e != cudaSuccess) return e;
+    Q.part = 2;
+    Q.split_k = 0;
+    return run_gemm<MODE, 256, 1>(h, a, b, c, Q, (long)ctas, ctas, true, st);
+  }
   if (plan.mh == 2) return run_gemm<MODE, 256, 2>(h, a, b, c, P, max_items, ctas, pdl, st);
   switch (plan.bn) {
     case 256: return run_gemm<MODE, 256, 1>(h, a, b, c, P, max_items, ctas, pdl, st);
@@ -1010,13 +1092,16 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   const int chunks = (d.T + BM - 1) / BM, chunks2 = (d.T + 2 * BM - 1) / (2 * BM);
   const long nk = (long)(kept + 0.5);
   const int ctas = h->num_sms - spare_sms > 1 ? h->num_sms - spare_sms : 1;
+  // the halves of a 256-row tile must both hold rows for the remainder launch to take them over
+  const bool rem_ok = h->tune_tile_m != 2 && ((d.T % (2 * BM)) == 0 || (d.T % (2 * BM)) > BM);
   Plan plan = plan_tiles(nk * chunks, nk * chunks2, d.d_in, (d.d_out + BK - 1) / BK, ctas, h->max_units,
-                         h->tune_dx_tile_n, h->tune_dx_split_k);
+                         h->tune_dx_tile_n, h->tune_dx_split_k, rem_ok);
   if (h->tune_tile_m == 1) plan.mh = 1;
   if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
+  if (h->tune_tile_m == 3 && plan.bn == 256 && rem_ok) { plan.mh = 3; plan.split = 1; }
   P.split_k = plan.split;
   // upper bound of work items: every datum kept and split, or every datum a zero tile
-  const long max_items = (long)d.N * (plan.mh == 2 ? chunks2 : chunks) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
+  const long max_items = (long)d.N * (plan.mh >= 2 ? chunks2 : chunks) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
   return run_gemm_bn<MODE_DX>(h, plan, tmA, tmB, tmC, P, max_items, ctas, !after_event, st);
 }
 
@@ -1057,12 +1142,14 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
   common_params(h, P, 1);
   P.cnt = cnt; P.dW = dW;
   const long mtiles = (d.d_out + BM - 1) / BM, mtiles2 = (d.d_out + 2 * BM - 1) / (2 * BM);
+  const bool rem_ok = h->tune_tile_m != 2 && ((d.d_out % (2 * BM)) == 0 || (d.d_out % (2 * BM)) > BM);
   Plan plan = plan_tiles(mtiles, mtiles2, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
-                         h->tune_dw_tile_n, h->tune_dw_split_k);
+                         h->tune_dw_tile_n, h->tune_dw_split_k, rem_ok);
   if (h->tune_tile_m == 1) plan.mh = 1;
   if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
+  if (h->tune_tile_m == 3 && plan.bn == 256 && rem_ok) { plan.mh = 3; plan.split = 1; }
   P.split_k = plan.split;
-  const long max_items = (plan.mh == 2 ? mtiles2 : mtiles) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
+  const long max_items = (plan.mh >= 2 ? mtiles2 : mtiles) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
   return run_gemm_bn<MODE_DW>(h, plan, tmA, tmB, tmC, P, max_items, h->num_sms, true, st);
 }
 

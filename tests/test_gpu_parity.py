@@ -163,6 +163,36 @@ def test_tensor_path_split_contraction_and_tile_widths(tile_n, split, tile_m, ex
     layer.close()
 
 
+@pytest.mark.parametrize("shape,rho,nu", [((48, 512, 512, 512), 0.85, 0.5), ((4, 256, 4096, 2560), 0.75, 0.5)])
+def test_tensor_path_whole_waves_and_remainder(shape, rho, nu):
+    """Problems of more tiles than SMs with 256-row tiles for whole waves of CTAs and a second launch of sliced
+    128-row tiles for the rest (the first shape leaves a remainder in the dX product, the second in the dW
+    product): sampled and dense products against the oracle, and bit-identical to a second run."""
+    N, T, d_in, d_out = shape
+    X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=0.3, sigma_B=0.5)
+    layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
+    layer.set_tuning(256, 256, 0, 0, 3, 0)
+    Xc, dYc, Wc = cuda(X, dY, W)
+    ref = o.linear_bwd(np64(X), np64(dY), np64(W), N, T, f32(rho), f32(nu), 9)
+    p_in, q_in = torch.from_numpy(ref["p32"]).cuda(), torch.from_numpy(ref["q32"]).cuda()
+    dX, dW = layer.linear_bwd(Xc, dYc, Wc, rho, nu, 9, p_in=p_in, q_in=q_in)
+    s = layer.last_sampling()
+    assert np.array_equal(s.idxA.cpu().numpy(), ref["idxA"]) and np.array_equal(s.idxW.cpu().numpy(), ref["idxW"])
+    assert rel_fro(np64(dX), ref["dX"]) <= tol_for(BF16) and rel_fro(np64(dW), ref["dW"]) <= tol_for(BF16)
+    assert not np64(dX)[np.repeat(~ref["keepA"], T)].any()
+    dX2, dW2 = layer.linear_bwd(Xc, dYc, Wc, rho, nu, 9, p_in=p_in, q_in=q_in)
+    assert torch.equal(dX, dX2) and torch.equal(dW, dW2)
+    dXd, dWd = o.dense_bwd(np64(X), np64(dY), np64(W))
+    dX3, dW3 = layer.dense_bwd(Xc, dYc, Wc)
+    assert rel_fro(np64(dX3), dXd) <= tol_for(BF16) and rel_fro(np64(dW3), dWd) <= tol_for(BF16)
+    # the same through one launch of 128-row tiles: every element within rounding of the other tiling
+    layer.set_tuning(256, 256, 1, 1, 1, 0)
+    dX4, dW4 = layer.dense_bwd(Xc, dYc, Wc)
+    assert rel_fro(np64(dX3), np64(dX4)) <= 1e-2 and rel_fro(np64(dW3), np64(dW4)) <= 1e-4
+    assert layer.device_status() == 0
+    layer.close()
+
+
 @pytest.mark.parametrize("name,dtype,path", PATHS)
 def test_linear_bwd_end_to_end(name, dtype, path):
     """No overrides: the library's own probabilities, masks and products against the oracle's."""
