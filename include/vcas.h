@@ -204,12 +204,11 @@ int vcas_last_device_status(vcas_handle h, int32_t* status);
  * split into (1..16; slices are combined in a fixed order, so results stay reproducible), and
  * the tile height (tile_m = 1: 128 rows, 2: 256 rows whenever the width is 256 and the
  * contraction is not sliced, 3: 256 rows for as many tiles as fill all SMs a whole number of
- * times and 128 rows with a sliced contraction, in a second launch, for the rest), and how the slices of a sliced contraction meet (exchange = 0 or 1:
- * through the handle's workspace; 2: inside thread-block clusters, through distributed shared
- * memory, for 2..8 slices).  0 = let the library choose from the shapes and ratios.
- * VCAS_ERR_BAD_ARG for a value outside these sets. */
+ * times and 128 rows with a sliced contraction, in a second launch, for the rest).
+ * 0 = let the library choose from the shapes and ratios.  VCAS_ERR_BAD_ARG for a value outside
+ * these sets. */
 int vcas_set_tuning(vcas_handle h, int32_t dx_tile_n, int32_t dw_tile_n, int32_t dx_split_k, int32_t dw_split_k,
-                    int32_t tile_m, int32_t exchange);
+                    int32_t tile_m);
 
 /* Stage timing for benchmarks (the paper has no counterpart; Sec. 6 only reports end-to-end
  * hours).  While enabled, vcas_linear_bwd(_ex) and vcas_dense_bwd record CUDA events on the

@@ -211,9 +211,9 @@ class Layer:
         return st.value
 
     def set_tuning(self, dx_tile_n: int = 0, dw_tile_n: int = 0, dx_split_k: int = 0, dw_split_k: int = 0,
-                   tile_m: int = 0, exchange: int = 0) -> None:
+                   tile_m: int = 0) -> None:
         _check(lib().vcas_set_tuning(self._h, C.c_int32(dx_tile_n), C.c_int32(dw_tile_n), C.c_int32(dx_split_k),
-                                     C.c_int32(dw_split_k), C.c_int32(tile_m), C.c_int32(exchange)), "vcas_set_tuning")
+                                     C.c_int32(dw_split_k), C.c_int32(tile_m)), "vcas_set_tuning")
 
     def set_profiling(self, enable: bool) -> None:
         _check(lib().vcas_set_profiling(self._h, C.c_int32(1 if enable else 0)), "vcas_set_profiling")

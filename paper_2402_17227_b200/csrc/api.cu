@@ -157,7 +157,6 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->prof_calls = h->prof_dense_calls = 0;
   h->tune_dx_tile_n = h->tune_dw_tile_n = h->tune_dx_split_k = h->tune_dw_split_k = 0;
   h->tune_tile_m = 0;
-  h->tune_exchange = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&h->device) != cudaSuccess || cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
     delete h;
@@ -423,19 +422,17 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
 }
 
 int vcas_set_tuning(vcas_handle hh, int32_t dx_tile_n, int32_t dw_tile_n, int32_t dx_split_k, int32_t dw_split_k,
-                    int32_t tile_m, int32_t exchange) {
+                    int32_t tile_m) {
   if (hh == nullptr) return VCAS_ERR_BAD_ARG;
   auto tile_ok = [](int32_t t) { return t == 0 || t == 64 || t == 128 || t == 256; };
   if (!tile_ok(dx_tile_n) || !tile_ok(dw_tile_n) || dx_split_k < 0 || dx_split_k > 16 ||
-      dw_split_k < 0 || dw_split_k > 16 || tile_m < 0 || tile_m > 3 || exchange < 0 || exchange > 2)
-    return VCAS_ERR_BAD_ARG;
+      dw_split_k < 0 || dw_split_k > 16 || tile_m < 0 || tile_m > 3) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   h->tune_dx_tile_n = dx_tile_n;
   h->tune_dw_tile_n = dw_tile_n;
   h->tune_dx_split_k = dx_split_k;
   h->tune_dw_split_k = dw_split_k;
   h->tune_tile_m = tile_m;
-  h->tune_exchange = exchange;
   return VCAS_OK;
 }
 

@@ -70,7 +70,6 @@ struct Handle {
   int tune_dx_tile_n, tune_dw_tile_n, tune_dx_split_k, tune_dw_split_k;
   int tune_tile_m;   // 0 auto, 1: 128-row tiles only, 2: 256-row tiles whenever the width is 256, 3: 256-row tiles for
                      // whole waves of CTAs and 128-row tiles, their contraction sliced, for the rest
-  int tune_exchange; // sliced contractions: 0, 1: exchanged through the workspace; 2: inside thread-block clusters
 };
 constexpr int PROF_RING = 2048;
 

@@ -86,56 +86,6 @@ __device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile 
   return true;
 }
 
-// ---- thread-block cluster: remote mbarrier arrivals and distributed-shared-memory loads
-__device__ __forceinline__ void cluster_sync_all() {     // every thread of every CTA of the cluster
-  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
-}
-__device__ __forceinline__ void fence_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
-// shared::cluster address of this CTA's shared-memory address `addr` in the CTA of rank `rank`
-__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// mbar_wait for a barrier that CTAs of the whole cluster arrive on
-__device__ __noinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  unsigned long long t0 = 0;
-  uint32_t spins = 0;
-  while (!mbar_try_wait_cluster(bar, parity)) {
-    if ((++spins & 0xfffu) == 0) {
-      if (*abort_flag) return false;
-      const unsigned long long now = global_ns();
-      if (t0 == 0) {
-        t0 = now;
-      } else if (now - t0 > WAIT_LIMIT_NS) {
-        *abort_flag = 1;
-        atomicExch(status, (int32_t)VCAS_ERR_TIMEOUT);
-        return false;
-      }
-    }
-  }
-  return true;
-}
-__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t cluster_addr) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr) : "memory");
-  return v;
-}
-
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -229,9 +179,6 @@ struct SmemLayout {
   uint64_t* empty;
   uint64_t* tmem_full;
   uint64_t* tmem_empty;
-  uint64_t* xfull;    // cluster exchange: all slices of the tile are in their CTAs' shared memory
-  uint64_t* xdone;    // cluster exchange: every CTA of the cluster has finished reading this CTA's slice
-  uint64_t* xfree;    // cluster exchange: the stage ring may be loaded again
   uint32_t* tmem_holder;
   int* abort_flag;
   int* flag;          // epilogue broadcast slot
@@ -250,24 +197,18 @@ __device__ __forceinline__ SmemLayout carve(uint8_t* raw) {
   s.empty = bars + C::STAGES;
   s.tmem_full = bars + 2 * C::STAGES;
   s.tmem_empty = bars + 2 * C::STAGES + 2;
-  s.xfull = bars + 2 * C::STAGES + 4;
-  s.xdone = bars + 2 * C::STAGES + 5;
-  s.xfree = bars + 2 * C::STAGES + 6;
-  s.tmem_holder = (uint32_t*)(bars + 2 * C::STAGES + 7);
+  s.tmem_holder = (uint32_t*)(bars + 2 * C::STAGES + 4);
   s.abort_flag = (int*)(s.tmem_holder + 1);
   s.flag = s.abort_flag + 1;
   return s;
 }
 
 template <int BN, int MH>
-__device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid, int cluster_size) {
+__device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid) {
   using C = TileCfg<BN, MH>;
   if (tid == 0) {
     for (int i = 0; i < C::STAGES; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&s.tmem_full[i], 1); mbar_init(&s.tmem_empty[i], 128); }
-    mbar_init(s.xfull, (uint32_t)(cluster_size > 0 ? cluster_size : 1));
-    mbar_init(s.xdone, (uint32_t)(cluster_size > 0 ? cluster_size : 1));
-    mbar_init(s.xfree, 1);
     *s.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -305,8 +246,6 @@ struct GemmParams {
   float* partial;          // [max_units][128 * BN] fp32 partial tiles (split contraction)
   int32_t* tickets;        // [2 * max_units]: slices stored / slices finished per tile; zero between launches
   int split_k;             // slices requested by the host
-  int xch;                 // > 0: launched in clusters of xch CTAs, one slice per CTA, slices exchanged through
-                           // distributed shared memory; 0: slices exchanged through the workspace
   int max_units;
   // Whole waves and remainder (256-wide tiles): part 1 is the launch with 256-row tiles, which takes only as
   // many tiles as fill its head_ctas CTAs a whole number of times (when the rest is at most half a wave);
@@ -332,8 +271,6 @@ struct GemmParams {
 
 struct Decomp {
   int gemm_tiles, zero_tiles, kblocks, S, kb_per, units;
-  int S_eff;               // slices that hold k-blocks (cluster exchange: S is the cluster size and the last
-                           // slices may be empty; otherwise equal to S)
   int upi;                 // units taken per pass of the grid: a multiple of S, so that the S slices of a tile
                            // are always worked on at the same time by S neighbouring CTAs
   int per_datum, ntiles;   // dX: tiles per datum; both: column tiles
@@ -382,14 +319,6 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
       if (split_req > d.kblocks / 4) split_req = d.kblocks / 4;      // slices of at least four k-blocks
     }
   }
-  if (P.xch > 0) {
-    d.S = P.xch;
-    d.kb_per = d.kblocks > 0 ? (d.kblocks + d.S - 1) / d.S : 0;
-    d.S_eff = d.kb_per > 0 ? (d.kblocks + d.kb_per - 1) / d.kb_per : 0;
-    d.units = d.gemm_tiles * d.S;
-    d.upi = (int)gridDim.x;          // a multiple of the cluster size
-    return d;
-  }
   int S = (split_req < 1 || MH == 2) ? 1 : split_req;
   if (S > d.kblocks) S = d.kblocks > 0 ? d.kblocks : 1;
   if (d.gemm_tiles > 0 && (long)d.gemm_tiles * S > P.max_units) S = P.max_units / d.gemm_tiles;
@@ -397,7 +326,6 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
   if (S < 1) S = 1;
   d.kb_per = d.kblocks > 0 ? (d.kblocks + S - 1) / S : 0;
   d.S = d.kb_per > 0 ? (d.kblocks + d.kb_per - 1) / d.kb_per : 1;   // every slice non-empty
-  d.S_eff = d.S;
   d.units = d.gemm_tiles * d.S;
   d.upi = ((int)gridDim.x / d.S) * d.S;
   return d;
@@ -438,25 +366,20 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   extern __shared__ uint8_t smem_raw[];
   const SmemLayout s = carve<BN, MH>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t tmem_base = setup<BN, MH>(s, warp, tid, P.xch);
+  const uint32_t tmem_base = setup<BN, MH>(s, warp, tid);
   volatile int* abort_flag = s.abort_flag;
-  if (P.xch > 0) cluster_sync_all();   // every CTA's exchange barriers are initialised before anyone arrives on them
   pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
   const Decomp D = decompose<MODE, BN, MH>(P);
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      int stage = 0; uint32_t phase = 0; int lt = 0;
+      int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi, ++lt) {
+      for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi) {
         const int tile = u / D.S, slice = u % D.S;
         const int kb0 = slice * D.kb_per;
         const int kb1 = min(D.kblocks, kb0 + D.kb_per);
-        if (P.xch > 0 && lt > 0) {      // the stage ring doubled as the exchange buffer of the unit before
-          ok = mbar_wait(s.xfree, (uint32_t)(lt - 1) & 1u, abort_flag, P.status);
-          if (!ok) break;
-        }
         int c0 = 0, c1 = 0, n = 0;   // dX: token chunk, column tile, datum; dW: row tile, column tile
         {
           int k;
@@ -495,7 +418,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi, ++lt) {
         const int slice = u % D.S;
         const int nkb = min(D.kblocks, (slice + 1) * D.kb_per) - slice * D.kb_per;
-        if (nkb <= 0) continue;         // an empty slice of a cluster exchange: this CTA never touches TMEM
         const int buf = lt % NACC; const uint32_t use = (uint32_t)(lt / NACC) & 1u;
         ok = mbar_wait(&s.tmem_empty[buf], use ^ 1u, abort_flag, P.status);
         if (!ok) break;
@@ -588,11 +510,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(tile, true, row0, rows_valid, col0, sc, n_out, t_out);
       const int buf = lt % NACC; const uint32_t use = (uint32_t)(lt / NACC) & 1u;
-      const bool empty = P.xch > 0 && slice >= D.S_eff;    // a cluster CTA without k-blocks: reduces only
-      if (!empty) {
-        if (!mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status)) break;
-        tc_fence_after();
-      }
+      if (!mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status)) break;
+      tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * BN);
       // Adds the slices of this unit's share of the tile's rows in slice order and writes that share of the
       // output.  A partial tile is laid out [32-column chunk][row][32 floats] with the eight 16-byte slots of
@@ -617,11 +536,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const size_t ob0 = slot_off(rb, cb, 0), ob1 = slot_off(rb, cb, 1);
           float fa[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
           float fb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          for (int sl0 = 0; sl0 < D.S_eff; sl0 += 4) {           // slices in order, four at a time in flight
+          for (int sl0 = 0; sl0 < D.S; sl0 += 4) {           // slices in order, four at a time in flight
             float4 x[4][4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const int sl = min(sl0 + q, D.S_eff - 1);
+              const int sl = min(sl0 + q, D.S - 1);
               x[q][0] = load4(sl, oa0);
               x[q][1] = load4(sl, oa1);
               x[q][2] = load4(sl, ob0);
@@ -629,7 +548,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              if (sl0 + q < D.S_eff) {
+              if (sl0 + q < D.S) {
                 fa[0] += x[q][0].x; fa[1] += x[q][0].y; fa[2] += x[q][0].z; fa[3] += x[q][0].w;
                 fa[4] += x[q][1].x; fa[5] += x[q][1].y; fa[6] += x[q][1].z; fa[7] += x[q][1].w;
                 fb[0] += x[q][2].x; fb[1] += x[q][2].y; fb[2] += x[q][2].z; fb[3] += x[q][2].w;
@@ -702,54 +621,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         mbar_arrive(&s.tmem_empty[buf]);
         if (lane == 0) bulk_wait_all();        // staging buffers are reused by the next unit
         __syncwarp();
-        continue;
-      }
-      if (P.xch > 0) {
-        // ---- one slice of the contraction, exchanged inside the cluster: the fp32 partial tile goes to
-        // this CTA's shared memory (the stage ring, idle once the accumulator is complete); when all CTAs
-        // of the cluster have theirs, each adds the slices of its share of the rows, reading the other
-        // CTAs' shared memory, in slice order.
-        uint8_t* xbuf = s.stages;
-        if (!empty) {
-#pragma unroll 1
-          for (int j = 0; j < BN / 32; ++j) {
-            if (col0 + j * 32 >= P.d_in) break;                       // warp-uniform
-            uint32_t v[32];
-            tmem_ld32(taddr + (uint32_t)(j * 32), v);
-            uint4* myrow = reinterpret_cast<uint4*>(xbuf + (size_t)j * (BM * 128) + (size_t)row * 128);
-#pragma unroll
-            for (int g4 = 0; g4 < 8; ++g4)
-              myrow[(uint32_t)g4 ^ swz] = make_uint4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
-          }
-          tc_fence_before();
-          mbar_arrive(&s.tmem_empty[buf]);        // the accumulator is free again
-        }
-        const uint32_t par = (uint32_t)lt & 1u;
-        fence_cluster();
-        epi_bar();
-        if (tid == 0) {
-          for (int j = 0; j < D.S; ++j) mbar_arrive_remote(mapa(smem_u32(s.xfull), (uint32_t)j));
-          *s.flag = mbar_wait_cluster(s.xfull, par, abort_flag, P.status) ? 1 : 0;
-        }
-        epi_bar();
-        ok = *(volatile int*)s.flag != 0;
-        if (!ok) break;
-        fence_cluster();
-        {
-          const uint32_t xaddr = smem_u32(xbuf);
-          reduce_share([&](int sl, size_t off) { return ld_dsmem_f4(mapa(xaddr, (uint32_t)sl) + (uint32_t)(off * 4)); });
-        }
-        epi_bar();                                  // this CTA has finished reading the others' slices
-        if (tid == 0) {
-          for (int j = 0; j < D.S; ++j) mbar_arrive_remote(mapa(smem_u32(s.xdone), (uint32_t)j));
-          const bool good = mbar_wait_cluster(s.xdone, par, abort_flag, P.status);   // ... and the others this CTA's
-          fence_async_smem();                       // the ring is written by TMA next
-          mbar_arrive(s.xfree);
-          *s.flag = good ? 1 : 0;
-        }
-        epi_bar();
-        ok = *(volatile int*)s.flag != 0;
-        if (!ok) break;
         continue;
       }
       // ---- one slice of the contraction: store the fp32 partial tile.  Layout in the workspace:
@@ -839,8 +710,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   __syncwarp();
   tc_fence_before();
   __syncthreads();
-  // no CTA of a cluster leaves while another may still read its shared memory or arrive on its barriers
-  if (P.xch > 0) cluster_sync_all();
   if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
 }
 
@@ -983,35 +852,6 @@ cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, cons
   cfg.attrs = attr;
   cfg.numAttrs = 0;
   int grid = (int)(max_items < ctas ? max_items : ctas);
-  // On request (vcas_set_tuning) a contraction in 2..8 slices runs as thread-block clusters of that many
-  // CTAs, one slice each, exchanged through distributed shared memory.  The default is the exchange
-  // through the workspace: on the benchmark layer it was measured 2-4 us per product faster (33 or fewer
-  // clusters of four 226 KB CTAs fit the GPU at once, and the cluster launch and barriers cost more than
-  // the L2 round trip they replace).
-  const int S = P.split_k;
-  if (MH == 1 && S >= 2 && S <= 8 && h->tune_exchange == 2) {
-    static int max_clusters[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};   // co-resident clusters per size, queried once
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)S;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.numAttrs = 1;
-    if (max_clusters[S] < 0) {
-      cfg.gridDim = dim3((unsigned)S);
-      int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, umma_kernel<MODE, BN, MH>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-      max_clusters[S] = n;
-    }
-    int clusters = max_clusters[S] < ctas / S ? max_clusters[S] : ctas / S;
-    const long tiles_max = (max_items + S - 1) / S;
-    if (tiles_max < clusters) clusters = (int)tiles_max;
-    if (clusters >= 1) {
-      P.xch = S;
-      grid = clusters * S;
-    } else {
-      cfg.numAttrs = 0;
-    }
-  }
   if (pdl) {
     attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;

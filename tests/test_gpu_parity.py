@@ -137,17 +137,15 @@ def test_linear_bwd_given_oracle_probabilities(name, dtype, path, shape):
     layer.close()
 
 
-@pytest.mark.parametrize("tile_n,split,tile_m,exchange", [
-    (256, 3, 1, 1), (128, 2, 1, 1), (64, 5, 1, 1), (256, 16, 1, 0), (256, 1, 1, 0), (64, 1, 1, 0), (256, 1, 2, 0),
-    (256, 0, 2, 0), (256, 2, 1, 2), (256, 3, 1, 2), (128, 4, 1, 2), (64, 5, 1, 2), (128, 8, 1, 2), (256, 4, 1, 0)])
-def test_tensor_path_split_contraction_and_tile_widths(tile_n, split, tile_m, exchange):
-    """Every tile width and a contraction cut into slices (combined in a fixed order; exchanged through the
-    workspace or inside thread-block clusters, some slices empty when the contraction is short) give the same
+@pytest.mark.parametrize("tile_n,split,tile_m", [(256, 3, 1), (128, 2, 1), (64, 5, 1), (256, 16, 1), (256, 1, 1),
+                                                 (64, 1, 1), (256, 1, 2), (256, 0, 2), (128, 8, 1), (256, 4, 1)])
+def test_tensor_path_split_contraction_and_tile_widths(tile_n, split, tile_m):
+    """Every tile width and a contraction cut into slices (combined in a fixed order) give the same
     results within tolerance, for the sampled and the dense products; repeated runs are bit-identical."""
     N, T, d_in, d_out = 5, 197, 320, 448
     X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.5, sigma_B=1.0)
     layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
-    layer.set_tuning(tile_n, tile_n, split, split, tile_m, exchange)
+    layer.set_tuning(tile_n, tile_n, split, split, tile_m)
     Xc, dYc, Wc = cuda(X, dY, W)
     ref = o.linear_bwd(np64(X), np64(dY), np64(W), N, T, 0.5, 0.5, 4)
     p_in, q_in = torch.from_numpy(ref["p32"]).cuda(), torch.from_numpy(ref["q32"]).cuda()
@@ -171,7 +169,7 @@ def test_tensor_path_whole_waves_and_remainder(shape, rho, nu):
     N, T, d_in, d_out = shape
     X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=0.3, sigma_B=0.5)
     layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
-    layer.set_tuning(256, 256, 0, 0, 3, 0)
+    layer.set_tuning(256, 256, 0, 0, 3)
     Xc, dYc, Wc = cuda(X, dY, W)
     ref = o.linear_bwd(np64(X), np64(dY), np64(W), N, T, f32(rho), f32(nu), 9)
     p_in, q_in = torch.from_numpy(ref["p32"]).cuda(), torch.from_numpy(ref["q32"]).cuda()
@@ -186,7 +184,7 @@ def test_tensor_path_whole_waves_and_remainder(shape, rho, nu):
     dX3, dW3 = layer.dense_bwd(Xc, dYc, Wc)
     assert rel_fro(np64(dX3), dXd) <= tol_for(BF16) and rel_fro(np64(dW3), dWd) <= tol_for(BF16)
     # the same through one launch of 128-row tiles: every element within rounding of the other tiling
-    layer.set_tuning(256, 256, 1, 1, 1, 0)
+    layer.set_tuning(256, 256, 1, 1, 1)
     dX4, dW4 = layer.dense_bwd(Xc, dYc, Wc)
     assert rel_fro(np64(dX3), np64(dX4)) <= 1e-2 and rel_fro(np64(dW3), np64(dW4)) <= 1e-4
     assert layer.device_status() == 0
