@@ -48,6 +48,9 @@ size_t layout(Handle* h, uint8_t* base) {
   w.idxA = carve<int32_t>(cur, N);
   w.dropA = carve<int32_t>(cur, N);
   w.idxW = carve<int32_t>(cur, R);
+  w.scaleA2 = carve<float>(cur, N);
+  w.idxA2 = carve<int32_t>(cur, N);
+  w.dropA2 = carve<int32_t>(cur, N);
   w.counts = carve<int32_t>(cur, 8);
   w.status = carve<int32_t>(cur, 1);
   w.acc = carve<double>(cur, 16);
@@ -229,11 +232,10 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   cudaStream_t st = S(stream);
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
-  a.a_done = fast_sampling(h->desc) ? 1 : 0;
   const int hint = (int)(rho * nu * (float)(h->desc.N * h->desc.T)) + 1;
   if (!h->tensor_path) {
     mark(h, 0, st);
-    VCAS_CUDA(launch_rownorms(h, dY, X, seed, a.a_done ? &a : nullptr, st));
+    VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
     mark(h, 1, st);
     VCAS_CUDA(launch_sampler(h, a, st));
     mark(h, 2, st);
@@ -246,7 +248,7 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   } else if (h->prof_enabled) {
     // stage profiling: everything on `st`, so that each pair of events brackets one kernel
     mark(h, 0, st);
-    VCAS_CUDA(launch_rownorms(h, dY, X, seed, a.a_done ? &a : nullptr, st));
+    VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
     mark(h, 1, st);
     VCAS_CUDA(launch_sampler(h, a, st));
     mark(h, 2, st);
@@ -257,24 +259,25 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     mark(h, 4, st);
     VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, st));
     mark(h, 5, st);
-  } else if (a.a_done) {
-    // SampleA ran in the tail of the row-norm kernel, and the dX product needs nothing else: it is
-    // forked onto the handle's side stream right after that kernel and overlaps SampleW, the pack
-    // and the dW product, which stay on `st` as a chain of programmatic dependent launches (the
-    // longer of the two branches).  The dX grid leaves one SM free: the sampling kernel is a single
-    // CTA that needs a whole SM's registers.
-    VCAS_CUDA(launch_rownorms(h, dY, X, seed, &a, st));
+  } else if (fast_sampling(h->desc)) {
+    // The dX product needs SampleA only.  On `st`, a small SampleA-only kernel and the dX product follow the
+    // row norms as programmatic dependent launches; the full sampling kernel (which draws the same SampleA
+    // masks, then SampleW), the pack and the dW product run beside them on the handle's side stream and are
+    // joined back before the call's work ends on `st`.  The dX grid leaves one SM free: the sampling kernel
+    // is a single CTA that needs a whole SM's registers.
+    VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-    VCAS_CUDA(launch_sampler(h, a, st));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, h->side_stream));
+    VCAS_CUDA(launch_sampler(h, a, h->side_stream, true));
+    VCAS_CUDA(launch_sample_a(h, a, st));
+    VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, h->side_stream));
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
-    VCAS_CUDA(launch_pack(h, dY, X, st));
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, st));
     VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   } else {
     // large layers (generic sampling kernel): the products fork once the sampler has run
-    VCAS_CUDA(launch_rownorms(h, dY, X, seed, nullptr, st));
+    VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
     VCAS_CUDA(launch_sampler(h, a, st));
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
@@ -333,8 +336,7 @@ int vcas_score(vcas_handle hh, const void* X, const void* dY, float rho, float n
   cudaStream_t st = S(stream);
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 1; a.accumulate_vw = 0;
-  a.a_done = fast_sampling(h->desc) ? 1 : 0;
-  VCAS_CUDA(launch_rownorms(h, dY, X, seed, a.a_done ? &a : nullptr, st));
+  VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
   VCAS_CUDA(launch_sampler(h, a, st));
   return copy_out(h, g, p, w, q, idxA, cntA, idxW, cntW, st);
 }
@@ -371,10 +373,10 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
     int rc = dense_dw(h, X_i[i], dY_i[i], h->ws.Gs, st);            // G_s,i
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(launch_probe_welford(h, i, st));
-    VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, nullptr, st));   // the probe draws no SampleW mask
+    VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, st));   // the probe draws no SampleW mask
     for (int j = 0; j < M; ++j) {
       SamplerArgs a;
-      a.rho = rho; a.nu = nu; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 0; a.accumulate_vw = 1; a.a_done = 0;
+      a.rho = rho; a.nu = nu; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 0; a.accumulate_vw = 1;
       a.seed = seed + (uint64_t)(i * M + j + 1) * 0x9E3779B97F4A7C15ull;
       VCAS_CUDA(launch_sampler(h, a, st));
       if (j == 0) VCAS_CUDA(launch_probe_sparsity(h, s_lo, s_hi, st));

@@ -28,7 +28,11 @@ struct Workspace {
   int32_t* idxA;   // [N]  kept data, ascending
   int32_t* dropA;  // [N]  dropped data, ascending
   int32_t* idxW;   // [R]  kept rows, ascending
-  int32_t* counts; // [8]  0: cntA, 1: cntW, 2: R (constant, for dense launches), 4: reduction ticket, 5: row-norm ticket
+  // second set of SampleA results (launch_sample_a), read by a dX product that runs beside the sampling kernel
+  float* scaleA2;  // [N]
+  int32_t* idxA2;  // [N]
+  int32_t* dropA2; // [N]
+  int32_t* counts; // [8]  0: cntA, 1: cntW, 2: R (constant, for dense launches), 4: reduction ticket, 6: cntA of the second SampleA set
   int32_t* status; // [1]  device status word
   double* acc;     // [16] probe accumulators (0: V_act, 1: V_w, 2: p_lo, 3: p_hi, 4: V_s)
   double* partial; // [PARTIAL_SLOTS] block partial sums of the probe reductions
@@ -250,7 +254,7 @@ __device__ __forceinline__ int sample_a_warp(const float* g, int N, float rho, c
     const unsigned lower = (1u << lane) - 1u;
     if (in) {
       const float sc = keep ? 1.0f / v[j] : 0.f;
-      o.p[n] = v[j];
+      if (o.p != nullptr) o.p[n] = v[j];
       o.scaleA[n] = sc;
       if (o.sh_p != nullptr) { o.sh_p[n] = v[j]; o.sh_scaleA[n] = sc; }
       if (keep) o.idxA[kept_before + __popc(bk & lower)] = n;
@@ -262,8 +266,8 @@ __device__ __forceinline__ int sample_a_warp(const float* g, int N, float rho, c
   return kept_before;
 }
 
-// The single-CTA register-resident sampling kernel, and with it SampleA in the tail of the row-norm
-// kernel, serve layers of at most this many data and rows.
+// The single-CTA register-resident sampling kernel, and with it the SampleA-only kernel that lets the dX
+// product start early, serve layers of at most this many data and rows.
 constexpr int FAST_MAX_N = 1024;
 constexpr int FAST_MAX_R = 16 * 1024;
 inline bool fast_sampling(const vcas_layer_desc& d) {
@@ -280,13 +284,13 @@ struct SamplerArgs {
   const float* q_in;
   int sample_w;      // 1: SampleW mask applied; 0: all rows of kept data survive (probe)
   int accumulate_vw; // 1: add Eq. 3 at ratio nu to acc[1]
-  int a_done;        // 1: SampleA's results are already in the workspace (row-norm kernel's tail)
 };
-// seed: the call's seed (the SampleW uniforms are drawn here, one per row).  tail != nullptr and
-// fast_sampling(desc): the last CTA to finish also runs SampleA with tail's rho, p_in and seed, so that
-// the dX product can follow directly; the caller then passes a_done = 1 to launch_sampler.
-cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, const SamplerArgs* tail,
-                            cudaStream_t st);
+// seed: the call's seed (the SampleW uniforms are drawn here, one per row)
+cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, cudaStream_t st);
+// SampleA alone (rho, p_in and seed of `a`), into the workspace's second set of SampleA arrays (idxA2, dropA2,
+// scaleA2, counts[6]): what the dX product needs, so that it can start while the full sampling kernel,
+// which draws the same masks, runs beside it on another stream.  Requires fast_sampling(desc).
+cudaError_t launch_sample_a(Handle* h, const SamplerArgs& a, cudaStream_t st);
 // after_event: launched plainly (its inputs come through an event from another stream)
 cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st, bool after_event = false);
 cudaError_t launch_mask_from_probs(Handle* h, const float* p, int n, uint64_t seed, int sampler,
@@ -300,9 +304,9 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 
 // tensor-core products
 // spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it);
-// after_event: launched plainly (its inputs come through an event from another stream)
+// second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a)
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, int spare_sms, bool after_event, cudaStream_t st);
+                           const void* H, void* dX, int spare_sms, bool second_set, cudaStream_t st);
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling

@@ -900,7 +900,7 @@ void common_params(Handle* h, GemmParams& P, int which) {
 }  // namespace
 
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint, const void* H,
-                           void* dX, int spare_sms, bool after_event, cudaStream_t st) {
+                           void* dX, int spare_sms, bool second_set, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -924,6 +924,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   GemmParams P;
   common_params(h, P, 0);
   P.idxA = h->ws.idxA; P.dropA = h->ws.dropA; P.counts = h->ws.counts; P.scaleA = h->ws.scaleA;
+  if (second_set) { P.idxA = h->ws.idxA2; P.dropA = h->ws.dropA2; P.counts = h->ws.counts + 6; P.scaleA = h->ws.scaleA2; }
   P.H = (const __nv_bfloat16*)H; P.dX = (__nv_bfloat16*)dX;
   P.N = d.N; P.T = d.T; P.dense = dense ? 1 : 0;
   P.a_tx_bytes = (d.T < BM ? d.T : BM) * BK * 2;
@@ -942,7 +943,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   P.split_k = plan.split;
   // upper bound of work items: every datum kept and split, or every datum a zero tile
   const long max_items = (long)d.N * (plan.mh >= 2 ? chunks2 : chunks) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
-  return run_gemm_bn<MODE_DX>(h, plan, tmA, tmB, tmC, P, max_items, ctas, !after_event, st);
+  return run_gemm_bn<MODE_DX>(h, plan, tmA, tmB, tmC, P, max_items, ctas, true, st);
 }
 
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st) {

@@ -131,7 +131,7 @@ struct SamplerParams {
   int N, T;
   float rho, nu;
   uint64_t seed;
-  int sample_w, accumulate_vw, a_done;
+  int sample_w, accumulate_vw;
 };
 
 __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_kernel(SamplerParams P) {
@@ -308,25 +308,19 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     return n < N ? n : N - 1;
   };
 
-  if (P.a_done) {
-    // SampleA already ran in the tail of the row-norm kernel: fetch its results
-    for (int n = tid; n < N; n += SAMPLER_THREADS) { sh.scaleA[n] = P.scaleA[n]; sh.pA[n] = P.p[n]; }
-    if (tid == 0) sh.cntA = P.counts[0];
-  } else {
-    // ---- ||G_n||_F: one warp per datum, fixed order
-    for (int n = warp; n < N; n += 32) {
-      const float s = datum_sqnorm_warp(P.a + (size_t)n * T, T, lane);
-      if (lane == 0) { const float g = sqrtf(s); P.g[n] = g; sh.pA[n] = g; }
-    }
-    __syncthreads();
-    // ---- SampleA inside warp 0 (Sec. 4.1): p_n, mask, kept / dropped lists
-    if (warp == 0) {
-      SampleAOut o;
-      o.p = P.p; o.scaleA = P.scaleA; o.idxA = P.idxA; o.dropA = P.dropA;
-      o.sh_p = sh.pA; o.sh_scaleA = sh.scaleA;
-      const int kept = sample_a_warp<SLOTS>(sh.pA, N, P.rho, P.p_in, P.seed, o, lane);
-      if (lane == 0) sh.cntA = kept;
-    }
+  // ---- ||G_n||_F: one warp per datum, fixed order
+  for (int n = warp; n < N; n += 32) {
+    const float s = datum_sqnorm_warp(P.a + (size_t)n * T, T, lane);
+    if (lane == 0) { const float g = sqrtf(s); P.g[n] = g; sh.pA[n] = g; }
+  }
+  __syncthreads();
+  // ---- SampleA inside warp 0 (Sec. 4.1): p_n, mask, kept / dropped lists
+  if (warp == 0) {
+    SampleAOut o;
+    o.p = P.p; o.scaleA = P.scaleA; o.idxA = P.idxA; o.dropA = P.dropA;
+    o.sh_p = sh.pA; o.sh_scaleA = sh.scaleA;
+    const int kept = sample_a_warp<SLOTS>(sh.pA, N, P.rho, P.p_in, P.seed, o, lane);
+    if (lane == 0) sh.cntA = kept;
   }
   __syncthreads();
   const int cntA = sh.cntA;
@@ -483,9 +477,32 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
         ++base;
       }
   }
-  if (tid == 0) {
-    if (!P.a_done) P.counts[0] = cntA;
-    P.counts[1] = total;
+  if (tid == 0) { P.counts[0] = cntA; P.counts[1] = total; }
+}
+
+// SampleA alone (Sec. 4.1), for the dX product: the same warp-level code as in the sampling kernels, so the
+// masks are identical; results go to arrays of their own because the full sampling kernel runs at the
+// same time on another stream.
+constexpr int SAMPLE_A_THREADS = 512;
+template <int SLOTS>
+__global__ void __launch_bounds__(SAMPLE_A_THREADS)
+sample_a_kernel(const float* __restrict__ a, int N, int T, float rho, const float* __restrict__ p_in, uint64_t seed,
+                float* scaleA, int32_t* idxA, int32_t* dropA, int32_t* cnt) {
+  __shared__ float s_g[32 * SLOTS];
+  pdl_wait();      // the row norms come from the kernel before this one
+  pdl_trigger();   // the dX product kernel may set itself up meanwhile
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int n = warp; n < N; n += SAMPLE_A_THREADS / 32) {
+    const float s = datum_sqnorm_warp(a + (size_t)n * T, T, lane);
+    if (lane == 0) s_g[n] = sqrtf(s);
+  }
+  __syncthreads();
+  if (warp == 0) {
+    SampleAOut o;
+    o.p = nullptr; o.scaleA = scaleA; o.idxA = idxA; o.dropA = dropA;
+    o.sh_p = nullptr; o.sh_scaleA = nullptr;
+    const int kept = sample_a_warp<SLOTS>(s_g, N, rho, p_in, seed, o, lane);
+    if (lane == 0) *cnt = kept;
   }
 }
 
@@ -516,7 +533,6 @@ cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st, boo
   P.N = h->desc.N; P.T = h->desc.T;
   P.rho = a.rho; P.nu = a.nu; P.seed = a.seed;
   P.sample_w = a.sample_w; P.accumulate_vw = a.accumulate_vw;
-  P.a_done = a.a_done && fast_sampling(h->desc);
   const int R = P.N * P.T;
   cudaError_t e = cudaSuccess;
   // after_event: the kernel before this one in the stream is not the producer of its inputs (those
@@ -533,6 +549,21 @@ cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st, boo
   } else {
     e = go(sampler_kernel);
   }
+  h->launches += 1;
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_sample_a(Handle* h, const SamplerArgs& a, cudaStream_t st) {
+  const Workspace& ws = h->ws;
+  const vcas_layer_desc& d = h->desc;
+  if (!fast_sampling(d)) return cudaErrorInvalidValue;
+  cudaError_t e;
+  if (d.N <= 32)
+    e = launch_after(sample_a_kernel<1>, dim3(1), dim3(SAMPLE_A_THREADS), 0, st, (const float*)ws.a, d.N, d.T, a.rho,
+                     a.p_in, a.seed, ws.scaleA2, ws.idxA2, ws.dropA2, ws.counts + 6);
+  else
+    e = launch_after(sample_a_kernel<32>, dim3(1), dim3(SAMPLE_A_THREADS), 0, st, (const float*)ws.a, d.N, d.T, a.rho,
+                     a.p_in, a.seed, ws.scaleA2, ws.idxA2, ws.dropA2, ws.counts + 6);
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
 }

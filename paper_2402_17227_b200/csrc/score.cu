@@ -68,122 +68,64 @@ __device__ __forceinline__ float row_partial(const T* __restrict__ src, int d, i
   return (acc0 + acc1) + (acc2 + acc3);
 }
 
-// SampleA in the tail of the row-norm kernel: what the last CTA needs besides the row norms.
-struct TailParams {
-  int N, T;
-  float rho;
-  const float* p_in;
-  uint64_t seed;
-  float* g; float* p; float* scaleA;
-  int32_t* idxA; int32_t* dropA; int32_t* counts;   // counts[0] = kept data, counts[5] = CTA ticket
-};
-
 // One warp per row r: a[r] = ||dY_r||^2, b[r] = ||X_r||^2, and two per-row values the sampling
 // stage would otherwise compute on its single SM: lev[r] = ||dY_r|| ||X_r|| (the leverage score of
 // Sec. 4.2 before the 1/p_n rescale) and u24[r], the 24-bit Philox uniform of SampleW for this row.
-// SLOTS > 0: the CTA that finishes last (a ticket in the workspace) goes on to SampleA (Sec. 4.1) over
-// N <= 32 * SLOTS data, so that the dX product, which needs only the kept data, can start right after
-// this kernel while SampleW is still being drawn.
-template <typename T, int SLOTS>
-__global__ void __launch_bounds__(256, 4) rownorm_kernel(const T* __restrict__ dY, const T* __restrict__ X,
-                                                         int R, int d_out, int d_in, uint64_t seed,
-                                                         float* __restrict__ a, float* __restrict__ b,
-                                                         float* __restrict__ lev, uint32_t* __restrict__ u24,
-                                                         TailParams tail) {
+template <typename T>
+__global__ void __launch_bounds__(256) rownorm_kernel(const T* __restrict__ dY, const T* __restrict__ X,
+                                                      int R, int d_out, int d_in, uint64_t seed,
+                                                      float* __restrict__ a, float* __restrict__ b,
+                                                      float* __restrict__ lev, uint32_t* __restrict__ u24) {
   pdl_trigger();   // the next kernel may be scheduled now; it waits for this grid before reading
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int row = blockIdx.x * (blockDim.x >> 5) + warp;
-  if (row < R) {
-    // the first four vectors per lane of the X row are requested before the dY row is touched
-    using V = typename Vec<T>::type;
-    constexpr int VN = Vec<T>::N;
-    const T* xrow = X + (size_t)row * d_in;
-    const bool xvec = (d_in % VN) == 0;
-    const int nvx = xvec ? d_in / VN : 0;
-    V xv[4];
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= R) return;
+  // the first four vectors per lane of the X row are requested before the dY row is touched
+  using V = typename Vec<T>::type;
+  constexpr int VN = Vec<T>::N;
+  const T* xrow = X + (size_t)row * d_in;
+  const bool xvec = (d_in % VN) == 0;
+  const int nvx = xvec ? d_in / VN : 0;
+  V xv[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    if (lane + 32 * k < nvx) xv[k] = __ldg(reinterpret_cast<const V*>(xrow) + lane + 32 * k);
+  const float pa = row_partial<T>(dY + (size_t)row * d_out, d_out, lane);
+  float pb = 0.f;
+  if (xvec) {
 #pragma unroll
     for (int k = 0; k < 4; ++k)
-      if (lane + 32 * k < nvx) xv[k] = __ldg(reinterpret_cast<const V*>(xrow) + lane + 32 * k);
-    const float pa = row_partial<T>(dY + (size_t)row * d_out, d_out, lane);
-    float pb = 0.f;
-    if (xvec) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (lane + 32 * k < nvx) pb += Vec<T>::sq(xv[k]);
-      for (int i = lane + 128; i < nvx; i += 32) pb += Vec<T>::sq(__ldg(reinterpret_cast<const V*>(xrow) + i));
-    } else {
-      pb = row_partial<T>(xrow, d_in, lane);
-    }
-    const float sa = warp_sum(pa), sb = warp_sum(pb);
-    if (lane == 0) {
-      a[row] = sa;
-      b[row] = sb;
-      lev[row] = sqrtf(sa) * sqrtf(sb);
-      u24[row] = philox_word0((uint32_t)row, 0u, 1u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32)) >> 8;
-      if (SLOTS > 0) __threadfence();
-    }
+      if (lane + 32 * k < nvx) pb += Vec<T>::sq(xv[k]);
+    for (int i = lane + 128; i < nvx; i += 32) pb += Vec<T>::sq(__ldg(reinterpret_cast<const V*>(xrow) + i));
+  } else {
+    pb = row_partial<T>(xrow, d_in, lane);
   }
-  if constexpr (SLOTS > 0) {
-    __shared__ int s_last;
-    __shared__ float s_g[32 * SLOTS];
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      __threadfence();
-      s_last = atomicAdd(tail.counts + 5, 1) == (int)gridDim.x - 1 ? 1 : 0;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();            // every other CTA's row norms are visible from here on
-    const int nw = blockDim.x >> 5;
-    for (int n = warp; n < tail.N; n += nw) {
-      const float s = datum_sqnorm_warp(a + (size_t)n * tail.T, tail.T, lane);
-      if (lane == 0) { const float gn = sqrtf(s); tail.g[n] = gn; s_g[n] = gn; }
-    }
-    __syncthreads();
-    if (warp == 0) {
-      SampleAOut o;
-      o.p = tail.p; o.scaleA = tail.scaleA; o.idxA = tail.idxA; o.dropA = tail.dropA;
-      o.sh_p = nullptr; o.sh_scaleA = nullptr;
-      const int cntA = sample_a_warp<SLOTS>(s_g, tail.N, tail.rho, tail.p_in, tail.seed, o, lane);
-      if (lane == 0) { tail.counts[0] = cntA; tail.counts[5] = 0; }
-    }
+  const float sa = warp_sum(pa), sb = warp_sum(pb);
+  if (lane == 0) {
+    a[row] = sa;
+    b[row] = sb;
+    lev[row] = sqrtf(sa) * sqrtf(sb);
+    u24[row] = philox_word0((uint32_t)row, 0u, 1u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32)) >> 8;
   }
 }
 
 }  // namespace
 
-namespace {
-template <typename T>
-cudaError_t launch_typed(Handle* h, const void* dY, const void* X, uint64_t seed, const SamplerArgs* tail,
-                         cudaStream_t st) {
+cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   const int R = d.N * d.T;
   const int warps_per_block = 8;
   const int blocks = (R + warps_per_block - 1) / warps_per_block;
-  const Workspace& ws = h->ws;
-  TailParams t = {};
-  const bool with_tail = tail != nullptr && fast_sampling(d);
-  if (with_tail) {
-    t.N = d.N; t.T = d.T; t.rho = tail->rho; t.p_in = tail->p_in; t.seed = tail->seed;
-    t.g = ws.g; t.p = ws.p; t.scaleA = ws.scaleA; t.idxA = ws.idxA; t.dropA = ws.dropA; t.counts = ws.counts;
+  if (d.dtype == VCAS_DTYPE_BF16) {
+    rownorm_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dY, (const __nv_bfloat16*)X, R,
+                                                          d.d_out, d.d_in, seed, h->ws.a, h->ws.b, h->ws.lev,
+                                                          h->ws.u24);
+  } else {
+    rownorm_kernel<float><<<blocks, 256, 0, st>>>((const float*)dY, (const float*)X, R, d.d_out, d.d_in, seed,
+                                                  h->ws.a, h->ws.b, h->ws.lev, h->ws.u24);
   }
-  const T* dy = (const T*)dY;
-  const T* x = (const T*)X;
-  if (!with_tail)
-    rownorm_kernel<T, 0><<<blocks, 256, 0, st>>>(dy, x, R, d.d_out, d.d_in, seed, ws.a, ws.b, ws.lev, ws.u24, t);
-  else if (d.N <= 32)
-    rownorm_kernel<T, 1><<<blocks, 256, 0, st>>>(dy, x, R, d.d_out, d.d_in, seed, ws.a, ws.b, ws.lev, ws.u24, t);
-  else
-    rownorm_kernel<T, 32><<<blocks, 256, 0, st>>>(dy, x, R, d.d_out, d.d_in, seed, ws.a, ws.b, ws.lev, ws.u24, t);
-  return cudaGetLastError();
-}
-}  // namespace
-
-cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, const SamplerArgs* tail,
-                            cudaStream_t st) {
   h->launches += 1;
-  return h->desc.dtype == VCAS_DTYPE_BF16 ? launch_typed<__nv_bfloat16>(h, dY, X, seed, tail, st)
-                                          : launch_typed<float>(h, dY, X, seed, tail, st);
+  return cudaGetLastError();
 }
 
 }  // namespace vcas

@@ -85,8 +85,7 @@ extern "C" int vcas_score_static(int32_t N, int32_t T, int32_t d_in, int32_t d_o
   if (cudaMemsetAsync(tail, 0, kTailBytes, st) != cudaSuccess) return VCAS_ERR_CUDA;
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 1; a.accumulate_vw = 0;
-  a.a_done = fast_sampling(h.desc) ? 1 : 0;
-  if (launch_rownorms(&h, dY, X, seed, a.a_done ? &a : nullptr, st) != cudaSuccess) return VCAS_ERR_CUDA;
+  if (launch_rownorms(&h, dY, X, seed, st) != cudaSuccess) return VCAS_ERR_CUDA;
   if (launch_sampler(&h, a, st) != cudaSuccess) return VCAS_ERR_CUDA;
 
   const size_t R = (size_t)N * T;
