@@ -58,8 +58,8 @@ size_t layout(Handle* h, uint8_t* base) {
   if (h->tensor_path) {
     w.packG = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_out);
     w.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
-    w.partial_tiles = carve<float>(cur, 2 * (size_t)h->max_units * 128 * 256);
-    w.tickets = carve<int32_t>(cur, 4 * (size_t)h->max_units);
+    w.partial_tiles = carve<float>(cur, 3 * (size_t)h->max_units * 128 * 256);
+    w.tickets = carve<int32_t>(cur, 6 * (size_t)h->max_units);
   } else {
     w.packG = nullptr;
     w.packX = nullptr;
@@ -70,6 +70,28 @@ size_t layout(Handle* h, uint8_t* base) {
   w.Gact = carve<float>(cur, DW);
   w.mean = carve<float>(cur, DW);
   w.m2 = carve<float>(cur, DW);
+  // second set (variance probe): see Handle::ws2
+  Workspace& v = h->ws2;
+  v = w;
+  v.g = carve<float>(cur, N);
+  v.p = carve<float>(cur, N);
+  v.w = carve<float>(cur, R);
+  v.q = carve<float>(cur, R);
+  v.scaleA = carve<float>(cur, N);
+  v.scaleW = carve<float>(cur, R);
+  v.idxA = carve<int32_t>(cur, N);
+  v.dropA = carve<int32_t>(cur, N);
+  v.idxW = carve<int32_t>(cur, R);
+  v.counts = carve<int32_t>(cur, 8);
+  v.acc = carve<double>(cur, 16);
+  v.partial = carve<double>(cur, PARTIAL_SLOTS);
+  if (h->tensor_path) {
+    v.packG = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_out);
+    v.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
+    v.partial_tiles = w.partial_tiles + (size_t)h->max_units * 128 * 256;   // dW slot of this set = third slot
+    v.tickets = w.tickets + 2 * (size_t)h->max_units;
+  }
+  v.Gact = carve<float>(cur, DW);
   return (size_t)(cur - base);
 }
 
@@ -177,7 +199,8 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   layout(h, reinterpret_cast<uint8_t*>(h->base));
   const int32_t R = desc->N * desc->T;
   if (cudaMemset(h->base, 0, h->bytes) != cudaSuccess ||
-      cudaMemcpy(h->ws.counts + 2, &R, sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+      cudaMemcpy(h->ws.counts + 2, &R, sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(h->ws2.counts + 2, &R, sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
     cudaFree(h->base);
     delete h;
     return VCAS_ERR_CUDA;
@@ -374,16 +397,29 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(launch_probe_welford(h, i, st));
     VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, st));   // the probe draws no SampleW mask
+    // The M draws of SampleA for this batch are independent chains (sampler, pack, product, squared
+    // difference): even draws run on `st` with the first workspace set, odd draws on the side stream with
+    // the second, so that the latency-bound kernels of one chain overlap the product of the other.
+    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
+    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+    const Workspace first = h->ws;
     for (int j = 0; j < M; ++j) {
+      const bool second = (j & 1) != 0;
+      cudaStream_t sj = second ? h->side_stream : st;
+      h->ws = second ? h->ws2 : first;
       SamplerArgs a;
       a.rho = rho; a.nu = nu; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 0; a.accumulate_vw = 1;
       a.seed = seed + (uint64_t)(i * M + j + 1) * 0x9E3779B97F4A7C15ull;
-      VCAS_CUDA(launch_sampler(h, a, st));
-      if (j == 0) VCAS_CUDA(launch_probe_sparsity(h, s_lo, s_hi, st));
-      rc = sampled_dw(h, X_i[i], dY_i[i], rho, h->ws.Gact, st);          // G_act,ij (SampleA only)
+      cudaError_t e = launch_sampler(h, a, sj, second);
+      if (e == cudaSuccess && j == 0) e = launch_probe_sparsity(h, s_lo, s_hi, sj);
+      if (e == cudaSuccess) rc = sampled_dw(h, X_i[i], dY_i[i], rho, h->ws.Gact, sj);   // G_act,ij (SampleA only)
+      if (e == cudaSuccess && rc == VCAS_OK) e = launch_probe_sqdiff(h, sj);
+      h->ws = first;
+      if (e != cudaSuccess) return VCAS_ERR_CUDA;
       if (rc != VCAS_OK) return rc;
-      VCAS_CUDA(launch_probe_sqdiff(h, st));
     }
+    VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
+    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   }
   VCAS_CUDA(launch_probe_finalize(h, M, V_s, V_act, V_w, p_lo, p_hi, st));
   return VCAS_OK;

@@ -39,8 +39,9 @@ struct Workspace {
   // compact operands of the weight-gradient product (tensor path)
   __nv_bfloat16* packG;  // [R_pad, d_out]
   __nv_bfloat16* packX;  // [R_pad, d_in]
-  float* partial_tiles;  // [2 products][max_units][128 * 256] fp32 partial tiles of a split contraction
-  int32_t* tickets;      // [2 products][2 * max_units]: slices stored, slices finished, per tile
+  float* partial_tiles;  // [3][max_units][128 * 256] fp32 partial tiles of a split contraction: dX, dW, and the dW
+                         // of the workspace's second set (see Handle::ws2)
+  int32_t* tickets;      // [3][2 * max_units]: slices stored, slices finished, per tile
   // probe buffers (App. D: the exact gradient, its running mean and running squared deviation)
   float* Gs;       // [d_out, d_in]
   float* Gact;     // [d_out, d_in]
@@ -61,6 +62,10 @@ struct Handle {
   void* base;
   size_t bytes;
   Workspace ws;
+  // Second set of everything a sampled dW chain writes (sampler outputs, packed operands, G_act, counters,
+  // accumulators, block partials, split-contraction slot); the row norms and G_s are shared.  The variance
+  // probe runs its SampleA draws alternately on the two sets and two streams.
+  Workspace ws2;
   uint64_t launches;
   // second stream and fork/join events: the dW branch (pack + product) runs beside the dX product
   cudaStream_t side_stream;
@@ -318,6 +323,7 @@ cudaError_t launch_probe_reset(Handle* h, cudaStream_t st);
 cudaError_t launch_probe_welford(Handle* h, int i, cudaStream_t st);
 cudaError_t launch_probe_sqdiff(Handle* h, cudaStream_t st);
 cudaError_t launch_probe_sparsity(Handle* h, double s_lo, double s_hi, cudaStream_t st);
+// adds the accumulators of the second set to the first (fixed order), then Alg. 1's averages
 cudaError_t launch_probe_finalize(Handle* h, int M, float* V_s, float* V_act, float* V_w,
                                   float* p_lo, float* p_hi, cudaStream_t st);
 

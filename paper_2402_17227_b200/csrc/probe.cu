@@ -111,13 +111,13 @@ __global__ void __launch_bounds__(1024) sparsity_kernel(const float* __restrict_
   }
 }
 
-__global__ void finalize_kernel(const double* __restrict__ acc, int M, float* V_s, float* V_act, float* V_w,
-                                float* p_lo, float* p_hi) {
+__global__ void finalize_kernel(const double* __restrict__ acc, const double* __restrict__ acc2, int M, float* V_s,
+                                float* V_act, float* V_w, float* p_lo, float* p_hi) {
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     const double mm = (double)M * (double)M;
     if (V_s) *V_s = (float)(acc[4] / (double)(M - 1));
-    if (V_act) *V_act = (float)(acc[0] / mm);
-    if (V_w) *V_w = (float)(acc[1] / mm);
+    if (V_act) *V_act = (float)((acc[0] + acc2[0]) / mm);     // even draws + odd draws
+    if (V_w) *V_w = (float)((acc[1] + acc2[1]) / mm);
     if (p_lo) *p_lo = (float)(acc[2] / (double)M);
     if (p_hi) *p_hi = (float)(acc[3] / (double)M);
   }
@@ -134,6 +134,8 @@ int reduce_blocks(size_t n4) {
 
 cudaError_t launch_probe_reset(Handle* h, cudaStream_t st) {
   cudaError_t e = cudaMemsetAsync(h->ws.acc, 0, 16 * sizeof(double), st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->ws2.acc, 0, 16 * sizeof(double), st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->ws2.counts + 4, 0, sizeof(int32_t), st);
   if (e != cudaSuccess) return e;
   return cudaMemsetAsync(h->ws.counts + 4, 0, sizeof(int32_t), st);
 }
@@ -165,7 +167,7 @@ cudaError_t launch_probe_finalize(Handle* h, int M, float* V_s, float* V_act, fl
   const size_t n4 = (size_t)h->desc.d_out * h->desc.d_in / 4;
   reduce_kernel<<<reduce_blocks(n4), 256, 0, st>>>((const float4*)h->ws.m2, nullptr, n4, 1, h->ws.partial,
                                                    h->ws.counts + 4, h->ws.acc + 4);
-  finalize_kernel<<<1, 32, 0, st>>>(h->ws.acc, M, V_s, V_act, V_w, p_lo, p_hi);
+  finalize_kernel<<<1, 32, 0, st>>>(h->ws.acc, h->ws2.acc, M, V_s, V_act, V_w, p_lo, p_hi);
   h->launches += 2;
   return cudaGetLastError();
 }
