@@ -273,6 +273,7 @@ __device__ __forceinline__ int sample_a_warp(const float* g, int N, float rho, c
 
 // The single-CTA register-resident sampling kernel, and with it the SampleA-only kernel that lets the dX
 // product start early, serve layers of at most this many data and rows.
+constexpr int INLINE_A_MAX_N = 128;   // data for which SampleA fits into the dX kernel's spare shared memory
 constexpr int FAST_MAX_N = 1024;
 constexpr int FAST_MAX_R = 16 * 1024;
 inline bool fast_sampling(const vcas_layer_desc& d) {
@@ -309,9 +310,12 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 
 // tensor-core products
 // spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it);
-// second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a)
+// second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a);
+// inline_a != nullptr (N <= INLINE_A_MAX_N): the kernel runs SampleA itself from the row norms with these
+// rho, p_in and seed, and reads no SampleA arrays
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, int spare_sms, bool second_set, cudaStream_t st);
+                           const void* H, void* dX, int spare_sms, bool second_set, const SamplerArgs* inline_a,
+                           cudaStream_t st);
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling

@@ -191,6 +191,34 @@ def test_tensor_path_whole_waves_and_remainder(shape, rho, nu):
     layer.close()
 
 
+@pytest.mark.parametrize("N,T", [(160, 16), (128, 24), (40, 8)])
+def test_tensor_path_many_data(N, T):
+    """Batches on both sides of the limit up to which the dX product derives SampleA in its own prologue
+    (beyond it a separate SampleA kernel feeds it): the kept data, the lists and both products against the
+    oracle, with given and with library-computed probabilities."""
+    d_in, d_out = 128, 192
+    X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.0, sigma_B=0.5)
+    layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
+    Xc, dYc, Wc = cuda(X, dY, W)
+    rho, nu, seed = 0.4, 0.5, 21
+    ref = o.linear_bwd(np64(X), np64(dY), np64(W), N, T, f32(rho), f32(nu), seed)
+    p_in, q_in = torch.from_numpy(ref["p32"]).cuda(), torch.from_numpy(ref["q32"]).cuda()
+    dX, dW = layer.linear_bwd(Xc, dYc, Wc, rho, nu, seed, p_in=p_in, q_in=q_in)
+    s = layer.last_sampling()
+    assert np.array_equal(s.idxA.cpu().numpy(), ref["idxA"]) and np.array_equal(s.idxW.cpu().numpy(), ref["idxW"])
+    assert rel_fro(np64(dX), ref["dX"]) <= tol_for(BF16) and rel_fro(np64(dW), ref["dW"]) <= tol_for(BF16)
+    kept_rows = np.repeat(ref["keepA"], T)
+    assert not np64(dX)[~kept_rows].any()
+    # library-computed probabilities: dX's kept data (from its own SampleA) must be the sampler's
+    dX2, dW2 = layer.linear_bwd(Xc, dYc, Wc, rho, nu, seed)
+    s2 = layer.last_sampling()
+    keep2 = np.zeros(N, bool); keep2[s2.idxA.cpu().numpy()] = True
+    nz = np64(dX2).reshape(N, -1).any(axis=1)
+    assert np.array_equal(nz, keep2 & (np64(dY).reshape(N, -1).any(axis=1)))
+    assert layer.device_status() == 0
+    layer.close()
+
+
 @pytest.mark.parametrize("name,dtype,path", PATHS)
 def test_linear_bwd_end_to_end(name, dtype, path):
     """No overrides: the library's own probabilities, masks and products against the oracle's."""
