@@ -174,6 +174,37 @@ __device__ __forceinline__ float datum_sqnorm_warp(const float* an, int T, int l
   return warp_sum((s0 + s1) + (s2 + s3));
 }
 
+// The same sums for G data n0 .. n0 + G - 1 at once (results for n >= N are meaningless): per datum the
+// additions happen in exactly the order of datum_sqnorm_warp, so the results are bit-identical, but the loads
+// of the G data are in flight together.  For T <= 480 only (longer data keep enough loads in flight alone).
+template <int G>
+__device__ __forceinline__ void datum_sqnorm_warp_multi(const float* a, int T, int n0, int N, int lane, float (&out)[G]) {
+  float s0[G], s1[G], s2[G], s3[G];
+  const float* an[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    s0[g] = s1[g] = s2[g] = s3[g] = 0.f;
+    an[g] = a + (size_t)(n0 + g < N ? n0 + g : N - 1) * T;
+  }
+  int t = lane;
+  for (; t + 96 < T; t += 128) {
+    float v[G][4];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      v[g][0] = __ldcg(an[g] + t); v[g][1] = __ldcg(an[g] + t + 32);
+      v[g][2] = __ldcg(an[g] + t + 64); v[g][3] = __ldcg(an[g] + t + 96);
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) { s0[g] += v[g][0]; s1[g] += v[g][1]; s2[g] += v[g][2]; s3[g] += v[g][3]; }
+  }
+  for (; t < T; t += 32) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) s0[g] += __ldcg(an[g] + t);
+  }
+#pragma unroll
+  for (int g = 0; g < G; ++g) out[g] = warp_sum((s0[g] + s1[g]) + (s2[g] + s3[g]));
+}
+
 // Keep probabilities proportional to v, capped at 1, summing to `budget` (the minimiser of
 // sum (1-p)/p v^2 under that budget): p = min(1, c v).  The saturated set is grown from empty; c only
 // increases, so the iteration reaches the least fixed point, which is the unique solution.  Value i of the

@@ -386,20 +386,33 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     __shared__ int32_t s_idx[INLINE_A_MAX_N], s_drop[INLINE_A_MAX_N];
     __shared__ int s_cnt;
     if (P.inline_a) {
-      // SampleA (Sec. 4.1) by the four epilogue warps: data norms, then probabilities, masks and lists in warp 0
-      if (warp < 4) {
-        for (int n = warp; n < P.N; n += 4) {
+      // SampleA (Sec. 4.1): data norms by all warps (eight data per warp at a time when the data are short,
+      // so that their loads overlap), then probabilities, masks and lists in warp 0
+      constexpr int NW = NUM_THREADS / 32;
+      if (P.T <= 480) {
+        for (int n0 = warp * 8; n0 < P.N; n0 += NW * 8) {
+          float ss[8];
+          datum_sqnorm_warp_multi<8>(P.a_norms, P.T, n0, P.N, lane, ss);
+          if (lane < 8 && n0 + lane < P.N) {
+            float mine = ss[0];
+#pragma unroll
+            for (int g = 1; g < 8; ++g) mine = lane == g ? ss[g] : mine;
+            s_scale[n0 + lane] = sqrtf(mine);
+          }
+        }
+      } else {
+        for (int n = warp; n < P.N; n += NW) {
           const float ss = datum_sqnorm_warp(P.a_norms + (size_t)n * P.T, P.T, lane);
           if (lane == 0) s_scale[n] = sqrtf(ss);
         }
-        epi_bar();
-        if (warp == 0) {
-          SampleAOut o;
-          o.p = nullptr; o.scaleA = s_scale; o.idxA = s_idx; o.dropA = s_drop;
-          o.sh_p = nullptr; o.sh_scaleA = nullptr;
-          const int kept = sample_a_warp<INLINE_A_MAX_N / 32>(s_scale, P.N, P.rho, P.p_in, P.seed, o, lane);
-          if (lane == 0) s_cnt = kept;
-        }
+      }
+      __syncthreads();
+      if (warp == 0) {
+        SampleAOut o;
+        o.p = nullptr; o.scaleA = s_scale; o.idxA = s_idx; o.dropA = s_drop;
+        o.sh_p = nullptr; o.sh_scaleA = nullptr;
+        const int kept = sample_a_warp<INLINE_A_MAX_N / 32>(s_scale, P.N, P.rho, P.p_in, P.seed, o, lane);
+        if (lane == 0) s_cnt = kept;
       }
       __syncthreads();
       idxA = s_idx; dropA = s_drop; scaleA = s_scale;
