@@ -275,7 +275,7 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     mark(h, 1, st);
     VCAS_CUDA(launch_sampler(h, a, st));
     mark(h, 2, st);
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, nullptr, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, st));
     mark(h, 3, st);
     mark(h, 6, st);
     VCAS_CUDA(launch_pack(h, dY, X, st));
@@ -283,20 +283,18 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, st));
     mark(h, 5, st);
   } else if (fast_sampling(h->desc)) {
-    // The dX product needs SampleA only, so it follows the row norms directly on `st` as a programmatic
-    // dependent launch: with at most INLINE_A_MAX_N data every CTA of the product derives SampleA itself in
-    // its prologue; with more, a small SampleA-only kernel sits between the two.  The full sampling kernel
-    // (which draws the same SampleA masks, then SampleW), the pack and the dW product run beside them on the
-    // handle's side stream and are joined back before the call's work ends on `st`.  The dX grid leaves one
-    // SM free: the sampling kernel is a single CTA that needs a whole SM's registers.
-    const bool inline_a = h->desc.N <= INLINE_A_MAX_N;
+    // The dX product needs SampleA only.  On `st`, a small SampleA-only kernel and the dX product follow the
+    // row norms as programmatic dependent launches; the full sampling kernel (which draws the same SampleA
+    // masks, then SampleW), the pack and the dW product run beside them on the handle's side stream and are
+    // joined back before the call's work ends on `st`.  The dX grid leaves one SM free: the sampling kernel
+    // is a single CTA that needs a whole SM's registers.
     VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
     VCAS_CUDA(launch_sampler(h, a, h->side_stream, true));
-    if (!inline_a) VCAS_CUDA(launch_sample_a(h, a, st));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, !inline_a, inline_a ? &a : nullptr, st));
+    VCAS_CUDA(launch_sample_a(h, a, st));
     VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, st));
     VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, h->side_stream));
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
     VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
@@ -306,7 +304,7 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     VCAS_CUDA(launch_sampler(h, a, st));
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, nullptr, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, st));
     VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
     VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, h->side_stream));
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
@@ -336,7 +334,7 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
   }
   mark_dense(h, 0, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, false, nullptr, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, false, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }

@@ -174,37 +174,6 @@ __device__ __forceinline__ float datum_sqnorm_warp(const float* an, int T, int l
   return warp_sum((s0 + s1) + (s2 + s3));
 }
 
-// The same sums for G data n0 .. n0 + G - 1 at once (results for n >= N are meaningless): per datum the
-// additions happen in exactly the order of datum_sqnorm_warp, so the results are bit-identical, but the loads
-// of the G data are in flight together.  For T <= 480 only (longer data keep enough loads in flight alone).
-template <int G>
-__device__ __forceinline__ void datum_sqnorm_warp_multi(const float* a, int T, int n0, int N, int lane, float (&out)[G]) {
-  float s0[G], s1[G], s2[G], s3[G];
-  const float* an[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    s0[g] = s1[g] = s2[g] = s3[g] = 0.f;
-    an[g] = a + (size_t)(n0 + g < N ? n0 + g : N - 1) * T;
-  }
-  int t = lane;
-  for (; t + 96 < T; t += 128) {
-    float v[G][4];
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      v[g][0] = __ldcg(an[g] + t); v[g][1] = __ldcg(an[g] + t + 32);
-      v[g][2] = __ldcg(an[g] + t + 64); v[g][3] = __ldcg(an[g] + t + 96);
-    }
-#pragma unroll
-    for (int g = 0; g < G; ++g) { s0[g] += v[g][0]; s1[g] += v[g][1]; s2[g] += v[g][2]; s3[g] += v[g][3]; }
-  }
-  for (; t < T; t += 32) {
-#pragma unroll
-    for (int g = 0; g < G; ++g) s0[g] += __ldcg(an[g] + t);
-  }
-#pragma unroll
-  for (int g = 0; g < G; ++g) out[g] = warp_sum((s0[g] + s1[g]) + (s2[g] + s3[g]));
-}
-
 // Keep probabilities proportional to v, capped at 1, summing to `budget` (the minimiser of
 // sum (1-p)/p v^2 under that budget): p = min(1, c v).  The saturated set is grown from empty; c only
 // increases, so the iteration reaches the least fixed point, which is the unique solution.  Value i of the
@@ -304,7 +273,6 @@ __device__ __forceinline__ int sample_a_warp(const float* g, int N, float rho, c
 
 // The single-CTA register-resident sampling kernel, and with it the SampleA-only kernel that lets the dX
 // product start early, serve layers of at most this many data and rows.
-constexpr int INLINE_A_MAX_N = 128;   // data for which SampleA fits into the dX kernel's spare shared memory
 constexpr int FAST_MAX_N = 1024;
 constexpr int FAST_MAX_R = 16 * 1024;
 inline bool fast_sampling(const vcas_layer_desc& d) {
@@ -341,12 +309,9 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 
 // tensor-core products
 // spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it);
-// second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a);
-// inline_a != nullptr (N <= INLINE_A_MAX_N): the kernel runs SampleA itself from the row norms with these
-// rho, p_in and seed, and reads no SampleA arrays
+// second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a)
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, int spare_sms, bool second_set, const SamplerArgs* inline_a,
-                           cudaStream_t st);
+                           const void* H, void* dX, int spare_sms, bool second_set, cudaStream_t st);
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling

@@ -255,14 +255,6 @@ struct GemmParams {
   int d_in, d_out;
   // dX: A = dY viewed [N][T][d_out] (K-major, one TMA box = 128 tokens x 64 k of one datum),
   //     B = W [d_out][d_in] (MN-major: n contiguous)
-  // SampleA inside the kernel (inline_a = 1, N <= INLINE_A_MAX_N): every CTA derives the kept / dropped data
-  // and their scales from the squared row norms itself (same warp-level code as the sampling kernels, so the
-  // same masks), into its own shared memory; the arrays below are then not read.
-  int inline_a;
-  const float* a_norms;    // [N*T] squared row norms of dY
-  float rho;
-  const float* p_in;       // optional given keep probabilities
-  uint64_t seed;
   const int32_t* idxA;     // kept data
   const int32_t* dropA;    // dropped data
   const int32_t* counts;   // counts[0] = number of kept data
@@ -285,13 +277,13 @@ struct Decomp {
   int head256, per_datum256;   // parts 1 and 2: 256-row tiles left to part 1; dX: 256-row tiles per datum
 };
 
-// cntA: number of kept data (dX only)
 template <int MODE, int BN, int MH>
-__device__ __forceinline__ Decomp decompose(const GemmParams& P, int cntA) {
+__device__ __forceinline__ Decomp decompose(const GemmParams& P) {
   constexpr int BMT = BM * MH;
   Decomp d;
   d.ntiles = (P.d_in + BN - 1) / BN;
   if (MODE == MODE_DX) {
+    const int cntA = P.dense ? P.N : P.counts[0];
     d.per_datum = ((P.T + BMT - 1) / BMT) * d.ntiles;
     d.gemm_tiles = cntA * d.per_datum;
     d.zero_tiles = (P.N - cntA) * d.per_datum;
@@ -310,7 +302,7 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P, int cntA) {
     int total256;
     if (MODE == MODE_DX) {
       d.per_datum256 = ((P.T + 2 * BM - 1) / (2 * BM)) * d.ntiles;
-      total256 = cntA * d.per_datum256;
+      total256 = (P.dense ? P.N : P.counts[0]) * d.per_datum256;
     } else {
       total256 = d.kblocks > 0 ? ((P.d_out + 2 * BM - 1) / (2 * BM)) * d.ntiles : 0;
     }
@@ -377,51 +369,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const uint32_t tmem_base = setup<BN, MH>(s, warp, tid);
   volatile int* abort_flag = s.abort_flag;
   pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
-  const int32_t* idxA = P.idxA;
-  const int32_t* dropA = P.dropA;
-  const float* scaleA = P.scaleA;
-  int cntA = 0;
-  if constexpr (MODE == MODE_DX) {
-    __shared__ float s_scale[INLINE_A_MAX_N];
-    __shared__ int32_t s_idx[INLINE_A_MAX_N], s_drop[INLINE_A_MAX_N];
-    __shared__ int s_cnt;
-    if (P.inline_a) {
-      // SampleA (Sec. 4.1): data norms by all warps (eight data per warp at a time when the data are short,
-      // so that their loads overlap), then probabilities, masks and lists in warp 0
-      constexpr int NW = NUM_THREADS / 32;
-      if (P.T <= 480) {
-        for (int n0 = warp * 8; n0 < P.N; n0 += NW * 8) {
-          float ss[8];
-          datum_sqnorm_warp_multi<8>(P.a_norms, P.T, n0, P.N, lane, ss);
-          if (lane < 8 && n0 + lane < P.N) {
-            float mine = ss[0];
-#pragma unroll
-            for (int g = 1; g < 8; ++g) mine = lane == g ? ss[g] : mine;
-            s_scale[n0 + lane] = sqrtf(mine);
-          }
-        }
-      } else {
-        for (int n = warp; n < P.N; n += NW) {
-          const float ss = datum_sqnorm_warp(P.a_norms + (size_t)n * P.T, P.T, lane);
-          if (lane == 0) s_scale[n] = sqrtf(ss);
-        }
-      }
-      __syncthreads();
-      if (warp == 0) {
-        SampleAOut o;
-        o.p = nullptr; o.scaleA = s_scale; o.idxA = s_idx; o.dropA = s_drop;
-        o.sh_p = nullptr; o.sh_scaleA = nullptr;
-        const int kept = sample_a_warp<INLINE_A_MAX_N / 32>(s_scale, P.N, P.rho, P.p_in, P.seed, o, lane);
-        if (lane == 0) s_cnt = kept;
-      }
-      __syncthreads();
-      idxA = s_idx; dropA = s_drop; scaleA = s_scale;
-      cntA = s_cnt;
-    } else {
-      cntA = P.dense ? P.N : P.counts[0];
-    }
-  }
-  const Decomp D = decompose<MODE, BN, MH>(P, cntA);
+  const Decomp D = decompose<MODE, BN, MH>(P);
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
@@ -436,7 +384,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         {
           int k;
           tile_coords<MODE>(P, D, tile, k, c0, c1);
-          if (MODE == MODE_DX) n = P.dense ? k : idxA[k];
+          if (MODE == MODE_DX) n = P.dense ? k : P.idxA[k];
         }
         for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(&s.empty[stage], phase ^ 1u, abort_flag, P.status);
@@ -514,12 +462,12 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const int rem = tile % D.per_datum;
           c = rem / D.ntiles; nt = rem % D.ntiles;
         }
-        const int n = is_gemm ? (P.dense ? k : idxA[k]) : dropA[k];
+        const int n = is_gemm ? (P.dense ? k : P.idxA[k]) : P.dropA[k];
         row0 = (size_t)n * P.T + (size_t)c * BMT;
         rows_valid = min(BMT, P.T - c * BMT);
         col0 = nt * BN;
         n_out = n; t_out = c * BMT;
-        if (is_gemm && !P.dense) sc = scaleA[n];
+        if (is_gemm && !P.dense) sc = P.scaleA[n];
       } else {
         int k, mt, nt;
         if (is_gemm) { tile_coords<MODE>(P, D, tile, k, mt, nt); } else { mt = tile / D.ntiles; nt = tile % D.ntiles; }
@@ -952,7 +900,7 @@ void common_params(Handle* h, GemmParams& P, int which) {
 }  // namespace
 
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint, const void* H,
-                           void* dX, int spare_sms, bool second_set, const SamplerArgs* inline_a, cudaStream_t st) {
+                           void* dX, int spare_sms, bool second_set, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -977,10 +925,6 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   common_params(h, P, 0);
   P.idxA = h->ws.idxA; P.dropA = h->ws.dropA; P.counts = h->ws.counts; P.scaleA = h->ws.scaleA;
   if (second_set) { P.idxA = h->ws.idxA2; P.dropA = h->ws.dropA2; P.counts = h->ws.counts + 6; P.scaleA = h->ws.scaleA2; }
-  if (inline_a != nullptr) {
-    if (dense || d.N > INLINE_A_MAX_N) return cudaErrorInvalidValue;
-    P.inline_a = 1; P.a_norms = h->ws.a; P.rho = inline_a->rho; P.p_in = inline_a->p_in; P.seed = inline_a->seed;
-  }
   P.H = (const __nv_bfloat16*)H; P.dX = (__nv_bfloat16*)dX;
   P.N = d.N; P.T = d.T; P.dense = dense ? 1 : 0;
   P.a_tx_bytes = (d.T < BM ? d.T : BM) * BK * 2;

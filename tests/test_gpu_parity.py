@@ -193,9 +193,9 @@ def test_tensor_path_whole_waves_and_remainder(shape, rho, nu):
 
 @pytest.mark.parametrize("N,T", [(160, 16), (128, 24), (40, 8)])
 def test_tensor_path_many_data(N, T):
-    """Batches on both sides of the limit up to which the dX product derives SampleA in its own prologue
-    (beyond it a separate SampleA kernel feeds it): the kept data, the lists and both products against the
-    oracle, with given and with library-computed probabilities."""
+    """Batches of more data than one warp holds in one slot per lane (SampleA's wide variant) and fewer: the
+    kept data, the lists and both products against the oracle with given probabilities; with the library's
+    own, the dX product's kept data (from the SampleA-only kernel) must be those of the sampling kernel."""
     d_in, d_out = 128, 192
     X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.0, sigma_B=0.5)
     layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
