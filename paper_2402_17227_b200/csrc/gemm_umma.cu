@@ -277,7 +277,7 @@ struct Decomp {
   int head256, per_datum256;   // parts 1 and 2: 256-row tiles left to part 1; dX: 256-row tiles per datum
 };
 
-template <int MODE, int BN, int MH>
+template <int MODE, int BN, int MH, bool LEAN>
 __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
   constexpr int BMT = BM * MH;
   Decomp d;
@@ -319,7 +319,7 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
       if (split_req > d.kblocks / 4) split_req = d.kblocks / 4;      // slices of at least four k-blocks
     }
   }
-  int S = (split_req < 1 || MH == 2) ? 1 : split_req;
+  int S = (split_req < 1 || MH == 2 || LEAN) ? 1 : split_req;
   if (S > d.kblocks) S = d.kblocks > 0 ? d.kblocks : 1;
   if (d.gemm_tiles > 0 && (long)d.gemm_tiles * S > P.max_units) S = P.max_units / d.gemm_tiles;
   if (S > (int)gridDim.x) S = (int)gridDim.x;
@@ -356,7 +356,10 @@ __device__ __forceinline__ void tile_coords(const GemmParams& P, const Decomp& D
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <int MODE, int BN, int MH>
+// LEAN: the instance for unsliced contractions (S = 1), without the code of the slice exchange; the other
+// instance has only the slice exchange (a contraction that ends up in one slice still goes through it).
+// Two instances because the product kernels are short: code that a launch never runs still costs it time.
+template <int MODE, int BN, int MH, bool LEAN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, GemmParams P) {
@@ -369,7 +372,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const uint32_t tmem_base = setup<BN, MH>(s, warp, tid);
   volatile int* abort_flag = s.abort_flag;
   pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
-  const Decomp D = decompose<MODE, BN, MH>(P);
+  const Decomp D = decompose<MODE, BN, MH, LEAN>(P);
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
@@ -560,7 +563,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (has1) store8((row0 + rb) * ld + col0 + cb * 8, sc, fb);
         }
       };
-      if (D.S == 1) {
+      if constexpr (LEAN) {
         // ---- whole contraction in this unit: accumulator -> (rescale, GELU', convert) -> swizzled
         // shared memory -> TMA store of 32 rows x 128 bytes per warp (rows / columns outside the
         // tensor are clipped by the tensor map, so rows of the next datum are never touched)
@@ -623,6 +626,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         __syncwarp();
         continue;
       }
+      if constexpr (!LEAN) {
       // ---- one slice of the contraction: store the fp32 partial tile.  Layout in the workspace:
       // [32-column chunk][row][32 floats], the eight 16-byte slots of a row swizzled by (row & 7) as
       // staged in shared memory, so each warp moves its 32 rows of a chunk with one 4 KB bulk copy.
@@ -684,6 +688,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           P.tickets[P.max_units + tile] = 0;
         }
       }
+      }  // !LEAN
     }
     // zero tiles (rows of dropped data; nothing kept at all): taken from the far end of the grid first,
     // where CTAs have no product units
@@ -833,12 +838,12 @@ Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks,
   return best;
 }
 
-template <int MODE, int BN, int MH>
-cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P0,
+template <int MODE, int BN, int MH, bool LEAN>
+cudaError_t run_gemm_k(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P0,
                      long max_items, int ctas, bool pdl, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN, MH, LEAN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          TileCfg<BN, MH>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
@@ -858,9 +863,20 @@ cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, cons
     cfg.numAttrs += 1;
   }
   cfg.gridDim = dim3((unsigned)grid);
-  cudaError_t e = cudaLaunchKernelEx(&cfg, umma_kernel<MODE, BN, MH>, a, b, c, P);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, umma_kernel<MODE, BN, MH, LEAN>, a, b, c, P);
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+template <int MODE, int BN, int MH>
+cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P,
+                     long max_items, int ctas, bool pdl, cudaStream_t st) {
+  if constexpr (MH == 2) {
+    return run_gemm_k<MODE, BN, MH, true>(h, a, b, c, P, max_items, ctas, pdl, st);
+  } else {
+    if (P.split_k == 1) return run_gemm_k<MODE, BN, MH, true>(h, a, b, c, P, max_items, ctas, pdl, st);
+    return run_gemm_k<MODE, BN, MH, false>(h, a, b, c, P, max_items, ctas, pdl, st);
+  }
 }
 
 template <int MODE>
