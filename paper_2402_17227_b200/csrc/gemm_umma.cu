@@ -220,7 +220,7 @@ __device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid
   return *(volatile uint32_t*)s.tmem_holder;
 }
 
-__device__ __forceinline__ float gelu_prime(float x) {
+__device__ __noinline__ float gelu_prime(float x) {   // one copy: rarely run, and the product kernels are sensitive to code size
   const float Phi = 0.5f * (1.0f + erff(x * 0.70710678118654752f));
   const float phi = 0.39894228040143268f * expf(-0.5f * x * x);
   return fmaf(x, phi, Phi);
