@@ -116,7 +116,7 @@ int sampled_dw(Handle* h, const void* X, const void* dY, float keep_hint, float*
   if (h->tensor_path) {
     VCAS_CUDA(launch_pack(h, dY, X, st));
     const int hint = (int)(keep_hint * (float)(h->desc.N * h->desc.T)) + 1;
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, out, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, true, out, st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, out, st));
   }
@@ -131,9 +131,11 @@ inline void mark_dense(Handle* h, int k, cudaStream_t st) {
   if (h->prof_enabled && h->prof_dense_calls < PROF_RING) cudaEventRecord(h->ev_dense[h->prof_dense_calls * 4 + k], st);
 }
 
-int dense_dw(Handle* h, const void* X, const void* dY, float* out, cudaStream_t st) {
+// concurrent: the dX product of the same call runs beside it
+int dense_dw(Handle* h, const void* X, const void* dY, bool concurrent, float* out, cudaStream_t st) {
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, h->desc.N * h->desc.T, out, st));
+    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, h->desc.N * h->desc.T, concurrent, out,
+                             st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, nullptr, nullptr, h->ws.counts + 2, out, st));
   }
@@ -275,12 +277,12 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     mark(h, 1, st);
     VCAS_CUDA(launch_sampler(h, a, st));
     mark(h, 2, st);
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, true, st));
     mark(h, 3, st);
     mark(h, 6, st);
     VCAS_CUDA(launch_pack(h, dY, X, st));
     mark(h, 4, st);
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, true, dW, st));
     mark(h, 5, st);
   } else if (fast_sampling(h->desc)) {
     // The dX product needs SampleA only.  On `st`, a small SampleA-only kernel and the dX product follow the
@@ -294,8 +296,8 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     VCAS_CUDA(launch_sampler(h, a, h->side_stream, true));
     VCAS_CUDA(launch_sample_a(h, a, st));
     VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, st));
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, h->side_stream));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, true, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, true, dW, h->side_stream));
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
     VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   } else {
@@ -304,9 +306,9 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     VCAS_CUDA(launch_sampler(h, a, st));
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, true, st));
     VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, dW, h->side_stream));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, true, dW, h->side_stream));
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
     VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   }
@@ -334,13 +336,13 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
   }
   mark_dense(h, 0, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, false, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, false, true, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }
   mark_dense(h, 1, st);
   mark_dense(h, 3, sw);
-  const int rc = dense_dw(h, X, dY, dW, sw);
+  const int rc = dense_dw(h, X, dY, true, dW, sw);
   mark_dense(h, 2, sw);
   if (fork) {
     VCAS_CUDA(cudaEventRecord(h->ev_join, sw));
@@ -393,7 +395,7 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
   if (s_hi > 1.0) s_hi = 1.0;
   VCAS_CUDA(launch_probe_reset(h, st));
   for (int i = 0; i < M; ++i) {
-    int rc = dense_dw(h, X_i[i], dY_i[i], h->ws.Gs, st);            // G_s,i
+    int rc = dense_dw(h, X_i[i], dY_i[i], false, h->ws.Gs, st);     // G_s,i
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(launch_probe_welford(h, i, st));
     VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, st));   // the probe draws no SampleW mask

@@ -309,14 +309,15 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 
 // tensor-core products
 // spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it);
-// second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a)
+// second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a);
+// concurrent: the call's other product runs beside this one (tiling is then chosen for the pair)
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, int spare_sms, bool second_set, cudaStream_t st);
+                           const void* H, void* dX, int spare_sms, bool second_set, bool concurrent, cudaStream_t st);
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity,
-                           const int32_t* cnt, int cnt_hint, float* dW, cudaStream_t st);
+                           const int32_t* cnt, int cnt_hint, bool concurrent, float* dW, cudaStream_t st);
 
 // probe reductions
 cudaError_t launch_probe_reset(Handle* h, cudaStream_t st);

@@ -795,9 +795,14 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
 struct Plan { int bn, split, mh; };   // mh: 1 = 128-row tiles, 2 = 256-row tiles, 3 = 256-row whole waves + 128-row remainder
 // row_tiles128: number of 128-row tile rows (for dX: kept data x 128-token chunks).  A 256-row tile
 // (mh = 2) covers two of them; its k-block costs about 0.62 us for twice the work.
-// remainder_ok: 256-row tiles may leave a last partial wave to a second launch with 128-row tiles (mh = 3)
+// remainder_ok: 256-row tiles may leave a last partial wave to a second launch with 128-row tiles (mh = 3).
+// concurrent: the other product of the call runs at the same time on another stream; the two then share the
+// SMs, and what counts is the SM time the units take in total (taken as twice this product's), not only
+// how soon this product alone would finish: measured on the benchmark layer, slicing a contraction that runs
+// beside the other product makes the pair slower (dense call 58.9 us with the dW contraction in two slices,
+// 51.6 us unsliced).
 Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks, int num_sms, int max_units,
-                int force_bn, int force_split, bool remainder_ok) {
+                int force_bn, int force_split, bool remainder_ok, bool concurrent) {
   const int widths[3] = {256, 128, 64};
   const double c_kb[3] = {0.50, 0.45, 0.43};
   Plan best = {256, 1, 1};
@@ -815,13 +820,16 @@ Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks,
       const long units = tiles * sp;
       const double waves = (double)((units + num_sms - 1) / num_sms);
       const double unit_fixed = sp > 1 ? 11.0 + 0.25 * sp : 4.0;
-      const double t = waves * ((double)((kblocks + sp - 1) / sp) * c_kb[i] + unit_fixed);
+      const double unit = (double)((kblocks + sp - 1) / sp) * c_kb[i] + unit_fixed;
+      double t = waves * unit;
+      if (concurrent && t < 2.0 * (double)units * unit / num_sms) t = 2.0 * (double)units * unit / num_sms;
       if (t < best_t - 1e-9) { best_t = t; best = {widths[i], sp, 1}; }
     }
     if (widths[i] == 256 && force_split <= 1) {                        // 256 x 256 tiles, never sliced
       const long units = row_tiles256 * ntiles;
       const double wave = (double)kblocks * 0.62 + 7.0;
-      const double t = (double)((units + num_sms - 1) / num_sms) * wave;
+      double t = (double)((units + num_sms - 1) / num_sms) * wave;
+      if (concurrent && t < 2.0 * (double)units * wave / num_sms) t = 2.0 * (double)units * wave / num_sms;
       if (t < best_t - 1e-9) { best_t = t; best = {256, 1, 2}; }
       const long frac = units % num_sms;
       if (remainder_ok && frac > 0 && 2 * frac <= num_sms) {            // whole waves, then the rest as sliced 128-row tiles
@@ -830,7 +838,8 @@ Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks,
         if (sp > kblocks / 4) sp = kblocks / 4;
         if (sp < 1) sp = 1;
         const double tail = (double)((kblocks + sp - 1) / sp) * 0.50 + (sp > 1 ? 11.0 + 0.25 * sp : 4.0) + 4.0;
-        const double t2 = (double)(units / num_sms) * wave + tail;
+        double t2 = (double)(units / num_sms) * wave + tail;
+        if (concurrent) t2 *= 2.0;        // (many units: the SM time is what the waves add up to)
         if (t2 < best_t - 1e-9) { best_t = t2; best = {256, 1, 3}; }
       }
     }
@@ -916,7 +925,7 @@ void common_params(Handle* h, GemmParams& P, int which) {
 }  // namespace
 
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint, const void* H,
-                           void* dX, int spare_sms, bool second_set, cudaStream_t st) {
+                           void* dX, int spare_sms, bool second_set, bool concurrent, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -952,7 +961,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   // the halves of a 256-row tile must both hold rows for the remainder launch to take them over
   const bool rem_ok = h->tune_tile_m != 2 && ((d.T % (2 * BM)) == 0 || (d.T % (2 * BM)) > BM);
   Plan plan = plan_tiles(nk * chunks, nk * chunks2, d.d_in, (d.d_out + BK - 1) / BK, ctas, h->max_units,
-                         h->tune_dx_tile_n, h->tune_dx_split_k, rem_ok);
+                         h->tune_dx_tile_n, h->tune_dx_split_k, rem_ok, concurrent);
   if (h->tune_tile_m == 1) plan.mh = 1;
   if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
   if (h->tune_tile_m == 3 && plan.bn == 256 && rem_ok) { plan.mh = 3; plan.split = 1; }
@@ -974,7 +983,7 @@ cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t s
 }
 
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity, const int32_t* cnt,
-                           int cnt_hint, float* dW, cudaStream_t st) {
+                           int cnt_hint, bool concurrent, float* dW, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -1001,7 +1010,7 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
   const long mtiles = (d.d_out + BM - 1) / BM, mtiles2 = (d.d_out + 2 * BM - 1) / (2 * BM);
   const bool rem_ok = h->tune_tile_m != 2 && ((d.d_out % (2 * BM)) == 0 || (d.d_out % (2 * BM)) > BM);
   Plan plan = plan_tiles(mtiles, mtiles2, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
-                         h->tune_dw_tile_n, h->tune_dw_split_k, rem_ok);
+                         h->tune_dw_tile_n, h->tune_dw_split_k, rem_ok, concurrent);
   if (h->tune_tile_m == 1) plan.mh = 1;
   if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
   if (h->tune_tile_m == 3 && plan.bn == 256 && rem_ok) { plan.mh = 3; plan.split = 1; }
