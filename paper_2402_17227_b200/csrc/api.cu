@@ -116,7 +116,7 @@ int sampled_dw(Handle* h, const void* X, const void* dY, float keep_hint, float*
   if (h->tensor_path) {
     VCAS_CUDA(launch_pack(h, dY, X, st));
     const int hint = (int)(keep_hint * (float)(h->desc.N * h->desc.T)) + 1;
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, true, out, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, nullptr, out, st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, out, st));
   }
@@ -131,11 +131,10 @@ inline void mark_dense(Handle* h, int k, cudaStream_t st) {
   if (h->prof_enabled && h->prof_dense_calls < PROF_RING) cudaEventRecord(h->ev_dense[h->prof_dense_calls * 4 + k], st);
 }
 
-// concurrent: the dX product of the same call runs beside it
-int dense_dw(Handle* h, const void* X, const void* dY, bool concurrent, float* out, cudaStream_t st) {
+// plan: the tiling made for a call whose dX product runs beside it (nullptr: planned alone)
+int dense_dw(Handle* h, const void* X, const void* dY, const Plan* plan, float* out, cudaStream_t st) {
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, h->desc.N * h->desc.T, concurrent, out,
-                             st));
+    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, h->desc.N * h->desc.T, plan, out, st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, nullptr, nullptr, h->ws.counts + 2, out, st));
   }
@@ -184,6 +183,7 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->prof_calls = h->prof_dense_calls = 0;
   h->tune_dx_tile_n = h->tune_dw_tile_n = h->tune_dx_split_k = h->tune_dw_split_k = 0;
   h->tune_tile_m = 0;
+  h->plan_valid = false;
   cudaDeviceProp prop;
   if (cudaGetDevice(&h->device) != cudaSuccess || cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
     delete h;
@@ -258,6 +258,9 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   SamplerArgs a;
   a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
   const int hint = (int)(rho * nu * (float)(h->desc.N * h->desc.T)) + 1;
+  const bool early_dx = fast_sampling(h->desc);     // dX forks right after the row norms
+  Plan px = {256, 1, 1}, pw = {256, 1, 1};
+  if (h->tensor_path) plan_products(h, false, rho, hint, early_dx ? 1 : 0, &px, &pw);
   if (!h->tensor_path) {
     mark(h, 0, st);
     VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
@@ -277,14 +280,14 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     mark(h, 1, st);
     VCAS_CUDA(launch_sampler(h, a, st));
     mark(h, 2, st);
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, true, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, early_dx ? 1 : 0, false, &px, st));
     mark(h, 3, st);
     mark(h, 6, st);
     VCAS_CUDA(launch_pack(h, dY, X, st));
     mark(h, 4, st);
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, true, dW, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, &pw, dW, st));
     mark(h, 5, st);
-  } else if (fast_sampling(h->desc)) {
+  } else if (early_dx) {
     // The dX product needs SampleA only.  On `st`, a small SampleA-only kernel and the dX product follow the
     // row norms as programmatic dependent launches; the full sampling kernel (which draws the same SampleA
     // masks, then SampleW), the pack and the dW product run beside them on the handle's side stream and are
@@ -296,8 +299,8 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     VCAS_CUDA(launch_sampler(h, a, h->side_stream, true));
     VCAS_CUDA(launch_sample_a(h, a, st));
     VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, true, st));
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, true, dW, h->side_stream));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, &px, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, &pw, dW, h->side_stream));
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
     VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   } else {
@@ -306,9 +309,9 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
     VCAS_CUDA(launch_sampler(h, a, st));
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, true, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, &px, st));
     VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, true, dW, h->side_stream));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, &pw, dW, h->side_stream));
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
     VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   }
@@ -334,15 +337,17 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
     sw = h->side_stream;
   }
+  Plan px = {256, 1, 1}, pw = {256, 1, 1};
+  if (h->tensor_path) plan_products(h, true, 1.0f, h->desc.N * h->desc.T, 0, &px, &pw);
   mark_dense(h, 0, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, false, true, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, false, &px, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }
   mark_dense(h, 1, st);
   mark_dense(h, 3, sw);
-  const int rc = dense_dw(h, X, dY, true, dW, sw);
+  const int rc = dense_dw(h, X, dY, h->tensor_path ? &pw : nullptr, dW, sw);
   mark_dense(h, 2, sw);
   if (fork) {
     VCAS_CUDA(cudaEventRecord(h->ev_join, sw));
@@ -395,7 +400,7 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
   if (s_hi > 1.0) s_hi = 1.0;
   VCAS_CUDA(launch_probe_reset(h, st));
   for (int i = 0; i < M; ++i) {
-    int rc = dense_dw(h, X_i[i], dY_i[i], false, h->ws.Gs, st);     // G_s,i
+    int rc = dense_dw(h, X_i[i], dY_i[i], nullptr, h->ws.Gs, st);   // G_s,i
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(launch_probe_welford(h, i, st));
     VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, st));   // the probe draws no SampleW mask

@@ -51,6 +51,11 @@ struct Workspace {
 
 constexpr int PARTIAL_SLOTS = 4096;
 
+// Tiling of one tensor-core product: tile width, slices of the contraction, and tile height
+// (mh: 1 = 128-row tiles, 2 = 256-row tiles, 3 = 256-row tiles for whole waves + 128-row tiles for the rest).
+struct Plan { int bn, split, mh; };
+constexpr int PLAN_KEY_INTS = 9;
+
 struct Handle {
   vcas_layer_desc desc;
   vcas_config cfg;
@@ -77,6 +82,10 @@ struct Handle {
   int prof_calls, prof_dense_calls;
   // tuning overrides (vcas_set_tuning); 0 = choose automatically
   int tune_dx_tile_n, tune_dw_tile_n, tune_dx_split_k, tune_dw_split_k;
+  // the last pair of plans made for the two products of a call, and what it was made for (plan_products)
+  bool plan_valid;
+  int plan_key[PLAN_KEY_INTS];
+  Plan plan_dx, plan_dw;
   int tune_tile_m;   // 0 auto, 1: 128-row tiles only, 2: 256-row tiles whenever the width is 256, 3: 256-row tiles for
                      // whole waves of CTAs and 128-row tiles, their contraction sliced, for the rest
 };
@@ -310,14 +319,18 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 // tensor-core products
 // spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it);
 // second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a);
-// concurrent: the call's other product runs beside this one (tiling is then chosen for the pair)
+// pair_plan: the tiling chosen by plan_products for a call whose two products run at the same time
+// (nullptr: chosen here, for this product alone)
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, int spare_sms, bool second_set, bool concurrent, cudaStream_t st);
+                           const void* H, void* dX, int spare_sms, bool second_set, const Plan* pair_plan, cudaStream_t st);
 cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity,
-                           const int32_t* cnt, int cnt_hint, bool concurrent, float* dW, cudaStream_t st);
+                           const int32_t* cnt, int cnt_hint, const Plan* pair_plan, float* dW, cudaStream_t st);
+// Tilings of the dX and dW products of one call, chosen together because they share the SMs (cached in the
+// handle until the expected kept counts or the tuning overrides change).
+void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spare_sms, Plan* dx, Plan* dw);
 
 // probe reductions
 cudaError_t launch_probe_reset(Handle* h, cudaStream_t st);

@@ -787,26 +787,27 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tile width and number of contraction slices from a small cost model, calibrated on B200 with
+// Tile shape and number of contraction slices from a small cost model, calibrated on B200 with
 // in-kernel timestamps: a k-block costs about 0.5 / 0.45 / 0.43 us for 256 / 128 / 64 wide tiles
 // (the shared-memory fill rate of one SM bounds it, so narrow tiles only pay off when they fill
 // more SMs); a unit costs about 4 us of set-up, pipeline fill and output store; a sliced unit
-// about 7 us more (partial store, wait for its siblings, reduction).
-struct Plan { int bn, split, mh; };   // mh: 1 = 128-row tiles, 2 = 256-row tiles, 3 = 256-row whole waves + 128-row remainder
-// row_tiles128: number of 128-row tile rows (for dX: kept data x 128-token chunks).  A 256-row tile
-// (mh = 2) covers two of them; its k-block costs about 0.62 us for twice the work.
+// about 7 us more (partial store, wait for its siblings, reduction); a 256 x 256 tile (mh = 2) costs
+// about 0.62 us per k-block for twice the work, and 7 us per tile.
+struct Cand {
+  Plan plan;
+  long units;      // (tile, slice) units
+  double unit;     // time of one unit, us
+  double alone;    // time of the product when it has the GPU to itself, us
+};
+constexpr int MAX_CANDS = 64;
+
+// row_tiles128: number of 128-row tile rows (for dX: kept data x 128-token chunks); a 256-row tile covers two.
 // remainder_ok: 256-row tiles may leave a last partial wave to a second launch with 128-row tiles (mh = 3).
-// concurrent: the other product of the call runs at the same time on another stream; the two then share the
-// SMs, and what counts is the SM time the units take in total (taken as twice this product's), not only
-// how soon this product alone would finish: measured on the benchmark layer, slicing a contraction that runs
-// beside the other product makes the pair slower (dense call 58.9 us with the dW contraction in two slices,
-// 51.6 us unsliced).
-Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks, int num_sms, int max_units,
-                int force_bn, int force_split, bool remainder_ok, bool concurrent) {
+int enumerate_plans(long row_tiles128, long row_tiles256, int n_extent, int kblocks, int num_sms, int max_units,
+                    int force_bn, int force_split, bool remainder_ok, Cand* out) {
   const int widths[3] = {256, 128, 64};
   const double c_kb[3] = {0.50, 0.45, 0.43};
-  Plan best = {256, 1, 1};
-  double best_t = 1e30;
+  int n = 0;
   if (kblocks < 1) kblocks = 1;
   for (int i = 0; i < 3; ++i) {
     if (force_bn != 0 && widths[i] != force_bn) continue;
@@ -819,18 +820,13 @@ Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks,
       if (sp > 1 && force_split == 0 && kblocks / sp < 4) continue;   // slices too short to pay off
       const long units = tiles * sp;
       const double waves = (double)((units + num_sms - 1) / num_sms);
-      const double unit_fixed = sp > 1 ? 11.0 + 0.25 * sp : 4.0;
-      const double unit = (double)((kblocks + sp - 1) / sp) * c_kb[i] + unit_fixed;
-      double t = waves * unit;
-      if (concurrent && t < 2.0 * (double)units * unit / num_sms) t = 2.0 * (double)units * unit / num_sms;
-      if (t < best_t - 1e-9) { best_t = t; best = {widths[i], sp, 1}; }
+      const double unit = (double)((kblocks + sp - 1) / sp) * c_kb[i] + (sp > 1 ? 11.0 + 0.25 * sp : 4.0);
+      if (n < MAX_CANDS) out[n++] = {{widths[i], sp, 1}, units, unit, waves * unit};
     }
     if (widths[i] == 256 && force_split <= 1) {                        // 256 x 256 tiles, never sliced
       const long units = row_tiles256 * ntiles;
       const double wave = (double)kblocks * 0.62 + 7.0;
-      double t = (double)((units + num_sms - 1) / num_sms) * wave;
-      if (concurrent && t < 2.0 * (double)units * wave / num_sms) t = 2.0 * (double)units * wave / num_sms;
-      if (t < best_t - 1e-9) { best_t = t; best = {256, 1, 2}; }
+      if (n < MAX_CANDS) out[n++] = {{256, 1, 2}, units, wave, (double)((units + num_sms - 1) / num_sms) * wave};
       const long frac = units % num_sms;
       if (remainder_ok && frac > 0 && 2 * frac <= num_sms) {            // whole waves, then the rest as sliced 128-row tiles
         long sp = num_sms / (2 * frac);
@@ -838,13 +834,52 @@ Plan plan_tiles(long row_tiles128, long row_tiles256, int n_extent, int kblocks,
         if (sp > kblocks / 4) sp = kblocks / 4;
         if (sp < 1) sp = 1;
         const double tail = (double)((kblocks + sp - 1) / sp) * 0.50 + (sp > 1 ? 11.0 + 0.25 * sp : 4.0) + 4.0;
-        double t2 = (double)(units / num_sms) * wave + tail;
-        if (concurrent) t2 *= 2.0;        // (many units: the SM time is what the waves add up to)
-        if (t2 < best_t - 1e-9) { best_t = t2; best = {256, 1, 3}; }
+        if (n < MAX_CANDS) out[n++] = {{256, 1, 3}, units, wave, (double)(units / num_sms) * wave + tail};
       }
     }
   }
-  return best;
+  if (n == 0) out[n++] = {{256, 1, 1}, 1, 1.0, 1.0};
+  return n;
+}
+
+// the tile-height override of vcas_set_tuning, applied to a chosen plan
+Plan apply_tile_m(const Handle* h, Plan plan, bool remainder_ok) {
+  if (h->tune_tile_m == 1) plan.mh = 1;
+  if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
+  if (h->tune_tile_m == 3 && plan.bn == 256 && remainder_ok) { plan.mh = 3; plan.split = 1; }
+  return plan;
+}
+
+Plan best_alone(const Cand* c, int n) {
+  int b = 0;
+  for (int i = 1; i < n; ++i)
+    if (c[i].alone < c[b].alone - 1e-9) b = i;
+  return c[b].plan;
+}
+
+// The two products of one call run at the same time on two streams.  Model: the first product's CTAs are
+// resident from time 0, the second's become ready `offset` us later and take the SMs that are free then, or,
+// if those are too few, wait for the first product's CTAs to leave.  (Measured on the benchmark layer: a
+// dense call takes 63 us when the two grids together exceed the SMs, 52 us when the dW product runs as 36
+// tiles of 256 x 256 beside the 96 CTAs of the dX product.)
+void best_pair(const Cand* c1, int n1, int ctas1, const Cand* c2, int n2, int ctas2, int num_sms, double offset,
+               Plan* p1, Plan* p2) {
+  double best = 1e30;
+  *p1 = c1[0].plan; *p2 = c2[0].plan;
+  for (int i = 0; i < n1; ++i) {
+    const bool split1 = c1[i].plan.mh == 3;
+    const long g1 = split1 || c1[i].units > ctas1 ? ctas1 : c1[i].units;
+    const double d1 = split1 ? c1[i].alone : (double)((c1[i].units + g1 - 1) / g1) * c1[i].unit;
+    for (int j = 0; j < n2; ++j) {
+      const bool split2 = c2[j].plan.mh == 3;
+      const long g2 = split2 || c2[j].units > ctas2 ? ctas2 : c2[j].units;
+      const double d2 = split2 ? c2[j].alone : (double)((c2[j].units + g2 - 1) / g2) * c2[j].unit;
+      const double start2 = g2 <= num_sms - g1 ? offset : (offset > d1 ? offset : d1);
+      const double end = d1 > start2 + d2 ? d1 : start2 + d2;
+      const double t = end + 1e-3 * ((double)g1 * d1 + (double)g2 * d2) / num_sms;    // ties: less SM time
+      if (t < best - 1e-9) { best = t; *p1 = c1[i].plan; *p2 = c2[j].plan; }
+    }
+  }
 }
 
 template <int MODE, int BN, int MH, bool LEAN>
@@ -924,8 +959,59 @@ void common_params(Handle* h, GemmParams& P, int which) {
 
 }  // namespace
 
+namespace {
+struct DxShape { long row_tiles128, row_tiles256; int kblocks; bool rem_ok; };
+DxShape dx_shape(const Handle* h, bool dense, float rho_hint) {
+  const vcas_layer_desc& d = h->desc;
+  double kept = dense ? (double)d.N : (double)rho_hint * d.N;
+  if (kept < 1.0) kept = 1.0;
+  const long nk = (long)(kept + 0.5);
+  DxShape g;
+  g.row_tiles128 = nk * ((d.T + BM - 1) / BM);
+  g.row_tiles256 = nk * ((d.T + 2 * BM - 1) / (2 * BM));
+  g.kblocks = (d.d_out + BK - 1) / BK;
+  // the halves of a 256-row tile must both hold rows for the remainder launch to take them over
+  g.rem_ok = h->tune_tile_m != 2 && ((d.T % (2 * BM)) == 0 || (d.T % (2 * BM)) > BM);
+  return g;
+}
+bool dw_remainder_ok(const Handle* h) {
+  const int d_out = h->desc.d_out;
+  return h->tune_tile_m != 2 && ((d_out % (2 * BM)) == 0 || (d_out % (2 * BM)) > BM);
+}
+}  // namespace
+
+void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spare_sms, Plan* dx, Plan* dw) {
+  const vcas_layer_desc& d = h->desc;
+  const DxShape g = dx_shape(h, dense, rho_hint);
+  const int kb_w = (cnt_hint + BK - 1) / BK;
+  const int key[PLAN_KEY_INTS] = {dense ? 1 : 0, (int)g.row_tiles128, kb_w, spare_sms, h->tune_dx_tile_n,
+                                  h->tune_dw_tile_n, h->tune_dx_split_k, h->tune_dw_split_k, h->tune_tile_m};
+  bool hit = h->plan_valid;
+  for (int i = 0; i < PLAN_KEY_INTS && hit; ++i) hit = h->plan_key[i] == key[i];
+  if (!hit) {
+    const int ctas = h->num_sms - spare_sms > 1 ? h->num_sms - spare_sms : 1;
+    Cand cx[MAX_CANDS], cw[MAX_CANDS];
+    const int nx = enumerate_plans(g.row_tiles128, g.row_tiles256, d.d_in, g.kblocks, ctas, h->max_units,
+                                   h->tune_dx_tile_n, h->tune_dx_split_k, g.rem_ok, cx);
+    const bool rem_w = dw_remainder_ok(h);
+    const int nw = enumerate_plans((d.d_out + BM - 1) / BM, (d.d_out + 2 * BM - 1) / (2 * BM), d.d_in, kb_w, h->num_sms,
+                                   h->max_units, h->tune_dw_tile_n, h->tune_dw_split_k, rem_w, cw);
+    // a sampled dW product becomes ready about this much later than the dX product (sampling and pack
+    // against the SampleA-only kernel); the dense products start together
+    const double offset = dense ? 0.0 : 14.0;
+    Plan px, pw;
+    best_pair(cx, nx, ctas, cw, nw, h->num_sms, h->num_sms, offset, &px, &pw);
+    h->plan_dx = apply_tile_m(h, px, g.rem_ok);
+    h->plan_dw = apply_tile_m(h, pw, rem_w);
+    for (int i = 0; i < PLAN_KEY_INTS; ++i) h->plan_key[i] = key[i];
+    h->plan_valid = true;
+  }
+  *dx = h->plan_dx;
+  *dw = h->plan_dw;
+}
+
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint, const void* H,
-                           void* dX, int spare_sms, bool second_set, bool concurrent, cudaStream_t st) {
+                           void* dX, int spare_sms, bool second_set, const Plan* pair_plan, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -953,18 +1039,18 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   P.H = (const __nv_bfloat16*)H; P.dX = (__nv_bfloat16*)dX;
   P.N = d.N; P.T = d.T; P.dense = dense ? 1 : 0;
   P.a_tx_bytes = (d.T < BM ? d.T : BM) * BK * 2;
-  double kept = dense ? (double)d.N : (double)rho_hint * d.N;
-  if (kept < 1.0) kept = 1.0;
   const int chunks = (d.T + BM - 1) / BM, chunks2 = (d.T + 2 * BM - 1) / (2 * BM);
-  const long nk = (long)(kept + 0.5);
   const int ctas = h->num_sms - spare_sms > 1 ? h->num_sms - spare_sms : 1;
-  // the halves of a 256-row tile must both hold rows for the remainder launch to take them over
-  const bool rem_ok = h->tune_tile_m != 2 && ((d.T % (2 * BM)) == 0 || (d.T % (2 * BM)) > BM);
-  Plan plan = plan_tiles(nk * chunks, nk * chunks2, d.d_in, (d.d_out + BK - 1) / BK, ctas, h->max_units,
-                         h->tune_dx_tile_n, h->tune_dx_split_k, rem_ok, concurrent);
-  if (h->tune_tile_m == 1) plan.mh = 1;
-  if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
-  if (h->tune_tile_m == 3 && plan.bn == 256 && rem_ok) { plan.mh = 3; plan.split = 1; }
+  Plan plan;
+  if (pair_plan != nullptr) {
+    plan = *pair_plan;
+  } else {
+    DxShape g = dx_shape(h, dense, rho_hint);
+    Cand cands[MAX_CANDS];
+    const int n = enumerate_plans(g.row_tiles128, g.row_tiles256, d.d_in, g.kblocks, ctas, h->max_units,
+                                  h->tune_dx_tile_n, h->tune_dx_split_k, g.rem_ok, cands);
+    plan = apply_tile_m(h, best_alone(cands, n), g.rem_ok);
+  }
   P.split_k = plan.split;
   // upper bound of work items: every datum kept and split, or every datum a zero tile
   const long max_items = (long)d.N * (plan.mh >= 2 ? chunks2 : chunks) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
@@ -983,7 +1069,7 @@ cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t s
 }
 
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity, const int32_t* cnt,
-                           int cnt_hint, bool concurrent, float* dW, cudaStream_t st) {
+                           int cnt_hint, const Plan* pair_plan, float* dW, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -1008,12 +1094,16 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
   common_params(h, P, 1);
   P.cnt = cnt; P.dW = dW;
   const long mtiles = (d.d_out + BM - 1) / BM, mtiles2 = (d.d_out + 2 * BM - 1) / (2 * BM);
-  const bool rem_ok = h->tune_tile_m != 2 && ((d.d_out % (2 * BM)) == 0 || (d.d_out % (2 * BM)) > BM);
-  Plan plan = plan_tiles(mtiles, mtiles2, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
-                         h->tune_dw_tile_n, h->tune_dw_split_k, rem_ok, concurrent);
-  if (h->tune_tile_m == 1) plan.mh = 1;
-  if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
-  if (h->tune_tile_m == 3 && plan.bn == 256 && rem_ok) { plan.mh = 3; plan.split = 1; }
+  Plan plan;
+  if (pair_plan != nullptr) {
+    plan = *pair_plan;
+  } else {
+    const bool rem_ok = dw_remainder_ok(h);
+    Cand cands[MAX_CANDS];
+    const int n = enumerate_plans(mtiles, mtiles2, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
+                                  h->tune_dw_tile_n, h->tune_dw_split_k, rem_ok, cands);
+    plan = apply_tile_m(h, best_alone(cands, n), rem_ok);
+  }
   P.split_k = plan.split;
   const long max_items = (plan.mh >= 2 ? mtiles2 : mtiles) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
   return run_gemm_bn<MODE_DW>(h, plan, tmA, tmB, tmC, P, max_items, h->num_sms, true, st);
