@@ -195,7 +195,7 @@ __device__ __forceinline__ void capped_prop_warp(float (&v)[SLOTS], float budget
   for (int j = 0; j < SLOTS; ++j)
     if (v[j] > 0.f) { S += v[j]; ++nz; }
   S = warp_sum(S);
-  nz = warp_sum(nz);
+  nz = __reduce_add_sync(0xffffffffu, nz);
   if (nz == 0 || budget <= 0.f) {
 #pragma unroll
     for (int j = 0; j < SLOTS; ++j) v[j] = 0.f;
@@ -217,7 +217,7 @@ __device__ __forceinline__ void capped_prop_warp(float (&v)[SLOTS], float budget
         if (c * v[j] >= 1.0f) ++ks; else Su += v[j];
       }
     Su = warp_sum(Su);
-    ks = warp_sum(ks);
+    ks = __reduce_add_sync(0xffffffffu, ks);
     if (ks == k) break;
     k = ks;
     if (Su > 0.f) {

@@ -212,8 +212,6 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_kernel(SamplerParams 
 struct FastShared {
   float part_f[2][32];
   int part_i[2][32];
-  float tot_f[2];
-  int tot_i[2];
   int warp_tot[32];
   float scaleA[1024];
   float pA[1024];
@@ -221,24 +219,19 @@ struct FastShared {
 };
 
 // Block-wide sum of one float and one int in a fixed order (lanes by shuffle tree, then the 32
-// warp totals by a shuffle tree in warp 0).  fp32 on purpose: this is a single-CTA kernel, and
-// double-precision arithmetic concentrated on one SM was measured to dominate its run time; a
-// tree sum of <= 16384 non-negative fp32 terms is accurate to about 1e-6, inside the 1e-5 the
-// probabilities are specified to.
+// warp totals by the same tree, which every warp runs for itself so that one barrier suffices; the
+// buffers alternate with `parity`, and a buffer is rewritten only after a later barrier).  fp32 on
+// purpose: this is a single-CTA kernel, and double-precision arithmetic concentrated on one SM was
+// measured to dominate its run time; a tree sum of <= 16384 non-negative fp32 terms is accurate to
+// about 1e-6, inside the 1e-5 the probabilities are specified to.
 __device__ __forceinline__ void fast_sum(float& s, int& c, FastShared* sh, int parity) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   s = warp_sum(s);
-  c = warp_sum(c);
+  c = __reduce_add_sync(0xffffffffu, c);
   if (lane == 0) { sh->part_f[parity][warp] = s; sh->part_i[parity][warp] = c; }
   __syncthreads();
-  if (warp == 0) {
-    const float ts = warp_sum(sh->part_f[parity][lane]);
-    const int tc = warp_sum(sh->part_i[parity][lane]);
-    if (lane == 0) { sh->tot_f[parity] = ts; sh->tot_i[parity] = tc; }
-  }
-  __syncthreads();
-  s = sh->tot_f[parity];
-  c = sh->tot_i[parity];
+  s = warp_sum(sh->part_f[parity][lane]);
+  c = __reduce_add_sync(0xffffffffu, sh->part_i[parity][lane]);
 }
 
 template <int E, int SLOTS>
@@ -461,13 +454,10 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerPa
     __syncthreads();                       // warp_tot of the previous group has been read by everyone
     if (lane == 31) sh.warp_tot[warp] = incl;
     __syncthreads();
-    int base = total + incl - mine;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const int t = sh.warp_tot[i];
-      if (i < warp) base += t;
-      total += t;
-    }
+    const int wt = sh.warp_tot[lane];
+    const int base0 = total + incl - mine + __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0);
+    total += __reduce_add_sync(0xffffffffu, wt);
+    int base = base0;
 #pragma unroll
     for (int i = 0; i < 4; ++i)
       if (bits & (1u << i)) {
