@@ -8,8 +8,6 @@ namespace vcas {
 namespace {
 
 constexpr int SAMPLER_THREADS = 1024;
-// threads of the register-resident sampling kernel for R rows (16 rows per thread)
-inline int SAMPLER_NT(int R) { return R <= 4096 ? 256 : (R <= 8192 ? 512 : 1024); }
 static_assert(FAST_MAX_N <= SAMPLER_THREADS && FAST_MAX_R == 16 * SAMPLER_THREADS, "fast sampling limits");
 
 struct Scratch {
@@ -226,19 +224,18 @@ struct FastShared {
 // purpose: this is a single-CTA kernel, and double-precision arithmetic concentrated on one SM was
 // measured to dominate its run time; a tree sum of <= 16384 non-negative fp32 terms is accurate to
 // about 1e-6, inside the 1e-5 the probabilities are specified to.
-template <int NT>
 __device__ __forceinline__ void fast_sum(float& s, int& c, FastShared* sh, int parity) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   s = warp_sum(s);
   c = __reduce_add_sync(0xffffffffu, c);
   if (lane == 0) { sh->part_f[parity][warp] = s; sh->part_i[parity][warp] = c; }
   __syncthreads();
-  s = warp_sum(lane < NT / 32 ? sh->part_f[parity][lane] : 0.f);
-  c = __reduce_add_sync(0xffffffffu, lane < NT / 32 ? sh->part_i[parity][lane] : 0);
+  s = warp_sum(sh->part_f[parity][lane]);
+  c = __reduce_add_sync(0xffffffffu, sh->part_i[parity][lane]);
 }
 
-template <int E, int SLOTS, int NT>
-__global__ void __launch_bounds__(NT) sampler_fast_kernel(SamplerParams P) {
+template <int E, int SLOTS>
+__global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerParams P) {
   __shared__ FastShared sh;
   pdl_wait();      // the row norms come from the kernel before this one
   pdl_trigger();   // the product kernel may set itself up meanwhile
@@ -246,7 +243,7 @@ __global__ void __launch_bounds__(NT) sampler_fast_kernel(SamplerParams P) {
   const int N = P.N, T = P.T, R = N * T;
   // Element e of this thread is row (e / 4) * 4096 + tid * 4 + (e % 4): four consecutive rows per
   // thread and group, so that every 16-byte load or store of a warp covers 512 contiguous bytes.
-  auto row_of = [&](int e) { return (e >> 2) * (4 * NT) + tid * 4 + (e & 3); };
+  auto row_of = [&](int e) { return (e >> 2) * (4 * SAMPLER_THREADS) + tid * 4 + (e & 3); };
 
   // this thread's rows: the unscaled leverage score and the SampleW uniform, both made per row by
   // the row-norm kernel
@@ -263,8 +260,8 @@ __global__ void __launch_bounds__(NT) sampler_fast_kernel(SamplerParams P) {
     }
   }
   // The rows' SampleW uniforms: requested now, together with the scores, when the registers allow it
-  // (fewer than 1024 threads); otherwise they are loaded just before the masks are drawn.
-  constexpr bool EARLY_U = NT < 1024;
+  // (E <= 8); with E = 16 they are loaded just before the masks are drawn.
+  constexpr bool EARLY_U = E <= 8;
   uint32_t ue[EARLY_U ? E : 4];
   if (EARLY_U) {
 #pragma unroll
@@ -305,7 +302,7 @@ __global__ void __launch_bounds__(NT) sampler_fast_kernel(SamplerParams P) {
   };
 
   // ---- ||G_n||_F: one warp per datum, fixed order
-  for (int n = warp; n < N; n += NT / 32) {
+  for (int n = warp; n < N; n += 32) {
     const float s = datum_sqnorm_warp(P.a + (size_t)n * T, T, lane);
     if (lane == 0) { const float g = sqrtf(s); P.g[n] = g; sh.pA[n] = g; }
   }
@@ -354,7 +351,7 @@ __global__ void __launch_bounds__(NT) sampler_fast_kernel(SamplerParams P) {
     for (int e = 0; e < E; ++e)
       if (w[e] > 0.f) { S += w[e]; ++nz; }
     int parity = 0;
-    fast_sum<NT>(S, nz, &sh, parity); parity ^= 1;
+    fast_sum(S, nz, &sh, parity); parity ^= 1;
     if (nz == 0 || budget <= 0.f) {
 #pragma unroll
       for (int e = 0; e < E; ++e) q[e] = 0.f;
@@ -372,7 +369,7 @@ __global__ void __launch_bounds__(NT) sampler_fast_kernel(SamplerParams P) {
           if (w[e] > 0.f) {
             if (c * w[e] >= 1.0f) ++ks; else Su += w[e];
           }
-        fast_sum<NT>(Su, ks, &sh, parity); parity ^= 1;
+        fast_sum(Su, ks, &sh, parity); parity ^= 1;
         if (ks == k) break;
         k = ks;
         if (Su > 0.f) {
@@ -409,7 +406,7 @@ __global__ void __launch_bounds__(NT) sampler_fast_kernel(SamplerParams P) {
 #pragma unroll
     for (int e = 0; e < E; ++e)
       if (q[e] > 0.f) vw += (1.0f - q[e]) / q[e] * w[e] * w[e];
-    fast_sum<NT>(vw, dummy, &sh, 0);
+    fast_sum(vw, dummy, &sh, 0);
     if (tid == 0) P.acc[1] += (double)vw;
   }
 
@@ -457,7 +454,7 @@ __global__ void __launch_bounds__(NT) sampler_fast_kernel(SamplerParams P) {
     __syncthreads();                       // warp_tot of the previous group has been read by everyone
     if (lane == 31) sh.warp_tot[warp] = incl;
     __syncthreads();
-    const int wt = lane < NT / 32 ? sh.warp_tot[lane] : 0;
+    const int wt = sh.warp_tot[lane];
     const int base0 = total + incl - mine + __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0);
     total += __reduce_add_sync(0xffffffffu, wt);
     int base = base0;
@@ -530,20 +527,17 @@ cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st, boo
   cudaError_t e = cudaSuccess;
   // after_event: the kernel before this one in the stream is not the producer of its inputs (those
   // arrive through an event from another stream), so it is launched without the programmatic attribute
-  auto go = [&](void (*k)(SamplerParams), int threads) {
-    if (after_event) { k<<<1, threads, 0, st>>>(P); return cudaSuccess; }
-    return launch_after(k, dim3(1), dim3(threads), 0, st, P);
+  auto go = [&](void (*k)(SamplerParams)) {
+    if (after_event) { k<<<1, SAMPLER_THREADS, 0, st>>>(P); return cudaSuccess; }
+    return launch_after(k, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
   };
   if (fast_sampling(h->desc)) {
-    // Sixteen rows per thread wherever the layer allows: with fewer warps the block-wide sums of the
-    // water-filling (shuffles and a barrier per step) cost less than the extra rows per thread.
     const bool wide = P.N > 32;       // SampleA slots per lane of warp 0
-    const int nt = SAMPLER_NT(R);
-    if (nt == 256) e = go(wide ? sampler_fast_kernel<16, 32, 256> : sampler_fast_kernel<16, 1, 256>, 256);
-    else if (nt == 512) e = go(wide ? sampler_fast_kernel<16, 32, 512> : sampler_fast_kernel<16, 1, 512>, 512);
-    else e = go(wide ? sampler_fast_kernel<16, 32, 1024> : sampler_fast_kernel<16, 1, 1024>, 1024);
+    if (R <= 4 * SAMPLER_THREADS) e = go(wide ? sampler_fast_kernel<4, 32> : sampler_fast_kernel<4, 1>);
+    else if (R <= 8 * SAMPLER_THREADS) e = go(wide ? sampler_fast_kernel<8, 32> : sampler_fast_kernel<8, 1>);
+    else e = go(wide ? sampler_fast_kernel<16, 32> : sampler_fast_kernel<16, 1>);
   } else {
-    e = go(sampler_kernel, SAMPLER_THREADS);
+    e = go(sampler_kernel);
   }
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
