@@ -58,8 +58,10 @@ def ncu_traffic(kernel: str):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """Samples nvidia-smi clocks and throttle reasons every 20 ms.  It is started before the warm-up (nvidia-smi
+    takes a while to deliver its first sample); stop(t0, t1) keeps the samples whose time stamps lie inside
+    the timed region [t0, t1] (host wall clock)."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -69,26 +71,35 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
+        import datetime
         if self.proc is None:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             out, _ = self.proc.communicate(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
+        sm, mx, reasons, seen = [], [], set(), 0
         for line in out.strip().splitlines():
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
                 continue
+            seen += 1
+            if t0 is not None and t1 is not None:
+                try:
+                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                except ValueError:
+                    continue
+                if ts < t0 or ts > t1 + 0.02:
+                    continue
             try:
                 sm.append(float(f[1])); mx.append(float(f[2]))
             except ValueError:
@@ -97,7 +108,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(name)
         return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
-                    reasons=sorted(reasons), samples=len(sm))
+                    reasons=sorted(reasons), samples=len(sm), samples_outside_timed_region=seen - len(sm))
 
 
 def oracle_call(case, batch=0, seed=0):
@@ -211,7 +222,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="vcas", choices=["vcas", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -315,14 +326,18 @@ def main():
         barrier()
         return dist_util.max_over_ranks(e0.elapsed_time(e1), dev)
 
-    for _ in range(args.warmup):
-        step()
     clocks = ClockSampler(local)
     if rank == 0:
         clocks.start()
+    for _ in range(args.warmup):
+        step()
+    if rank == 0:
+        time.sleep(0.3)           # nvidia-smi is delivering samples by now
+    wall0 = time.time()
     total_ms = timed(step, args.steps)
+    wall1 = time.time()
     launches = args.steps * (launches_per_period + probe_launches[0])
-    clock_info = clocks.stop() if rank == 0 else None
+    clock_info = clocks.stop(wall0, wall1) if rank == 0 else None
     ms_per_step = total_ms / args.steps
     value = dist_util.ms_per_layer(ms_per_step, F_CALLS, world)      # whole-job: all ranks' calls per unit time
 
