@@ -862,6 +862,7 @@ Plan best_alone(const Cand* c, int n) {
 // if those are too few, wait for the first product's CTAs to leave.  (Measured on the benchmark layer: a
 // dense call takes 63 us when the two grids together exceed the SMs, 52 us when the dW product runs as 36
 // tiles of 256 x 256 beside the 96 CTAs of the dX product.)
+constexpr double KERNEL_US = 3.0;   // launch ramp and exit of a product kernel, on top of its units (timeline measurements)
 void best_pair(const Cand* c1, int n1, int ctas1, const Cand* c2, int n2, int ctas2, int num_sms, double offset,
                Plan* p1, Plan* p2) {
   double best = 1e30;
@@ -869,11 +870,11 @@ void best_pair(const Cand* c1, int n1, int ctas1, const Cand* c2, int n2, int ct
   for (int i = 0; i < n1; ++i) {
     const bool split1 = c1[i].plan.mh == 3;
     const long g1 = split1 || c1[i].units > ctas1 ? ctas1 : c1[i].units;
-    const double d1 = split1 ? c1[i].alone : (double)((c1[i].units + g1 - 1) / g1) * c1[i].unit;
+    const double d1 = (split1 ? c1[i].alone : (double)((c1[i].units + g1 - 1) / g1) * c1[i].unit) + KERNEL_US;
     for (int j = 0; j < n2; ++j) {
       const bool split2 = c2[j].plan.mh == 3;
       const long g2 = split2 || c2[j].units > ctas2 ? ctas2 : c2[j].units;
-      const double d2 = split2 ? c2[j].alone : (double)((c2[j].units + g2 - 1) / g2) * c2[j].unit;
+      const double d2 = (split2 ? c2[j].alone : (double)((c2[j].units + g2 - 1) / g2) * c2[j].unit) + KERNEL_US;
       const double start2 = g2 <= num_sms - g1 ? offset : (offset > d1 ? offset : d1);
       const double end = d1 > start2 + d2 ? d1 : start2 + d2;
       const double t = end + 1e-3 * ((double)g1 * d1 + (double)g2 * d2) / num_sms;    // ties: less SM time
@@ -997,8 +998,9 @@ void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spar
     const int nw = enumerate_plans((d.d_out + BM - 1) / BM, (d.d_out + 2 * BM - 1) / (2 * BM), d.d_in, kb_w, h->num_sms,
                                    h->max_units, h->tune_dw_tile_n, h->tune_dw_split_k, rem_w, cw);
     // a sampled dW product becomes ready about this much later than the dX product (sampling and pack
-    // against the SampleA-only kernel); the dense products start together
-    const double offset = dense ? 0.0 : 14.0;
+    // against the SampleA-only kernel: 20.7 against 10.2 us after the call's start on the benchmark
+    // layer); the dense products start together
+    const double offset = dense ? 0.0 : 10.5;
     Plan px, pw;
     best_pair(cx, nx, ctas, cw, nw, h->num_sms, h->num_sms, offset, &px, &pw);
     h->plan_dx = apply_tile_m(h, px, g.rem_ok);
