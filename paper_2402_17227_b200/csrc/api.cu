@@ -60,11 +60,13 @@ size_t layout(Handle* h, uint8_t* base) {
     w.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
     w.partial_tiles = carve<float>(cur, 3 * (size_t)h->max_units * 128 * 256);
     w.tickets = carve<int32_t>(cur, 6 * (size_t)h->max_units);
+    w.sched = carve<int32_t>(cur, 8);
   } else {
     w.packG = nullptr;
     w.packX = nullptr;
     w.partial_tiles = nullptr;
     w.tickets = nullptr;
+    w.sched = nullptr;
   }
   w.Gs = carve<float>(cur, DW);
   w.Gact = carve<float>(cur, DW);
@@ -90,6 +92,7 @@ size_t layout(Handle* h, uint8_t* base) {
     v.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
     v.partial_tiles = w.partial_tiles + (size_t)h->max_units * 128 * 256;   // dW slot of this set = third slot
     v.tickets = w.tickets + 2 * (size_t)h->max_units;
+    v.sched = w.sched + 2;
   }
   v.Gact = carve<float>(cur, DW);
   return (size_t)(cur - base);
@@ -529,6 +532,11 @@ int vcas_last_device_status(vcas_handle hh, int32_t* status) {
   VCAS_CUDA(cudaDeviceSynchronize());
   VCAS_CUDA(cudaMemcpy(status, h->ws.status, sizeof(int32_t), cudaMemcpyDeviceToHost));
   VCAS_CUDA(cudaMemset(h->ws.status, 0, sizeof(int32_t)));
+  if (*status != VCAS_OK && h->tensor_path) {
+    // a product kernel that gave up may have left its slice tickets and work counters non-zero
+    VCAS_CUDA(cudaMemset(h->ws.tickets, 0, 6 * (size_t)h->max_units * sizeof(int32_t)));
+    VCAS_CUDA(cudaMemset(h->ws.sched, 0, 8 * sizeof(int32_t)));
+  }
   return VCAS_OK;
 }
 

@@ -42,6 +42,7 @@ struct Workspace {
   float* partial_tiles;  // [3][max_units][128 * 256] fp32 partial tiles of a split contraction: dX, dW, and the dW
                          // of the workspace's second set (see Handle::ws2)
   int32_t* tickets;      // [3][2 * max_units]: slices stored, slices finished, per tile
+  int32_t* sched;        // [3][2]: next work item and finished CTAs of an unsliced product (dynamic tile order)
   // probe buffers (App. D: the exact gradient, its running mean and running squared deviation)
   float* Gs;       // [d_out, d_in]
   float* Gact;     // [d_out, d_in]

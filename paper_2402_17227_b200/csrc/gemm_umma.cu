@@ -173,15 +173,19 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn, bool b_mn) {
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
+constexpr int QD = 2;   // depth of the work queue: the producer may be this many items ahead of the other roles
 struct SmemLayout {
   uint8_t* stages;
   uint64_t* full;
   uint64_t* empty;
   uint64_t* tmem_full;
   uint64_t* tmem_empty;
+  uint64_t* q_full;   // work queue (unsliced instance): slot holds a work item
+  uint64_t* q_empty;  // ... slot has been read by the MMA thread and the 128 epilogue threads
   uint32_t* tmem_holder;
   int* abort_flag;
   int* flag;          // epilogue broadcast slot
+  int* tile_q;        // [QD] work items handed from the producer thread to the other roles
   uint8_t* epi;       // [4 warps][2][32 rows][128 B] staging for bulk / TMA stores
 };
 
@@ -197,9 +201,12 @@ __device__ __forceinline__ SmemLayout carve(uint8_t* raw) {
   s.empty = bars + C::STAGES;
   s.tmem_full = bars + 2 * C::STAGES;
   s.tmem_empty = bars + 2 * C::STAGES + 2;
-  s.tmem_holder = (uint32_t*)(bars + 2 * C::STAGES + 4);
+  s.q_full = bars + 2 * C::STAGES + 4;
+  s.q_empty = bars + 2 * C::STAGES + 4 + QD;
+  s.tmem_holder = (uint32_t*)(bars + 2 * C::STAGES + 4 + 2 * QD);
   s.abort_flag = (int*)(s.tmem_holder + 1);
   s.flag = s.abort_flag + 1;
+  s.tile_q = s.flag + 1;
   return s;
 }
 
@@ -209,6 +216,7 @@ __device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid
   if (tid == 0) {
     for (int i = 0; i < C::STAGES; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&s.tmem_full[i], 1); mbar_init(&s.tmem_empty[i], 128); }
+    for (int i = 0; i < QD; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 129); }
     *s.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -245,6 +253,7 @@ struct GemmParams {
   int32_t* status;
   float* partial;          // [max_units][128 * BN] fp32 partial tiles (split contraction)
   int32_t* tickets;        // [2 * max_units]: slices stored / slices finished per tile; zero between launches
+  int32_t* sched;          // [2]: next work item, CTAs that have finished (unsliced instance); zero between launches
   int split_k;             // slices requested by the host
   int max_units;
   // Whole waves and remainder (256-wide tiles): part 1 is the launch with 256-row tiles, which takes only as
@@ -379,7 +388,28 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi) {
+      int qi = 0; uint32_t qph = 0;
+      // Next unit of this CTA, or -1.  Sliced instance: units blockIdx.x, + upi, ... (the slices of a tile
+      // run side by side).  Unsliced instance: the next item of a device-wide counter (product tiles first,
+      // then zero tiles), so that CTAs which start late - the SMs are shared with the call's other
+      // product - or get cheap items simply take fewer; the item is handed to the MMA and epilogue
+      // roles through a small queue in shared memory.
+      auto next_unit = [&](int prev) -> int {
+        if constexpr (LEAN) {
+          if (!mbar_wait(&s.q_empty[qi], qph ^ 1u, abort_flag, P.status)) { ok = false; return -1; }
+          int t = atomicAdd(P.sched, 1);
+          if (t >= D.units + D.zero_tiles) t = -1;
+          *(volatile int*)&s.tile_q[qi] = t;
+          mbar_arrive(&s.q_full[qi]);
+          if (++qi == QD) { qi = 0; qph ^= 1u; }
+          return t;
+        } else {
+          const int u = prev < 0 ? (int)blockIdx.x : prev + D.upi;
+          return ((int)blockIdx.x < D.upi && u < D.units) ? u : -1;
+        }
+      };
+      for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
+        if (u >= D.units) continue;            // a zero tile: nothing to load
         const int tile = u / D.S, slice = u % D.S;
         const int kb0 = slice * D.kb_per;
         const int kb1 = min(D.kblocks, kb0 + D.kb_per);
@@ -410,6 +440,12 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
+      if constexpr (LEAN) {
+        if (ok) {        // the last CTA to run out of work re-arms the counters for the next launch
+          __threadfence();
+          if (atomicAdd(P.sched + 1, 1) == (int)gridDim.x - 1) { P.sched[0] = 0; P.sched[1] = 0; }
+        }
+      }
     }
   } else if (warp == 5) {
     // ------------------------------------------------------------------ MMA issuer
@@ -418,10 +454,25 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       constexpr uint32_t a_step = MODE == MODE_DW ? (UMMA_K * 128 >> 4) : (UMMA_K * 2 >> 4);
       int stage = 0; uint32_t phase = 0; int lt = 0;
       bool ok = true;
-      for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi, ++lt) {
+      int qi = 0; uint32_t qph = 0;
+      auto next_unit = [&](int prev) -> int {
+        if constexpr (LEAN) {
+          if (!mbar_wait(&s.q_full[qi], qph, abort_flag, P.status)) { ok = false; return -1; }
+          const int t = *(volatile int*)&s.tile_q[qi];
+          mbar_arrive(&s.q_empty[qi]);
+          if (++qi == QD) { qi = 0; qph ^= 1u; }
+          return t;
+        } else {
+          const int u = prev < 0 ? (int)blockIdx.x : prev + D.upi;
+          return ((int)blockIdx.x < D.upi && u < D.units) ? u : -1;
+        }
+      };
+      for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
+        if (u >= D.units) continue;            // a zero tile: the epilogue warps write it
+        const int lt_now = lt++;
         const int slice = u % D.S;
         const int nkb = min(D.kblocks, (slice + 1) * D.kb_per) - slice * D.kb_per;
-        const int buf = lt % NACC; const uint32_t use = (uint32_t)(lt / NACC) & 1u;
+        const int buf = lt_now % NACC; const uint32_t use = (uint32_t)(lt_now / NACC) & 1u;
         ok = mbar_wait(&s.tmem_empty[buf], use ^ 1u, abort_flag, P.status);
         if (!ok) break;
         tc_fence_after();
@@ -508,11 +559,46 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t swz = (uint32_t)(lane & 7);                   // 128-byte swizzle: 16-byte slot ^= row & 7
     int lt = 0;
     bool ok = true;
-    for (int u = blockIdx.x; (int)blockIdx.x < D.upi && u < D.units && ok; u += D.upi, ++lt) {
+    int qi = 0; uint32_t qph = 0;
+    auto next_unit = [&](int prev) -> int {
+      if constexpr (LEAN) {
+        if (!mbar_wait(&s.q_full[qi], qph, abort_flag, P.status)) { ok = false; return -1; }
+        const int t = *(volatile int*)&s.tile_q[qi];
+        mbar_arrive(&s.q_empty[qi]);
+        if (++qi == QD) { qi = 0; qph ^= 1u; }
+        return t;
+      } else {
+        const int u = prev < 0 ? (int)blockIdx.x : prev + D.upi;
+        return ((int)blockIdx.x < D.upi && u < D.units) ? u : -1;
+      }
+    };
+    // writes the zero tile z (rows of dropped data; nothing kept at all)
+    auto zero_tile = [&](int z) {
+      size_t row0; int rows_valid, col0, n_out, t_out; float sc;
+      geometry(z, false, row0, rows_valid, col0, sc, n_out, t_out);
+#pragma unroll 1
+      for (int hh = 0; hh < MH; ++hh) {
+        const int hrow = hh * BM + row;
+        if (hrow >= rows_valid) continue;
+        const size_t off = (row0 + hrow) * ld + col0;
+        if (MODE == MODE_DX) {
+#pragma unroll
+          for (int j = 0; j < BN / 8; ++j)
+            if (col0 + j * 8 < P.d_in) *reinterpret_cast<uint4*>(P.dX + off + j * 8) = make_uint4(0u, 0u, 0u, 0u);
+        } else {
+#pragma unroll
+          for (int j = 0; j < BN / 4; ++j)
+            if (col0 + j * 4 < P.d_in) *reinterpret_cast<uint4*>(P.dW + off + j * 4) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+    };
+    for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
+      if (u >= D.units) { zero_tile(u - D.units); continue; }
+      const int lt_now = lt++;
       const int tile = u / D.S, slice = u % D.S;
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(tile, true, row0, rows_valid, col0, sc, n_out, t_out);
-      const int buf = lt % NACC; const uint32_t use = (uint32_t)(lt / NACC) & 1u;
+      const int buf = lt_now % NACC; const uint32_t use = (uint32_t)(lt_now / NACC) & 1u;
       if (!mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * BN);
@@ -690,26 +776,9 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       }  // !LEAN
     }
-    // zero tiles (rows of dropped data; nothing kept at all): taken from the far end of the grid first,
-    // where CTAs have no product units
-    for (int z = (int)gridDim.x - 1 - (int)blockIdx.x; z < D.zero_tiles && ok; z += gridDim.x) {
-      size_t row0; int rows_valid, col0, n_out, t_out; float sc;
-      geometry(z, false, row0, rows_valid, col0, sc, n_out, t_out);
-#pragma unroll 1
-      for (int hh = 0; hh < MH; ++hh) {
-        const int hrow = hh * BM + row;
-        if (hrow >= rows_valid) continue;
-        const size_t off = (row0 + hrow) * ld + col0;
-        if (MODE == MODE_DX) {
-#pragma unroll
-          for (int j = 0; j < BN / 8; ++j)
-            if (col0 + j * 8 < P.d_in) *reinterpret_cast<uint4*>(P.dX + off + j * 8) = make_uint4(0u, 0u, 0u, 0u);
-        } else {
-#pragma unroll
-          for (int j = 0; j < BN / 4; ++j)
-            if (col0 + j * 4 < P.d_in) *reinterpret_cast<uint4*>(P.dW + off + j * 4) = make_uint4(0u, 0u, 0u, 0u);
-        }
-      }
+    // sliced instance: zero tiles are taken from the far end of the grid first, where CTAs have no product units
+    if constexpr (!LEAN) {
+      for (int z = (int)gridDim.x - 1 - (int)blockIdx.x; z < D.zero_tiles && ok; z += gridDim.x) zero_tile(z);
     }
   }
   __syncwarp();
@@ -953,6 +1022,7 @@ void common_params(Handle* h, GemmParams& P, int which) {
   P.status = h->ws.status;
   P.partial = h->ws.partial_tiles + (size_t)which * h->max_units * (BM * 256);
   P.tickets = h->ws.tickets + (size_t)which * 2 * h->max_units;
+  P.sched = h->ws.sched + which * 2;
   P.max_units = h->max_units;
   P.d_in = h->desc.d_in;
   P.d_out = h->desc.d_out;
