@@ -1,14 +1,16 @@
 // The two products of the sampled backward on the 5th-generation tensor cores (tcgen05):
 //   dX[rows of kept data] = (1/p_n) dY[rows] W          (App. E; rows of dropped data are zero-filled)
 //   dW = A_rows^T B_rows over the compacted kept rows    (Sec. 4.2: G_tilde^T X)
-// One persistent CTA per SM walks a tile list whose length depends on the kept counts, which
+// One persistent CTA per SM works through tiles whose number depends on the kept counts, which
 // are read from device memory.  Per CTA: warps 0-3 are the epilogue (TMEM -> registers ->
-// global), warp 4 issues TMA loads into a ring of shared-memory stages, warp 5 issues
-// tcgen05.mma into one of two TMEM accumulators, so the epilogue of a tile overlaps the main
-// loop of the next one.  bf16 operands, fp32 accumulation.  Outputs leave through 128-byte-swizzled
-// shared-memory staging and TMA / bulk stores.  A contraction can be cut into slices worked on by
-// neighbouring CTAs; the slices are added in a fixed order.  Every wait (mbarrier or sibling
-// CTA) is bounded: when it runs out the CTA records VCAS_ERR_TIMEOUT in the status word and leaves.
+// shared memory -> global), warp 4 issues TMA loads into a ring of shared-memory stages, warp 5
+// issues tcgen05.mma into TMEM accumulators (two of 128 rows, so that the epilogue of a tile overlaps
+// the main loop of the next one, or one of 256 rows).  bf16 operands, fp32 accumulation.  Outputs leave
+// through 128-byte-swizzled shared-memory staging and TMA / bulk stores.  Two instances per tile
+// shape: the unsliced one draws its tiles from a device-wide counter; the sliced one cuts each
+// contraction into slices worked on by neighbouring CTAs and adds the slices in a fixed order.
+// Every wait (mbarrier or sibling CTA) is bounded: when it runs out the CTA records
+// VCAS_ERR_TIMEOUT in the status word and leaves.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -382,6 +384,10 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile int* abort_flag = s.abort_flag;
   pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
   const Decomp D = decompose<MODE, BN, MH, LEAN>(P);
+  // unsliced instance: with at most one work item per CTA the item is the CTA's index; with more, the items
+  // are drawn from the device-wide counter
+  const int total_items = D.units + D.zero_tiles;
+  const bool dynamic = LEAN && total_items > (int)gridDim.x;
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
@@ -391,11 +397,12 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int qi = 0; uint32_t qph = 0;
       // Next unit of this CTA, or -1.  Sliced instance: units blockIdx.x, + upi, ... (the slices of a tile
       // run side by side).  Unsliced instance: the next item of a device-wide counter (product tiles first,
-      // then zero tiles), so that CTAs which start late - the SMs are shared with the call's other
-      // product - or get cheap items simply take fewer; the item is handed to the MMA and epilogue
-      // roles through a small queue in shared memory.
+      // then zero tiles) when there are more items than CTAs, so that CTAs which start late - the SMs are
+      // shared with the call's other product - or get cheap items simply take fewer; the item is handed
+      // to the MMA and epilogue roles through a small queue in shared memory.
       auto next_unit = [&](int prev) -> int {
         if constexpr (LEAN) {
+          if (!dynamic) return (prev < 0 && (int)blockIdx.x < total_items) ? (int)blockIdx.x : -1;
           if (!mbar_wait(&s.q_empty[qi], qph ^ 1u, abort_flag, P.status)) { ok = false; return -1; }
           int t = atomicAdd(P.sched, 1);
           if (t >= D.units + D.zero_tiles) t = -1;
@@ -441,7 +448,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       }
       if constexpr (LEAN) {
-        if (ok) {        // the last CTA to run out of work re-arms the counters for the next launch
+        if (ok && dynamic) {   // the last CTA to run out of work re-arms the counters for the next launch
           __threadfence();
           if (atomicAdd(P.sched + 1, 1) == (int)gridDim.x - 1) { P.sched[0] = 0; P.sched[1] = 0; }
         }
@@ -457,6 +464,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int qi = 0; uint32_t qph = 0;
       auto next_unit = [&](int prev) -> int {
         if constexpr (LEAN) {
+          if (!dynamic) return (prev < 0 && (int)blockIdx.x < total_items) ? (int)blockIdx.x : -1;
           if (!mbar_wait(&s.q_full[qi], qph, abort_flag, P.status)) { ok = false; return -1; }
           const int t = *(volatile int*)&s.tile_q[qi];
           mbar_arrive(&s.q_empty[qi]);
@@ -562,6 +570,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     int qi = 0; uint32_t qph = 0;
     auto next_unit = [&](int prev) -> int {
       if constexpr (LEAN) {
+        if (!dynamic) return (prev < 0 && (int)blockIdx.x < total_items) ? (int)blockIdx.x : -1;
         if (!mbar_wait(&s.q_full[qi], qph, abort_flag, P.status)) { ok = false; return -1; }
         const int t = *(volatile int*)&s.tile_q[qi];
         mbar_arrive(&s.q_empty[qi]);
