@@ -250,6 +250,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // share of the tile's rows in slice order (a fixed order: results do not depend on timing) and
 // writes that share of the output.
 constexpr int MODE_DX = 0, MODE_DW = 1;
+constexpr int KIND_SLICED = 0, KIND_STATIC = 1, KIND_DYNAMIC = 2;
 
 struct GemmParams {
   int32_t* status;
@@ -367,10 +368,15 @@ __device__ __forceinline__ void tile_coords(const GemmParams& P, const Decomp& D
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// LEAN: the instance for unsliced contractions (S = 1), without the code of the slice exchange; the other
-// instance has only the slice exchange (a contraction that ends up in one slice still goes through it).
-// Two instances because the product kernels are short: code that a launch never runs still costs it time.
-template <int MODE, int BN, int MH, bool LEAN>
+// KIND: three instances per tile shape.  KIND_STATIC and KIND_DYNAMIC are for unsliced contractions (S = 1)
+// and carry no code of the slice exchange; the static one takes work items blockIdx.x, + gridDim.x, ...,
+// the dynamic one draws them from a device-wide counter (chosen when there are more items than CTAs) and
+// hands them to the MMA and epilogue roles through a small queue in shared memory, so that CTAs which start
+// late - the SMs are shared with the call's other product - or get cheap items simply take fewer.
+// KIND_SLICED has only the slice exchange (a contraction that ends up in one slice still goes through it).
+// Separate instances because the product kernels are short: code that a launch never runs still costs it
+// time.
+template <int MODE, int BN, int MH, int KIND>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, GemmParams P) {
@@ -383,11 +389,10 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const uint32_t tmem_base = setup<BN, MH>(s, warp, tid);
   volatile int* abort_flag = s.abort_flag;
   pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
+  constexpr bool LEAN = KIND != KIND_SLICED;
+  constexpr bool DYN = KIND == KIND_DYNAMIC;
   const Decomp D = decompose<MODE, BN, MH, LEAN>(P);
-  // unsliced instance: with at most one work item per CTA the item is the CTA's index; with more, the items
-  // are drawn from the device-wide counter
-  const int total_items = D.units + D.zero_tiles;
-  const bool dynamic = LEAN && total_items > (int)gridDim.x;
+  const int total_items = D.units + D.zero_tiles;     // unsliced instances: product tiles, then zero tiles
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
@@ -395,14 +400,9 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       int qi = 0; uint32_t qph = 0;
-      // Next unit of this CTA, or -1.  Sliced instance: units blockIdx.x, + upi, ... (the slices of a tile
-      // run side by side).  Unsliced instance: the next item of a device-wide counter (product tiles first,
-      // then zero tiles) when there are more items than CTAs, so that CTAs which start late - the SMs are
-      // shared with the call's other product - or get cheap items simply take fewer; the item is handed
-      // to the MMA and epilogue roles through a small queue in shared memory.
+      // next unit of this CTA, or -1 (see KIND above)
       auto next_unit = [&](int prev) -> int {
-        if constexpr (LEAN) {
-          if (!dynamic) return (prev < 0 && (int)blockIdx.x < total_items) ? (int)blockIdx.x : -1;
+        if constexpr (DYN) {
           if (!mbar_wait(&s.q_empty[qi], qph ^ 1u, abort_flag, P.status)) { ok = false; return -1; }
           int t = atomicAdd(P.sched, 1);
           if (t >= D.units + D.zero_tiles) t = -1;
@@ -410,6 +410,9 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           mbar_arrive(&s.q_full[qi]);
           if (++qi == QD) { qi = 0; qph ^= 1u; }
           return t;
+        } else if constexpr (LEAN) {
+          const int u = prev < 0 ? (int)blockIdx.x : prev + (int)gridDim.x;
+          return u < total_items ? u : -1;
         } else {
           const int u = prev < 0 ? (int)blockIdx.x : prev + D.upi;
           return ((int)blockIdx.x < D.upi && u < D.units) ? u : -1;
@@ -447,8 +450,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if constexpr (LEAN) {
-        if (ok && dynamic) {   // the last CTA to run out of work re-arms the counters for the next launch
+      if constexpr (DYN) {
+        if (ok) {        // the last CTA to run out of work re-arms the counters for the next launch
           __threadfence();
           if (atomicAdd(P.sched + 1, 1) == (int)gridDim.x - 1) { P.sched[0] = 0; P.sched[1] = 0; }
         }
@@ -463,13 +466,15 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       bool ok = true;
       int qi = 0; uint32_t qph = 0;
       auto next_unit = [&](int prev) -> int {
-        if constexpr (LEAN) {
-          if (!dynamic) return (prev < 0 && (int)blockIdx.x < total_items) ? (int)blockIdx.x : -1;
+        if constexpr (DYN) {
           if (!mbar_wait(&s.q_full[qi], qph, abort_flag, P.status)) { ok = false; return -1; }
           const int t = *(volatile int*)&s.tile_q[qi];
           mbar_arrive(&s.q_empty[qi]);
           if (++qi == QD) { qi = 0; qph ^= 1u; }
           return t;
+        } else if constexpr (LEAN) {
+          const int u = prev < 0 ? (int)blockIdx.x : prev + (int)gridDim.x;
+          return u < total_items ? u : -1;
         } else {
           const int u = prev < 0 ? (int)blockIdx.x : prev + D.upi;
           return ((int)blockIdx.x < D.upi && u < D.units) ? u : -1;
@@ -569,13 +574,15 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     bool ok = true;
     int qi = 0; uint32_t qph = 0;
     auto next_unit = [&](int prev) -> int {
-      if constexpr (LEAN) {
-        if (!dynamic) return (prev < 0 && (int)blockIdx.x < total_items) ? (int)blockIdx.x : -1;
+      if constexpr (DYN) {
         if (!mbar_wait(&s.q_full[qi], qph, abort_flag, P.status)) { ok = false; return -1; }
         const int t = *(volatile int*)&s.tile_q[qi];
         mbar_arrive(&s.q_empty[qi]);
         if (++qi == QD) { qi = 0; qph ^= 1u; }
         return t;
+      } else if constexpr (LEAN) {
+        const int u = prev < 0 ? (int)blockIdx.x : prev + (int)gridDim.x;
+        return u < total_items ? u : -1;
       } else {
         const int u = prev < 0 ? (int)blockIdx.x : prev + D.upi;
         return ((int)blockIdx.x < D.upi && u < D.units) ? u : -1;
@@ -961,12 +968,12 @@ void best_pair(const Cand* c1, int n1, int ctas1, const Cand* c2, int n2, int ct
   }
 }
 
-template <int MODE, int BN, int MH, bool LEAN>
+template <int MODE, int BN, int MH, int KIND>
 cudaError_t run_gemm_k(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P0,
                      long max_items, int ctas, bool pdl, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN, MH, LEAN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN, MH, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          TileCfg<BN, MH>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
@@ -986,7 +993,7 @@ cudaError_t run_gemm_k(Handle* h, const CUtensorMap& a, const CUtensorMap& b, co
     cfg.numAttrs += 1;
   }
   cfg.gridDim = dim3((unsigned)grid);
-  cudaError_t e = cudaLaunchKernelEx(&cfg, umma_kernel<MODE, BN, MH, LEAN>, a, b, c, P);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, umma_kernel<MODE, BN, MH, KIND>, a, b, c, P);
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -994,11 +1001,14 @@ cudaError_t run_gemm_k(Handle* h, const CUtensorMap& a, const CUtensorMap& b, co
 template <int MODE, int BN, int MH>
 cudaError_t run_gemm(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P,
                      long max_items, int ctas, bool pdl, cudaStream_t st) {
+  const bool many = max_items > ctas;      // more work items than CTAs: dynamic order
   if constexpr (MH == 2) {
-    return run_gemm_k<MODE, BN, MH, true>(h, a, b, c, P, max_items, ctas, pdl, st);
+    if (many) return run_gemm_k<MODE, BN, MH, KIND_DYNAMIC>(h, a, b, c, P, max_items, ctas, pdl, st);
+    return run_gemm_k<MODE, BN, MH, KIND_STATIC>(h, a, b, c, P, max_items, ctas, pdl, st);
   } else {
-    if (P.split_k == 1) return run_gemm_k<MODE, BN, MH, true>(h, a, b, c, P, max_items, ctas, pdl, st);
-    return run_gemm_k<MODE, BN, MH, false>(h, a, b, c, P, max_items, ctas, pdl, st);
+    if (P.split_k != 1) return run_gemm_k<MODE, BN, MH, KIND_SLICED>(h, a, b, c, P, max_items, ctas, pdl, st);
+    if (many) return run_gemm_k<MODE, BN, MH, KIND_DYNAMIC>(h, a, b, c, P, max_items, ctas, pdl, st);
+    return run_gemm_k<MODE, BN, MH, KIND_STATIC>(h, a, b, c, P, max_items, ctas, pdl, st);
   }
 }
 
