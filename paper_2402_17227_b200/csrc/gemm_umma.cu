@@ -213,12 +213,13 @@ __device__ __forceinline__ SmemLayout carve(uint8_t* raw) {
 }
 
 template <int BN, int MH>
-__device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid) {
+__device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid, bool with_queue) {
   using C = TileCfg<BN, MH>;
   if (tid == 0) {
     for (int i = 0; i < C::STAGES; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&s.tmem_full[i], 1); mbar_init(&s.tmem_empty[i], 128); }
-    for (int i = 0; i < QD; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 129); }
+    if (with_queue)
+      for (int i = 0; i < QD; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 129); }
     *s.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -386,7 +387,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   extern __shared__ uint8_t smem_raw[];
   const SmemLayout s = carve<BN, MH>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t tmem_base = setup<BN, MH>(s, warp, tid);
+  const uint32_t tmem_base = setup<BN, MH>(s, warp, tid, KIND == KIND_DYNAMIC);
   volatile int* abort_flag = s.abort_flag;
   pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
   constexpr bool LEAN = KIND != KIND_SLICED;
@@ -419,7 +420,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       };
       for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
-        if (u >= D.units) continue;            // a zero tile: nothing to load
+        if (LEAN && u >= D.units) continue;    // a zero tile: nothing to load
         const int tile = u / D.S, slice = u % D.S;
         const int kb0 = slice * D.kb_per;
         const int kb1 = min(D.kblocks, kb0 + D.kb_per);
@@ -481,7 +482,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       };
       for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
-        if (u >= D.units) continue;            // a zero tile: the epilogue warps write it
+        if (LEAN && u >= D.units) continue;    // a zero tile: the epilogue warps write it
         const int lt_now = lt++;
         const int slice = u % D.S;
         const int nkb = min(D.kblocks, (slice + 1) * D.kb_per) - slice * D.kb_per;
@@ -609,7 +610,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     };
     for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
-      if (u >= D.units) { zero_tile(u - D.units); continue; }
+      if (LEAN && u >= D.units) { zero_tile(u - D.units); continue; }
       const int lt_now = lt++;
       const int tile = u / D.S, slice = u % D.S;
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
