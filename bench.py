@@ -66,15 +66,29 @@ class ClockSampler:
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
-        self.index, self.proc = index, None
+        self.index, self.proc, self.lines, self.thread = index, None, [], None
 
     def start(self):
+        import threading
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
                                           "--format=csv,noheader,nounits", "-lms", "20"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True, bufsize=1)
         except OSError:
             self.proc = None
+            return
+
+        def pump():
+            for line in self.proc.stdout:
+                self.lines.append(line)
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def wait_ready(self, timeout=8.0):
+        """Blocks until nvidia-smi has delivered its first sample (it can take seconds on a busy host)."""
+        t_end = time.time() + timeout
+        while self.proc is not None and not self.lines and time.time() < t_end:
+            time.sleep(0.02)
 
     def stop(self, t0=None, t1=None):
         import datetime
@@ -83,10 +97,12 @@ class ClockSampler:
         time.sleep(0.05)
         self.proc.terminate()
         try:
-            out, _ = self.proc.communicate(timeout=5)
+            self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-            out, _ = self.proc.communicate()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        out = "".join(self.lines)
         sm, mx, reasons, seen = [], [], set(), 0
         for line in out.strip().splitlines():
             f = [x.strip() for x in line.split(",")]
@@ -332,7 +348,7 @@ def main():
     for _ in range(args.warmup):
         step()
     if rank == 0:
-        time.sleep(0.3)           # nvidia-smi is delivering samples by now
+        clocks.wait_ready()       # nvidia-smi is delivering samples from here on
     wall0 = time.time()
     total_ms = timed(step, args.steps)
     wall1 = time.time()
