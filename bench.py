@@ -149,7 +149,7 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def measure_extra(case, vb, inputs, torch, dev, pk):
+def measure_extra(case, vb, inputs, torch, dev, pk, ratios=((0.3, 0.3), (0.5, 0.5), (1.0, 1.0))):
     """Sampled and dense backward of a second, larger layer (not the headline metric): times per call
     and per stage, achieved rates of each kernel against the measured peaks."""
     N, T, d_in, d_out, R = case.N, case.T, case.d_in, case.d_out, case.R
@@ -158,7 +158,7 @@ def measure_extra(case, vb, inputs, torch, dev, pk):
     dX = torch.empty(R, d_in, dtype=case.dtype, device=dev)
     dW = torch.empty(d_out, d_in, dtype=torch.float32, device=dev)
     out = {"N": N, "T": T, "d_in": d_in, "d_out": d_out, "points": []}
-    for rho, nu in ((0.3, 0.3), (0.5, 0.5), (1.0, 1.0)):
+    for rho, nu in ratios:
         seeds = list(range(8))
         for sd in seeds[:2]:
             layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
@@ -417,7 +417,10 @@ def main():
     if world == 1 and not args.no_extra:
         del Xs, dYs, host
         torch.cuda.empty_cache()
-        extra = {"llm_mlp_up": measure_extra(inputs.CASES["llm_mlp_up"], vb, inputs, torch, dev, pk)}
+        extra = {"llm_mlp_up": measure_extra(inputs.CASES["llm_mlp_up"], vb, inputs, torch, dev, pk),
+                 # a BERT-large FFN linear at the keep ratios of a top, a middle and a bottom layer
+                 "bert_large_ffn_up": measure_extra(inputs.CASES["bert_large_ffn_up"], vb, inputs, torch, dev, pk,
+                                                    ratios=((0.8, 0.3), (0.5, 0.3), (0.2, 0.3)))}
 
     if rank != 0:
         if world > 1:
