@@ -352,3 +352,36 @@ def test_unbiasedness_on_gpu():
         slope = np.log(err[2000][k] / err[20][k]) / np.log(100.0)
         assert -1.6 < slope < -0.4, (k, err)
     layer.close()
+
+
+def test_interleaved_calls_on_two_handles_repeat_bitwise():
+    """Sampled, dense and probe calls of two layers, interleaved on two streams for many rounds: every round
+    reproduces the first bit for bit (the kernels keep counters in the workspace between launches - slice
+    tickets, work counters, probe accumulators - which each launch must leave re-armed), and no wait times out."""
+    shapes = [(48, 512, 512, 256), (40, 64, 256, 640)]      # the first has more tiles than SMs (work counter)
+    layers, data, first = [], [], []
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for (N, T, d_in, d_out) in shapes:
+        X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.0, sigma_B=0.5)
+        layers.append(vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR))
+        data.append(cuda(X, dY, W))
+    layers[0].set_tuning(256, 256, 0, 0, 3)        # whole waves + remainder on the first, automatic on the second
+    torch.cuda.synchronize()
+    for rnd in range(12):
+        outs = []
+        for k, (layer, (X, dY, W)) in enumerate(zip(layers, data)):
+            with torch.cuda.stream(streams[k]):
+                dX, dW = layer.linear_bwd(X, dY, W, 0.5, 0.5, 17 + k)
+                dXd, dWd = layer.dense_bwd(X, dY, W)
+                pr = layer.variance_probe([X, X], [dY, dY], W, 0.5, 0.5, 0.5, 99)
+                outs.append((dX.clone(), dW.clone(), dXd.clone(), dWd.clone(), pr.clone()))
+        torch.cuda.synchronize()
+        if rnd == 0:
+            first = outs
+        else:
+            for a, b in zip(first, outs):
+                for x, y in zip(a, b):
+                    assert torch.equal(x, y)
+    for layer in layers:
+        assert layer.device_status() == 0
+        layer.close()
