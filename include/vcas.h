@@ -196,7 +196,9 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
                        const vcas_config* cfg);
 
 /* Synchronises the device and returns the handle's device status word in *status
- * (VCAS_OK or VCAS_ERR_TIMEOUT / VCAS_ERR_INTERNAL); the word is then cleared. */
+ * (VCAS_OK or VCAS_ERR_TIMEOUT / VCAS_ERR_INTERNAL); the word is then cleared.  After an
+ * error the outputs of the calls since the last check are undefined; the workspace counters
+ * that a kernel which gave up may have left behind are reset, so the handle stays usable. */
 int vcas_last_device_status(vcas_handle h, int32_t* status);
 
 /* Tuning overrides for the tensor-core products (the paper has no counterpart): output tile
