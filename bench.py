@@ -1,22 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the sampled linear backward (VCAS) on B200.
 
-Workload: the BERT-base FFN up-projection layer (N=32, T=128, 768 -> 3072, bf16 inputs, fp32
-accumulation) at keep ratios rho = 0.3, nu = 0.4, with the variance probe (M = 4 Monte-Carlo
-batches) and the ratio update run once every F = 100 backward calls.
+Headline workload: the LLM-sized MLP up-projection (N=8, T=2048, 4096 -> 11008, bf16 inputs, fp32
+accumulation) at keep ratios rho = nu = 0.3, with the variance probe (M = 2 Monte-Carlo batches) and the
+ratio update run once every F = 100 backward calls.
 
-One STEP = one adaptation period of Alg. 1: 1 probe + 1 ratio update + F sampled backward
-calls.  The metric is milliseconds per layer backward = step time / F (probe amortised in).
-Inputs rotate over 8 distinct (X, dY) batches (252 MB > the 126 MB L2), so every call reads
-its inputs from HBM.
+One STEP = one adaptation period of Alg. 1: 1 probe + 1 ratio update + F sampled backward calls.  The
+metric is milliseconds per layer backward = step time / F (probe amortised in).  One call reads 495 MB of
+inputs (> the 126 MB L2) and the calls alternate between distinct batches, so every call reads HBM.
 
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.  The other workloads
+(fp32 layer, BERT-base FFN layer with its probe, ViT MLP block, BERT-large stack, the ratio sweep) are
+reported under `other_workloads` of the same line.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -26,11 +28,14 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-WORKLOAD = "bert_base_ffn_up"
+WORKLOAD = "llm_mlp_up"
+RHO = NU = 0.3
 F_CALLS = 100
-PROBE_M = 4
-N_BATCHES = 8
+PROBE_M = 2
+N_BATCHES = 2
 METRIC = "sampled linear-bwd ms/layer"
+SLAB = 1024            # d_out columns of the layer that one oracle sample computes (CPU baseline)
+SWEEP = (1.0, 0.7, 0.5, 0.3, 0.1)
 
 
 def peaks():
@@ -42,19 +47,23 @@ def peaks():
     return dict(hbm=6650.0, tc_burst=1590.0, tc_sustained=1400.0, source="fallback")
 
 
-def ncu_traffic(kernel: str):
-    """DRAM bytes per launch of `kernel` from the last ncu capture (profiles/), or None when the kernel's
-    source file has changed since that capture."""
+def ncu_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of `kernel` on `workload` from the ncu capture summarised in
+    profiles/dram_traffic.md, or None when there is no capture or the kernel's source file has changed
+    since it was taken (the table stores the file's SHA-256)."""
     import hashlib
-    path = os.path.join(ROOT, "paper_2402_17227_b200", "ncu_traffic.json")
+    path = os.path.join(ROOT, "profiles", "dram_traffic.md")
     if not os.path.exists(path):
         return None
-    rec = json.load(open(path)).get(kernel)
-    if rec is None:
-        return None
-    src = os.path.join(ROOT, "paper_2402_17227_b200", "csrc", rec["source"])
-    sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
-    return rec["dram_bytes_per_launch"] if sha == rec["source_sha256"] else None
+    for line in open(path):
+        f = [x.strip().strip("`") for x in line.strip().strip("|").split("|")]
+        if len(f) >= 5 and f[0] == kernel and f[1] == workload:
+            src = os.path.join(ROOT, "paper_2402_17227_b200", "csrc", f[3])
+            if not os.path.exists(src):
+                return None
+            sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+            return float(f[2]) if sha == f[4] else None
+    return None
 
 
 class ClockSampler:
@@ -127,17 +136,21 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm), samples_outside_timed_region=seen - len(sm))
 
 
-def oracle_call(case, batch=0, seed=0):
-    """One sampled backward of the workload by the CPU oracle; returns seconds."""
+# ------------------------------------------------------------------------------------ CPU oracle
+def oracle_slab_call(case, rho, nu, batch=0, seed=0, slab=SLAB):
+    """One sampled backward by the CPU oracle of the layer restricted to its first `slab` output features
+    (all N*T rows, all d_in; dY[:, :slab], W[:slab]).  Returns (seconds, scale) where scale = d_out / slab is
+    the factor by which the layer's two products are larger than the sample's."""
     import numpy as np
     from oracle import vcas_oracle as o
     from paper_2402_17227_b200 import inputs
-    X, dY, W = inputs.make_layer(case, batch=batch)
+    slab = min(slab, case.d_out)
+    X, dY, W = inputs.make_layer(case, batch=batch, d_out=slab)
     to64 = lambda t: t.float().numpy().astype(np.float64)
     X, dY, W = to64(X), to64(dY), to64(W)
     t0 = time.perf_counter()
-    o.linear_bwd(X, dY, W, case.N, case.T, float(np.float32(case.rho)), float(np.float32(case.nu)), seed)
-    return time.perf_counter() - t0
+    o.linear_bwd(X, dY, W, case.N, case.T, float(np.float32(rho)), float(np.float32(nu)), seed)
+    return time.perf_counter() - t0, case.d_out / slab
 
 
 def blas_threads() -> int:
@@ -149,106 +162,314 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def measure_extra(case, vb, inputs, torch, dev, pk, ratios=((0.3, 0.3), (0.5, 0.5), (1.0, 1.0))):
-    """Sampled and dense backward of a second, larger layer (not the headline metric): times per call
-    and per stage, achieved rates of each kernel against the measured peaks."""
-    N, T, d_in, d_out, R = case.N, case.T, case.d_in, case.d_out, case.R
-    X, dY, W = [t.to(dev) for t in inputs.make_layer(case)]
-    layer = vb.Layer(N, T, d_in, d_out, case.dtype)
-    dX = torch.empty(R, d_in, dtype=case.dtype, device=dev)
-    dW = torch.empty(d_out, d_in, dtype=torch.float32, device=dev)
-    out = {"N": N, "T": T, "d_in": d_in, "d_out": d_out, "points": []}
-    for rho, nu in ratios:
-        seeds = list(range(8))
-        for sd in seeds[:2]:
-            layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
-            layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
-        torch.cuda.synchronize()
-        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-        e[0].record()
-        for sd in seeds:
-            layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
-        e[1].record()
-        for sd in seeds:
-            layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
-        e[2].record()
-        torch.cuda.synchronize()
-        layer.set_profiling(True)                 # stage times: kernels one after the other
-        for sd in seeds:
-            layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
-            layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
-        ms, calls = layer.stage_times()
-        layer.set_profiling(False)
-        kA = kW = 0
-        for sd in seeds:
-            smp = layer.score(X, dY, rho, nu, sd)
-            kA += smp.cntA * T / len(seeds)
-            kW += smp.cntW / len(seeds)
-        n = len(seeds)
-        t_s, t_d = e[0].elapsed_time(e[1]) / n, e[1].elapsed_time(e[2]) / n
-        per = [m / n for m in ms]
-        flops_ratio = 2.0 * R / max(1.0, kA + kW)
-        out["points"].append({
-            "rho": rho, "nu": nu, "kept_A": kA, "kept_W": kW,
-            "sampled_ms": t_s, "dense_ms": t_d, "speedup_vs_dense": t_d / t_s, "flops_reduction_ratio": flops_ratio,
-            "speedup_over_flops_ratio": t_d / t_s / flops_ratio,
-            "rownorm": {"ms": per[0], "GBs": (R * (d_in + d_out) * 2) / per[0] / 1e6,
-                        "frac_of_hbm_peak": (R * (d_in + d_out) * 2) / per[0] / 1e6 / pk["hbm"]},
-            "sampler_ms": per[1],
-            "dx": {"ms": per[2], "TFLOPs": 2.0 * kA * d_in * d_out / per[2] / 1e9,
-                   "frac_of_bf16_peak": 2.0 * kA * d_in * d_out / per[2] / 1e9 / pk["tc_burst"]},
-            "pack_ms": per[3],
-            "dw": {"ms": per[4], "TFLOPs": 2.0 * kW * d_in * d_out / per[4] / 1e9,
-                   "frac_of_bf16_peak": 2.0 * kW * d_in * d_out / per[4] / 1e9 / pk["tc_burst"]},
-            "dense_dx_TFLOPs": 2.0 * R * d_in * d_out / per[5] / 1e9,
-            "dense_dw_TFLOPs": 2.0 * R * d_in * d_out / per[6] / 1e9,
-        })
-    assert layer.device_status() == 0
-    layer.close()
-    return out
+def cpu_baseline(case, rho, nu, reps):
+    ts = []
+    scale = 1.0
+    for k in range(reps):
+        t, scale = oracle_slab_call(case, rho, nu, batch=k % N_BATCHES, seed=k)
+        ts.append(t)
+    ms = 1e3 * scale * sum(ts) / len(ts)
+    return {"value": ms, "unit": "ms", "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{reps} oracle calls (numpy float64, BLAS threads = cores) on a slab of {min(SLAB, case.d_out)} of the "
+                      f"layer's {case.d_out} output features with all rows; time scaled by {scale:.2f} (extrapolated)"}
 
 
 def run_reference(args):
-    """The oracle as it stands, on the host cores: each step is one sampled backward of the workload."""
+    """The oracle as it stands, on the host cores: each step is one bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import numpy  # noqa: F401  (loads BLAS so that the thread count can be read)
     from paper_2402_17227_b200 import inputs
     case = inputs.CASES[WORKLOAD]
-    for w in range(args.warmup):
-        oracle_call(case, batch=w % N_BATCHES, seed=w)
-    ts = [oracle_call(case, batch=k % N_BATCHES, seed=1000 + k) for k in range(args.steps)]
-    ms = 1e3 * sum(ts) / len(ts)
+    for w in range(min(args.warmup, 1)):
+        oracle_slab_call(case, RHO, NU, batch=w % N_BATCHES, seed=w)
+    ts, scale = [], 1.0
+    for k in range(args.steps):
+        t, scale = oracle_slab_call(case, RHO, NU, batch=k % N_BATCHES, seed=1000 + k)
+        ts.append(t)
+    ms = 1e3 * scale * sum(ts) / len(ts)
     cores = blas_threads()
     line = {
         "impl": "reference", "metric": METRIC, "value": ms, "unit": "ms", "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "N": case.N, "T": case.T, "d_in": case.d_in, "d_out": case.d_out,
-                   "rho": case.rho, "nu": case.nu, "step": "one sampled backward of the layer by the CPU oracle"},
+        "warmup": args.warmup, "ms_per_step": 1e3 * sum(ts) / len(ts), "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(case, 1, "one sampled backward by the CPU oracle of a slab of "
+                                  f"{SLAB} of the layer's {case.d_out} output features; value = time x {scale:.2f}"),
         "cpu_baseline": {"value": ms, "unit": "ms", "cores": cores, "kind": "oracle",
-                         "sample": f"{args.steps} full-size sampled backward calls, one per step"},
+                         "sample": f"{args.steps} slab calls, one per step ({SLAB} of {case.d_out} output features, "
+                                   f"all rows), time scaled by {scale:.2f} (extrapolated)"},
         "e2e": {"value": ms, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
 
+def workload_config(case, world, step):
+    return {"workload": WORKLOAD, "N": case.N, "T": case.T, "d_in": case.d_in, "d_out": case.d_out,
+            "rho": RHO, "nu": NU, "step": step,
+            "l2": "each call reads 495 MB of inputs (> 126 MB L2); calls alternate between distinct batches",
+            "parallelism": f"{world} data-parallel replica(s), no exchange"}
+
+
+# ---------------------------------------------------------------------------------- GPU helpers
+class Timer:
+    def __init__(self, torch, dist, dist_util, dev, world):
+        self.torch, self.dist, self.du, self.dev, self.world = torch, dist, dist_util, dev, world
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def __call__(self, fn, reps):
+        """Milliseconds of `reps` runs of fn (CUDA events on the current stream), max over ranks."""
+        torch = self.torch
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        self.barrier()
+        return self.du.max_over_ranks(e0.elapsed_time(e1), self.dev)
+
+
+def stage_profile(torch, layer, calls_sampled, calls_dense):
+    """Per-stage milliseconds per call from CUDA events at the stage boundaries (kernels serialised on one
+    stream).  The calls are enqueued behind a spinning kernel so that their launches are queued when the
+    GPU reaches them and the events bracket GPU time, not the host's launch cost."""
+    layer.set_profiling(True)
+    torch.cuda.synchronize()
+    torch.cuda._sleep(4_000_000)
+    n_s = calls_sampled()
+    ms_s, _ = layer.stage_times()
+    torch.cuda._sleep(4_000_000)
+    n_d = calls_dense()
+    ms_d, _ = layer.stage_times()
+    layer.set_profiling(False)
+    per = [m / max(1, n_s) for m in ms_s[:5]] + [ms_d[5] / max(1, n_d), ms_d[6] / max(1, n_d)]
+    return per
+
+
+def point_report(case, rho, nu, kA, kW, t_s, t_d, per, pk):
+    """One (rho, nu) point in the layout of the report: kept rows, times, achieved rates and fractions."""
+    R, d_in, d_out = case.R, case.d_in, case.d_out
+    b = 4 if str(case.dtype).endswith("float32") else 2
+    score_bytes = R * (d_in + d_out) * b
+    flops_ratio = 2.0 * R / max(1.0, kA + kW)
+    rate = lambda work, ms: (work / ms / 1e9) if ms and ms > 0 else None
+    out = {
+        "rho": rho, "nu": nu, "kept_A": kA, "kept_W": kW,
+        "sampled_ms": t_s, "dense_ms": t_d, "speedup_vs_dense": t_d / t_s if t_s else None,
+        "flops_reduction_ratio": flops_ratio,
+        "speedup_over_flops_ratio": (t_d / t_s / flops_ratio) if t_s else None,
+    }
+    if per is not None:
+        gbs = score_bytes / per[0] / 1e6 if per[0] else None
+        out.update({
+            "rownorm": {"ms": per[0], "GBs": gbs, "frac_of_hbm_peak": gbs / pk["hbm"] if gbs else None},
+            "sampler_ms": per[1],
+            "dx": {"ms": per[2], "TFLOPs": rate(2.0 * kA * d_in * d_out, per[2]),
+                   "frac_of_bf16_peak": (rate(2.0 * kA * d_in * d_out, per[2]) or 0) / pk["tc_burst"]},
+            "pack_ms": per[3],
+            "dw": {"ms": per[4], "TFLOPs": rate(2.0 * kW * d_in * d_out, per[4]),
+                   "frac_of_bf16_peak": (rate(2.0 * kW * d_in * d_out, per[4]) or 0) / pk["tc_burst"]},
+            "dense_dx_TFLOPs": rate(2.0 * R * d_in * d_out, per[5]),
+            "dense_dw_TFLOPs": rate(2.0 * R * d_in * d_out, per[6]),
+        })
+    return out
+
+
+def measure_layer(case, vb, inputs, torch, dev, pk, ratios, seeds, profile=True, tensors=None, layer=None):
+    """Sampled and dense backward of one layer at several (rho, nu): per call and per stage."""
+    N, T, d_in, d_out, R = case.N, case.T, case.d_in, case.d_out, case.R
+    if tensors is None:
+        tensors = [t.to(dev) for t in inputs.make_layer(case)]
+    X, dY, W = tensors
+    own = layer is None
+    if own:
+        layer = vb.Layer(N, T, d_in, d_out, case.dtype)
+    dX = torch.empty(R, d_in, dtype=case.dtype, device=dev)
+    dW = torch.empty(d_out, d_in, dtype=torch.float32, device=dev)
+    out = {"N": N, "T": T, "d_in": d_in, "d_out": d_out, "seeds_per_point": len(seeds),
+           "workspace_bytes": layer.workspace_bytes(), "points": []}
+    n = len(seeds)
+    for _ in range(3):
+        layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
+    torch.cuda.synchronize()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    e[0].record()
+    for _ in seeds:
+        layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
+    e[1].record()
+    torch.cuda.synchronize()
+    t_d = e[0].elapsed_time(e[1]) / n
+    for rho, nu in ratios:
+        for sd in seeds[:3]:
+            layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
+        torch.cuda.synchronize()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        e[0].record()
+        for sd in seeds:
+            layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
+        e[1].record()
+        torch.cuda.synchronize()
+        t_s = e[0].elapsed_time(e[1]) / n
+        per = None
+        if profile:
+            def cs():
+                for sd in seeds:
+                    layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
+                return n
+
+            def cd():
+                for _ in range(4):
+                    layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
+                return 4
+            per = stage_profile(torch, layer, cs, cd)
+        kA = kW = 0.0
+        for sd in seeds:
+            smp = layer.score(X, dY, rho, nu, sd)
+            kA += smp.cntA * T / n
+            kW += smp.cntW / n
+        out["points"].append(point_report(case, rho, nu, kA, kW, t_s, t_d, per, pk))
+    assert layer.device_status() == 0, "device-side wait timed out"
+    if own:
+        layer.close()
+    return out
+
+
+def measure_bert_base_with_probe(vb, inputs, torch, dev, pk):
+    """BERT-base FFN up-projection (rho = .3, nu = .4) with the variance probe (M = 4) every 100 calls: ms per
+    layer backward with the probe amortised in, and the sampled / dense call alone (CUDA-graph replays)."""
+    case = inputs.CASES["bert_base_ffn_up"]
+    F, M, NB = 100, 4, 8
+    cfg = vb.default_config()
+    cfg.F, cfg.M = F, M
+    layer = vb.Layer(case.N, case.T, case.d_in, case.d_out, case.dtype, vb.GEMM_AUTO, cfg)
+    host = [inputs.make_layer(case, batch=b) for b in range(NB)]
+    W = host[0][2].to(dev)
+    Xs, dYs = [h[0].to(dev) for h in host], [h[1].to(dev) for h in host]
+    dX = torch.empty(case.R, case.d_in, dtype=case.dtype, device=dev)
+    dW = torch.empty(case.d_out, case.d_in, dtype=torch.float32, device=dev)
+    probe_out = torch.zeros(5, dtype=torch.float32, device=dev)
+    k = [0]
+
+    def calls():
+        for _ in range(F):
+            b = k[0] % NB
+            layer.linear_bwd_plain(Xs[b], dYs[b], W, case.rho, case.nu, k[0], dX, dW)
+            k[0] += 1
+
+    def dense():
+        for _ in range(F):
+            b = k[0] % NB
+            layer.dense_bwd(Xs[b], dYs[b], W, dX=dX, dW=dW)
+            k[0] += 1
+    calls(); dense()
+    torch.cuda.synchronize()
+    g_calls, g_dense = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_calls):
+        calls()
+    with torch.cuda.graph(g_dense):
+        dense()
+
+    def period():
+        layer.variance_probe(Xs[:M], dYs[:M], W, case.rho, case.nu, 1.0, 7777 + k[0], out=probe_out)
+        v = probe_out.cpu().numpy()
+        vb.update_ratios(1.0, [1.0], [1.0], [v[0]], [v[1]], [v[2]], [v[3]], [v[4]], cfg)
+        g_calls.replay()
+
+    def ms_of(fn, reps):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+    for _ in range(3):
+        period()
+    t_period = ms_of(period, 10)
+    t_calls = ms_of(g_calls.replay, 10)
+    t_dense = ms_of(g_dense.replay, 10)
+    pt = measure_layer(case, vb, inputs, torch, dev, pk, [(case.rho, case.nu)], list(range(16)),
+                       tensors=(Xs[0], dYs[0], W), layer=layer)
+    pt.update({"ms_per_layer_with_probe_every_100_calls": t_period / F, "sampled_call_ms_graph_replay": t_calls / F,
+               "dense_call_ms_graph_replay": t_dense / F, "probe_M": M,
+               "speedup_vs_dense_graph_replay": t_dense / t_calls})
+    layer.close()
+    return pt
+
+
+def measure_vit_block(vb, inputs, torch, dev, pk):
+    """ViT-base MLP block (N=64, T=197, 768 -> 3072 -> 768): backward through fc2 with the GELU Jacobian fused
+    into its dX epilogue, then fc1 on the library's own output (data dropped by fc2 arrive as zero rows)."""
+    fc2, fc1 = inputs.CASES["vit_base_mlp_fc2"], inputs.CASES["vit_base_mlp_fc1"]
+    N, T, hidden, d = fc2.N, fc2.T, fc2.d_in, fc2.d_out
+    R = N * T
+    H = inputs.make_preactivation(fc2, width=hidden).to(dev)
+    A = torch.nn.functional.gelu(H.float()).to(torch.bfloat16)
+    _, dZ2, W2 = [t.to(dev) for t in inputs.make_layer(fc2)]
+    X1, _, W1 = [t.to(dev) for t in inputs.make_layer(fc1)]
+    l2, l1 = vb.Layer(N, T, hidden, d, torch.bfloat16), vb.Layer(N, T, d, hidden, torch.bfloat16)
+    dZ1 = torch.empty(R, hidden, dtype=torch.bfloat16, device=dev)
+    dW2 = torch.empty(d, hidden, dtype=torch.float32, device=dev)
+    dX1 = torch.empty(R, d, dtype=torch.bfloat16, device=dev)
+    dW1 = torch.empty(hidden, d, dtype=torch.float32, device=dev)
+    seeds = list(range(20))
+
+    def sampled(sd):
+        l2.linear_bwd(A, dZ2, W2, fc2.rho, fc2.nu, sd, H=H, dX=dZ1, dW=dW2)
+        l1.linear_bwd_plain(X1, dZ1, W1, fc2.rho, fc2.nu, sd + 1000, dX1, dW1)
+
+    def dense():
+        l2.dense_bwd(A, dZ2, W2, dX=dZ1, dW=dW2)
+        l1.dense_bwd(X1, dZ1, W1, dX=dX1, dW=dW1)
+    for sd in seeds[:3]:
+        sampled(sd); dense()
+    torch.cuda.synchronize()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    e[0].record()
+    for sd in seeds:
+        sampled(sd)
+    e[1].record()
+    for _ in seeds:
+        dense()
+    e[2].record()
+    torch.cuda.synchronize()
+    kept = []
+    for sd in seeds:
+        sampled(sd)
+        s2, s1 = l2.last_sampling(), l1.last_sampling()
+        kept.append((s2.cntA * T, s2.cntW, s1.cntA * T, s1.cntW))
+    kA2, kW2, kA1, kW1 = [sum(k[i] for k in kept) / len(kept) for i in range(4)]
+    t_s, t_d = e[0].elapsed_time(e[1]) / len(seeds), e[1].elapsed_time(e[2]) / len(seeds)
+    ratio = 4.0 * R / max(1.0, kA2 + kW2 + kA1 + kW1)
+    assert l1.device_status() == 0 and l2.device_status() == 0
+    l1.close(); l2.close()
+    return {"N": N, "T": T, "d": d, "hidden": hidden, "rho": fc2.rho, "nu": fc2.nu, "seeds": len(seeds),
+            "sampled_block_ms": t_s, "dense_block_ms": t_d, "speedup_vs_dense": t_d / t_s,
+            "kept_rows": {"fc2_A": kA2, "fc2_W": kW2, "fc1_A": kA1, "fc1_W": kW1},
+            "flops_reduction_ratio": ratio, "speedup_over_flops_ratio": t_d / t_s / ratio,
+            "note": "dense block: exact products of both linears, without the GELU Jacobian"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="vcas", choices=["vcas", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extra", action="store_true", help="skip the LLM-sized layer reported under other_workloads")
+    ap.add_argument("--no-extra", action="store_true", help="skip the workloads reported under other_workloads")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
     args.warmup = max(args.warmup, 3)
 
-    import numpy as np
     import torch
     import torch.distributed as dist
 
@@ -269,10 +490,11 @@ def main():
     if world > 1:
         dist.barrier()
     vb.lib()
+    pk = peaks()
+    timed = Timer(torch, dist, dist_util, dev, world)
 
     case = inputs.CASES[WORKLOAD]
     N, T, d_in, d_out, R = case.N, case.T, case.d_in, case.d_out, case.R
-    rho, nu = case.rho, case.nu
     cfg = vb.default_config()
     cfg.F, cfg.M = F_CALLS, PROBE_M
     layer = vb.Layer(N, T, d_in, d_out, case.dtype, vb.GEMM_AUTO, cfg)
@@ -291,7 +513,7 @@ def main():
     def calls_only():
         for _ in range(F_CALLS):
             b = call_no[0] % N_BATCHES
-            layer.linear_bwd_plain(Xs[b], dYs[b], W, rho, nu, call_no[0], dX, dW)
+            layer.linear_bwd_plain(Xs[b], dYs[b], W, RHO, NU, call_no[0], dX, dW)
             call_no[0] += 1
 
     def dense_only():
@@ -318,7 +540,7 @@ def main():
     def step():
         # Alg. 1: every F calls probe the variances on M batches and update (s, rho_l, nu_l) ...
         l0 = layer.launch_count()
-        layer.variance_probe(Xs[:PROBE_M], dYs[:PROBE_M], W, rho, nu, state["s"], 7777 + call_no[0], out=probe_out)
+        layer.variance_probe(Xs[:PROBE_M], dYs[:PROBE_M], W, RHO, NU, state["s"], 7777 + call_no[0], out=probe_out)
         probe_launches[0] = layer.launch_count() - l0
         v = probe_out.cpu().numpy()
         s_new, rho_new, nu_new = vb.update_ratios(state["s"], state["rho"], state["nu"], [v[0]], [v[1]], [v[2]],
@@ -326,21 +548,6 @@ def main():
         state.update(s=s_new, rho=rho_new, nu=nu_new)
         # ... then F sampled backward calls (at the workload's fixed ratios, so that every step does the same work)
         graph_calls.replay()
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, reps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(reps):
-            fn()
-        e1.record()
-        barrier()
-        return dist_util.max_over_ranks(e0.elapsed_time(e1), dev)
 
     clocks = ClockSampler(local)
     if rank == 0:
@@ -358,37 +565,26 @@ def main():
     value = dist_util.ms_per_layer(ms_per_step, F_CALLS, world)      # whole-job: all ranks' calls per unit time
 
     # -- the same period without the probe, the dense backward (graph replays), and per-stage times
-    reps = max(3, min(args.steps, 10))
+    reps = 3
     ms_sampled = timed(graph_calls.replay, reps) / (reps * F_CALLS)
     ms_dense = timed(graph_dense.replay, reps) / (reps * F_CALLS)
-    ms_sampled_eager = timed(calls_only, 3) / (3 * F_CALLS)
-    # Stage times with CUDA events at the stage boundaries.  The calls are enqueued behind 2 ms of a
-    # spinning kernel, so that all their launches are already queued when the GPU reaches them and the
-    # events bracket GPU time, not the host's launch cost.  (While profiling, the library runs its kernels
-    # one after the other; in the timed runs dX runs beside pack + dW, so a call takes less than the sum.)
     prof_seeds = [99000 + k for k in range(40)]
-    layer.set_profiling(True)
-    torch.cuda.synchronize()
-    torch.cuda._sleep(4_000_000)          # a spinning kernel of about 2 ms: low power, does not disturb the clocks
-    for k, sd in enumerate(prof_seeds):
-        b = k % N_BATCHES
-        layer.linear_bwd_plain(Xs[b], dYs[b], W, rho, nu, sd, dX, dW)
-    stage_ms, stage_calls = layer.stage_times()
-    torch.cuda._sleep(4_000_000)
-    for k in range(40):
-        b = k % N_BATCHES
-        layer.dense_bwd(Xs[b], dYs[b], W, dX=dX, dW=dW)
-    dense_stage_ms, dense_calls = layer.stage_times()
-    layer.set_profiling(False)
-    # realised kept rows of those calls (the FLOPs the products actually did)
-    kept_A = kept_W = 0
-    for k, sd in enumerate(prof_seeds):
-        b = k % N_BATCHES
-        smp = layer.score(Xs[b], dYs[b], rho, nu, sd)
-        kept_A += smp.cntA * T
-        kept_W += smp.cntW
-    kept_A /= len(prof_seeds)
-    kept_W /= len(prof_seeds)
+
+    def prof_sampled():
+        for k, sd in enumerate(prof_seeds):
+            layer.linear_bwd_plain(Xs[k % N_BATCHES], dYs[k % N_BATCHES], W, RHO, NU, sd, dX, dW)
+        return len(prof_seeds)
+
+    def prof_dense():
+        for k in range(8):
+            layer.dense_bwd(Xs[k % N_BATCHES], dYs[k % N_BATCHES], W, dX=dX, dW=dW)
+        return 8
+    per = stage_profile(torch, layer, prof_sampled, prof_dense)
+    kept_A = kept_W = 0.0
+    for k, sd in enumerate(prof_seeds):      # realised kept rows of those calls (the FLOPs the products did)
+        smp = layer.score(Xs[k % N_BATCHES], dYs[k % N_BATCHES], RHO, NU, sd)
+        kept_A += smp.cntA * T / len(prof_seeds)
+        kept_W += smp.cntW / len(prof_seeds)
     assert layer.device_status() == 0, "device-side wait timed out"
 
     # -- end to end through the C ABI from pinned host buffers (H2D of X, dY; D2H of dX, dW every call)
@@ -401,34 +597,42 @@ def main():
         for k in range(n):
             hX.copy_(pin[k % 2][0], non_blocking=True)
             hdY.copy_(pin[k % 2][1], non_blocking=True)
-            layer.linear_bwd_plain(hX, hdY, W, rho, nu, 424242 + k, dX, dW)
+            layer.linear_bwd_plain(hX, hdY, W, RHO, NU, 424242 + k, dX, dW)
             out_dX.copy_(dX, non_blocking=True)
             out_dW.copy_(dW, non_blocking=True)
         torch.cuda.synchronize()
 
-    e2e_calls(3)
-    n_e2e = 20
+    e2e_calls(2)
+    n_e2e = 6
     e2e_ms = timed(lambda: e2e_calls(n_e2e), 1) / (n_e2e * world)
     h2d = Xs[0].numel() * 2 + dYs[0].numel() * 2
     d2h = dX.numel() * 2 + dW.numel() * 4
+    del pin, hX, hdY, out_dX, out_dW
 
-    pk = peaks()
     extra = None
     if world == 1 and not args.no_extra:
+        sweep_seeds = list(range(20))
+        grid = [(r, n) for r in SWEEP for n in SWEEP]
+        extra = {
+            # BASELINE configs[4]: the 5 x 5 grid of keep ratios on the headline layer, 20 seeds per point
+            "llm_mlp_up_ratio_sweep": measure_layer(case, vb, inputs, torch, dev, pk, grid, sweep_seeds,
+                                                    tensors=(Xs[0], dYs[0], W), layer=layer),
+        }
         del Xs, dYs, host
         torch.cuda.empty_cache()
-        extra = {"llm_mlp_up": measure_extra(inputs.CASES["llm_mlp_up"], vb, inputs, torch, dev, pk),
-                 # a BERT-large FFN linear at the keep ratios of a top, a middle and a bottom layer
-                 "bert_large_ffn_up": measure_extra(inputs.CASES["bert_large_ffn_up"], vb, inputs, torch, dev, pk,
-                                                    ratios=((0.8, 0.3), (0.5, 0.3), (0.2, 0.3)))}
+        extra["fp32_small"] = measure_layer(inputs.CASES["fp32_small"], vb, inputs, torch, dev, pk, [(0.5, 0.5)],
+                                            list(range(50)))
+        extra["bert_base_ffn_up"] = measure_bert_base_with_probe(vb, inputs, torch, dev, pk)
+        extra["vit_base_mlp_block"] = measure_vit_block(vb, inputs, torch, dev, pk)
+        # a BERT-large FFN linear at the keep ratios of a top, a middle and a bottom layer
+        extra["bert_large_ffn_up"] = measure_layer(inputs.CASES["bert_large_ffn_up"], vb, inputs, torch, dev, pk,
+                                                   [(0.8, 0.3), (0.5, 0.3), (0.2, 0.3)], list(range(20)))
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    nc = max(1, stage_calls[0])
-    per = [m / nc for m in stage_ms[:5]]
     names = ["rownorm_kernel", "sampler_kernel", "umma_dx_kernel", "pack_kernel", "umma_dw_kernel"]
     bytes_score = (R * d_out + R * d_in) * 2                      # every input byte read once
     flops_dx = 2.0 * kept_A * d_in * d_out
@@ -440,16 +644,19 @@ def main():
         "pack_kernel": dict(ms=per[3], bound="hbm"),
         "umma_dw_kernel": dict(ms=per[4], bound="tensor", achieved=flops_dw / per[4] / 1e9 if per[4] else None),
     }
+    for k, v in stages.items():
+        if v.get("achieved"):
+            v["frac"] = v["achieved"] / (pk["hbm"] if v["bound"] == "hbm" else pk["tc_burst"])
     dom = max(range(5), key=lambda i: per[i])
     dname = names[dom]
     if stages[dname]["bound"] == "tensor":
         roof = dict(bound="tensor", kernel=dname, achieved=stages[dname]["achieved"], peak=pk["tc_burst"],
-                    unit="TFLOP/s", traffic=ncu_traffic(dname), peak_source=pk["source"] + " bf16 burst")
+                    unit="TFLOP/s", traffic=ncu_traffic(dname, WORKLOAD), peak_source=pk["source"] + " bf16 burst")
     else:
         if dname != "rownorm_kernel":   # the small latency-bound stages are reported under the scoring pass
             dname = "rownorm_kernel"
         roof = dict(bound="hbm", kernel=dname, achieved=stages[dname]["achieved"], peak=pk["hbm"], unit="GB/s",
-                    traffic=ncu_traffic(dname), peak_source=pk["source"] + " copy bandwidth")
+                    traffic=ncu_traffic(dname, WORKLOAD), peak_source=pk["source"] + " copy bandwidth")
     roof["frac"] = roof["achieved"] / roof["peak"] if roof["achieved"] else None
     roof["kernel_ms"] = stages[dname]["ms"]
 
@@ -458,11 +665,8 @@ def main():
         "metric": METRIC, "value": value, "unit": "ms", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "N": N, "T": T, "d_in": d_in, "d_out": d_out, "rho": rho, "nu": nu,
-                   "step": f"1 variance probe (M={PROBE_M}) + 1 ratio update + {F_CALLS} sampled backward calls "
-                           "(the calls replayed from one CUDA graph)",
-                   "l2": f"inputs rotate over {N_BATCHES} batches (252 MB > 126 MB L2)",
-                   "parallelism": f"{world} data-parallel replica(s), no exchange"},
+        "config": workload_config(case, world, f"1 variance probe (M={PROBE_M}) + 1 ratio update + {F_CALLS} sampled "
+                                  "backward calls (the calls replayed from one CUDA graph)"),
         "clocks": clock_info,
         "e2e": {"value": e2e_ms, "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "note": "one vcas_linear_bwd per step with X, dY copied from pinned host memory and dX, dW copied back"},
@@ -470,21 +674,18 @@ def main():
         "roofline": roof,
         "stages": stages,
         "sampled_ms_per_layer": ms_sampled, "dense_ms_per_layer": ms_dense,
-        "sampled_ms_per_layer_eager_launch": ms_sampled_eager,
-        "dense_stages_ms": {"umma_dx_kernel": dense_stage_ms[5] / max(1, dense_calls[1]),
-                            "umma_dw_kernel": dense_stage_ms[6] / max(1, dense_calls[1])},
+        "dense_stages_ms": {"umma_dx_kernel": per[5], "umma_dw_kernel": per[6]},
         "speedup_vs_dense": ms_dense / ms_sampled if ms_sampled else None,
         "flops_reduction_ratio": flops_ratio,
         "speedup_over_flops_ratio": (ms_dense / ms_sampled) / flops_ratio if ms_sampled else None,
         "dense_tflops": 4.0 * R * d_in * d_out / ms_dense / 1e9,
         "kept_rows": {"kept_A": kept_A, "kept_W": kept_W, "R": R, "note": "mean over the 40 profiled calls"},
+        "workspace_bytes": layer.workspace_bytes(),
         "adaptation_state": state,
         "other_workloads": extra,
     }
     if not args.no_cpu_baseline and world == 1:
-        ts = [oracle_call(case, batch=k % N_BATCHES, seed=k) for k in range(30)]
-        line["cpu_baseline"] = {"value": 1e3 * sum(ts) / len(ts), "unit": "ms", "cores": blas_threads(),
-                                "kind": "oracle", "sample": "30 full-size sampled backward calls of the workload"}
+        line["cpu_baseline"] = cpu_baseline(case, RHO, NU, reps=3)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -176,7 +176,8 @@ int vcas_mask_from_probs(vcas_handle h, const float* p, int32_t n, uint64_t seed
  *   V_act = 1/M^2 sum_ij ||G_act,ij - G_s,i||_F^2,
  *   V_w   = 1/M^2 sum_ij V_w,ij,
  *   p_lo, p_hi = Eq. 4's sparsity p(s - alpha), p(s + alpha) averaged over the batches
- *   (App. D), s -+ alpha clipped to [0, 1].
+ *   (App. D), s -+ alpha clipped to [0, 1]; Eq. 4's n starts at 1, so p >= 1/N and the ratios
+ *   that vcas_update_ratios derives from them stay valid arguments of vcas_linear_bwd.
  * M >= 2 (the 1/(M-1) of V_s).  alpha comes from the handle's config.
  */
 int vcas_variance_probe(vcas_handle h, int32_t M, const void* const* X_i, const void* const* dY_i,

@@ -245,15 +245,17 @@ def var_sample_w(G_hat, X, q):
 # Ratio adaptation (Sec. 5, Alg. 1, App. D)
 # --------------------------------------------------------------------------------------
 def sparsity_p(g, s: float) -> float:
-    """Eq. 4: the smallest fraction n/N of data whose largest norms hold a share s of the total."""
+    """Eq. 4: the smallest fraction n/N of data whose largest norms hold a share s of the total.
+
+    n ranges over 1..N, as the sum over i = 1..n in Eq. 4 does: at least one datum is always
+    kept, so p(0) = 1/N, and an all-zero gradient gives 1/N as well (every n meets 0 >= 0).
+    """
     g = np.sort(np.asarray(g, dtype=np.float64))[::-1]
     total = 0.0
     for x in g:                      # sequential sum in descending order: the cumulative
         total += x                   # sum of all N terms equals the total bit for bit
-    if total == 0.0:
-        return 0.0
     target = s * total
-    cum, n = 0.0, 0
+    cum, n = g[0], 1
     while cum < target:
         cum += g[n]
         n += 1
@@ -364,3 +366,41 @@ def dW_rows(dY, X, p32, q32, keepW, T: int, outs):
     for i, oo in enumerate(outs):
         out[i] = (np.asarray(dY[kept, oo], dtype=np.float64) * scale) @ Xk
     return out
+
+
+def scores_and_masks_large(X, dY, N: int, T: int, rho: float, nu: float, seed: int, p_override=None,
+                           q_override=None, chunk: int = 2048):
+    """Steps of sample_a / sample_w that precede the products, without forming G_hat: the row norm of
+    G_hat_r is ||dY_r|| / p_n on rows of kept data and 0 elsewhere (Sec. 4.1), so the leverage scores of
+    Sec. 4.2 follow from the row square-norms.  Returns dict(a, b, g, p32, keepA, w, q32, keepW)."""
+    a = row_sqnorms_chunked(dY, chunk)
+    b = row_sqnorms_chunked(X, chunk)
+    g = datum_norms(a, N, T)
+    p32 = capped_prop(g, N * rho).astype(np.float32) if p_override is None else np.asarray(p_override, np.float32)
+    keepA = bernoulli_keep(p32, seed, 0)
+    inv = np.zeros(N)
+    inv[keepA] = 1.0 / p32[keepA].astype(np.float64)
+    w = np.sqrt(a) * np.repeat(inv, T) * np.sqrt(b)
+    if q_override is None:
+        q32 = capped_prop(w, nu * T * int(np.count_nonzero(keepA))).astype(np.float32)
+    else:
+        q32 = np.asarray(q_override, dtype=np.float32)
+    keepW = bernoulli_keep(q32, seed, 1)
+    return dict(a=a, b=b, g=g, p32=p32, keepA=keepA, w=w, q32=q32, keepW=keepW)
+
+
+def products_on_kept_rows(X, dY, W, p32, q32, keepA, keepW, T: int):
+    """dX = G_hat W and dW = G_tilde^T X (Eq. 2) computed from the kept rows alone: every other row of
+    G_hat and of G_tilde is zero by definition (Sec. 4.1, 4.2), so it contributes a zero row to dX and
+    nothing to dW.  Returns (dX [R, d_in], dW [d_out, d_in])."""
+    W = np.asarray(W, dtype=np.float64)
+    p = np.asarray(p32, dtype=np.float64)
+    q = np.asarray(q32, dtype=np.float64)
+    rowsA = np.flatnonzero(np.repeat(np.asarray(keepA, dtype=bool), T))
+    dX = np.zeros((dY.shape[0], W.shape[1]))
+    G_hat = np.asarray(dY[rowsA], dtype=np.float64) * (1.0 / p[rowsA // T])[:, None]
+    dX[rowsA] = G_hat @ W
+    rowsW = np.flatnonzero(np.asarray(keepW, dtype=bool))
+    G_tilde = np.asarray(dY[rowsW], dtype=np.float64) * (1.0 / p[rowsW // T])[:, None] * (1.0 / q[rowsW])[:, None]
+    dW = G_tilde.T @ np.asarray(X[rowsW], dtype=np.float64)
+    return dX, dW

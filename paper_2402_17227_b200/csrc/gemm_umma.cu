@@ -13,6 +13,8 @@
 // VCAS_ERR_TIMEOUT in the status word and leaves.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace vcas {
@@ -848,14 +850,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
+  static const EncodeTiledFn fn = []() -> EncodeTiledFn {     // initialised once, thread-safe
     void* p = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
         q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
+      return (EncodeTiledFn)p;
+    return nullptr;
+  }();
   return fn;
 }
 
@@ -886,6 +888,7 @@ struct Cand {
   double alone;    // time of the product when it has the GPU to itself, us
 };
 constexpr int MAX_CANDS = 64;
+constexpr int MAX_DEVICES = 64;
 
 // row_tiles128: number of 128-row tile rows (for dX: kept data x 128-token chunks); a 256-row tile covers two.
 // remainder_ok: 256-row tiles may leave a last partial wave to a second launch with 128-row tiles (mh = 3).
@@ -972,12 +975,14 @@ void best_pair(const Cand* c1, int n1, int ctas1, const Cand* c2, int n2, int ct
 template <int MODE, int BN, int MH, int KIND>
 cudaError_t run_gemm_k(Handle* h, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const GemmParams& P0,
                      long max_items, int ctas, bool pdl, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
+  static std::atomic<bool> attr_set[MAX_DEVICES];
+  if (h->device < 0 || h->device >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (!attr_set[h->device].load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(umma_kernel<MODE, BN, MH, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          TileCfg<BN, MH>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[h->device].store(true, std::memory_order_release);
   }
   GemmParams P = P0;
   cudaLaunchConfig_t cfg = {};

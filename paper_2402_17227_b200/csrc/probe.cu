@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(256) reduce_kernel(const float4* __restrict__ 
   }
 }
 
-// Eq. 4: p(s) = min{ n/N : sum of the n largest norms >= s * sum of all norms }, for two values of s.
+// Eq. 4: p(s) = min{ n/N, n >= 1 : sum of the n largest norms >= s * sum of all norms }, for two values of s.
 __global__ void __launch_bounds__(1024) sparsity_kernel(const float* __restrict__ g, float* __restrict__ sorted,
                                                         int N, double s_lo, double s_hi, double* __restrict__ acc) {
   // rank of g[i] in descending order (ties broken by index): a counting sort, N is a batch size
@@ -95,16 +95,15 @@ __global__ void __launch_bounds__(1024) sparsity_kernel(const float* __restrict_
   if (threadIdx.x == 0) {
     double total = 0.0;
     for (int i = 0; i < N; ++i) total += (double)sorted[i];
-    double res[2] = {0.0, 0.0};
+    // n ranges over 1..N (the sum over i = 1..n of Eq. 4): at least one datum is always kept
+    double res[2];
     const double ss[2] = {s_lo, s_hi};
-    if (total > 0.0) {
-      for (int k = 0; k < 2; ++k) {
-        const double target = ss[k] * total;
-        double cum = 0.0;
-        int n = 0;
-        while (cum < target && n < N) { cum += (double)sorted[n]; ++n; }
-        res[k] = (double)n / (double)N;
-      }
+    for (int k = 0; k < 2; ++k) {
+      const double target = ss[k] * total;
+      double cum = (double)sorted[0];
+      int n = 1;
+      while (cum < target && n < N) { cum += (double)sorted[n]; ++n; }
+      res[k] = (double)n / (double)N;
     }
     acc[2] += res[0];
     acc[3] += res[1];

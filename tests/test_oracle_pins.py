@@ -323,6 +323,35 @@ def test_probe_definitions():
     assert len(seeds) == M * M and 5 not in seeds
 
 
+def test_probe_sparsity_candidates_hand_case():
+    """p_lo / p_hi of the probe (App. D): Eq. 4 at s - alpha and s + alpha, averaged over the M batches,
+    with s -+ alpha clipped to [0, 1].  Norms are set by hand (T = 1, one non-zero entry per row), so the
+    expected values below come from Eq. 4 by mental arithmetic, not from the oracle."""
+    def batch(norms):
+        dY = np.zeros((4, 3)); dY[:, 1] = norms
+        return dY
+    X = np.ones((4, 2)); W = np.ones((3, 2))
+    # batch 0 norms 4 3 2 1 (total 10), batch 1 norms 8 1 .5 .5 (total 10); s = 0.7, alpha = 0.05
+    #   s - alpha = 0.65: batch 0 needs 4 + 3 >= 6.5 -> 2/4;   batch 1: 8 >= 6.5 -> 1/4;   mean 0.375
+    #   s + alpha = 0.75: batch 0 needs 4 + 3 + 2 >= 7.5 -> 3/4; batch 1: 8 >= 7.5 -> 1/4; mean 0.5
+    dYs = [batch([3.0, 1.0, 4.0, 2.0]), batch([0.5, 8.0, 0.5, 1.0])]
+    out = o.variance_probe([X, X], dYs, W, 4, 1, 0.5, 0.5, s=0.7, alpha=0.05, seed=0)
+    assert out["p_lo"] == 0.375 and out["p_hi"] == 0.5
+    # a swap of the two, a missing 1/M or a sum over the wrong side would give .5/.375, .75/1.0, ...
+    # clip at the top: s + alpha = 1.03 -> 1: all non-zero data, 3/4 in both batches (unclipped, no n exists)
+    dYs = [batch([3.0, 0.0, 4.0, 3.0]), batch([1.0, 8.0, 0.0, 1.0])]
+    out = o.variance_probe([X, X], dYs, W, 4, 1, 0.5, 0.5, s=0.98, alpha=0.05, seed=0)
+    assert out["p_hi"] == 0.75
+    assert out["p_lo"] == 0.75                    # 0.93: 4 + 3 + 3 and 8 + 1 + 1 are needed
+    # clip at the bottom: s - alpha < 0 -> 0: one datum (n >= 1); s + alpha = 0.07: the largest suffices
+    out = o.variance_probe([X, X], dYs, W, 4, 1, 0.5, 0.5, s=0.02, alpha=0.05, seed=0)
+    assert out["p_lo"] == 0.25 and out["p_hi"] == 0.25
+    # three batches, unequal results: the mean is over M
+    dYs = [batch([4.0, 3.0, 2.0, 1.0]), batch([8.0, 1.0, 0.5, 0.5]), batch([1.0, 1.0, 1.0, 1.0])]
+    out = o.variance_probe([X, X, X], dYs, W, 4, 1, 0.5, 0.5, s=0.7, alpha=0.05, seed=0)
+    assert np.isclose(out["p_lo"], (0.5 + 0.25 + 0.75) / 3) and np.isclose(out["p_hi"], (0.75 + 0.25 + 0.75) / 3)
+
+
 def test_probe_v_act_approaches_closed_form():
     # E ||G_act - G_s||^2 = sum_n (1-p_n)/p_n ||G_n^T X_n||_F^2 (Sec. 4.1 form, by linearity)
     r = rng(10)
@@ -344,9 +373,10 @@ def test_sparsity_p_hand_cases():
     assert o.sparsity_p(g, 0.71) == 0.75
     assert o.sparsity_p(g, 0.4) == 0.25
     assert o.sparsity_p(g, 1.0) == 1.0
-    assert o.sparsity_p(g, 0.0) == 0.0
+    assert o.sparsity_p(g, 0.0) == 0.25             # n starts at 1: one datum is always kept
+    assert o.sparsity_p(g, 0.39) == 0.25 and o.sparsity_p(g, 0.41) == 0.5
     assert o.sparsity_p([0.0, 5.0, 0.0, 0.0], 1.0) == 0.25     # only non-zero data are needed
-    assert o.sparsity_p(np.zeros(3), 0.5) == 0.0
+    assert o.sparsity_p(np.zeros(3), 0.5) == 1 / 3             # 0 >= 0 holds from n = 1 on
     r = rng(12)
     g = np.exp(r.standard_normal(33))
     vals = [o.sparsity_p(g, s) for s in np.linspace(0, 1, 21)]
@@ -408,3 +438,22 @@ def test_entrywise_forms_agree_with_whole_matrix_forms():
     assert np.allclose(o.dW_rows(dY, X, out["p32"], out["q32"], out["keepW"], T, outs), out["dW"][outs],
                        rtol=1e-12, atol=1e-12)
     assert np.allclose(o.row_sqnorms_chunked(dY, chunk=4), o.row_sqnorms(dY), rtol=1e-15)
+
+
+def test_kept_row_forms_agree_with_whole_matrix_forms():
+    # the forms the full-size GPU tests use are the same numbers as linear_bwd's, with and without overrides
+    N, T, di, do = 7, 6, 5, 8
+    X, dY, W = _tiny(22, N, T, di, do)
+    dY[2 * T:3 * T] = 0.0                                   # a datum dropped upstream
+    for over in (False, True):
+        ref = o.linear_bwd(X, dY, W, N, T, 0.6, 0.5, seed=9)
+        kw = dict(p_override=ref["p32"] * np.float32(0.9), q_override=np.minimum(1, ref["q32"] * np.float32(1.1))) if over else {}
+        ref = o.linear_bwd(X, dY, W, N, T, 0.6, 0.5, seed=9, **kw)
+        sm = o.scores_and_masks_large(X, dY, N, T, 0.6, 0.5, 9, chunk=5, **kw)
+        for k in ("a", "b", "g", "w"):
+            assert np.allclose(sm[k], ref[k], rtol=1e-13, atol=0)
+        for k in ("p32", "q32", "keepA", "keepW"):
+            assert np.array_equal(sm[k], ref[k])
+        dX, dW = o.products_on_kept_rows(X, dY, W, sm["p32"], sm["q32"], sm["keepA"], sm["keepW"], T)
+        assert np.allclose(dX, ref["dX"], rtol=1e-12, atol=1e-13) and np.allclose(dW, ref["dW"], rtol=1e-12, atol=1e-13)
+        assert 0 < sm["keepA"].sum() < N and 0 < sm["keepW"].sum() < sm["keepA"].sum() * T
