@@ -116,6 +116,39 @@ int vcas_linear_bwd_ex(vcas_handle h, const void* X, const void* dY, const void*
                        const float* p_in, const float* q_in, const void* H,
                        void* dX, float* dW, vcas_stream stream);
 
+/*
+ * Eq. 2 down a stack of layers.  Sec. 4: SampleA is applied at every layer, so "the activation gradient
+ * becomes increasingly sparse when backpropagating" - the dY of a layer is the dX of the layer above, whose
+ * rows of dropped data are exactly zero.  This variant lets a layer take what the layer above already
+ * knows instead of re-reading dY, and hand the same down; all fields optional (NULL), all pointers device:
+ *   H            as for vcas_linear_bwd_ex;
+ *   a_in         row square-norms of this call's dY as partial sums: ||dY_r||^2 = sum of the a_in_parts
+ *                consecutive floats a_in[r * a_in_parts ...]; with it dY is not read for scoring at all
+ *                (the a_out of the call that produced dY, with a_in_parts = that handle's vcas_chain_parts);
+ *   alive_in     ascending list of the data whose rows of dY may be non-zero, alive_cnt_in [1] its length
+ *                (the kept_out / kept_cnt_out of the layer above); every other datum is taken to be zero:
+ *                its rows of dY and a_in are never read, it is never kept, its rows of dX are zero;
+ *   a_out        [R][vcas_chain_parts] fp32: partial sums of the square-norm of every row of dX as stored
+ *                (after the GELU' factor and the rounding to the layer dtype), written by the dX product;
+ *   kept_out     [N] int32: ascending list of the data this call kept, kept_cnt_out [1] its length.
+ * alive_in / alive_cnt_in and kept_out / kept_cnt_out come in pairs; the lists must not alias.
+ */
+typedef struct {
+  const void* H;
+  const float* a_in;
+  int32_t a_in_parts;
+  const int32_t* alive_in;
+  const int32_t* alive_cnt_in;
+  float* a_out;
+  int32_t* kept_out;
+  int32_t* kept_cnt_out;
+} vcas_chain_args;
+int vcas_linear_bwd_chain(vcas_handle h, const void* X, const void* dY, const void* W,
+                          float rho, float nu, uint64_t seed, const vcas_chain_args* chain,
+                          void* dX, float* dW, vcas_stream stream);
+/* Number of partial sums per row that this handle's dX product writes to a_out (host out). */
+int vcas_chain_parts(vcas_handle h, int32_t* parts);
+
 /* Exact backprop dX = dY W, dW = dY^T X with the same kernels at ratio 1 and no scoring. */
 int vcas_dense_bwd(vcas_handle h, const void* X, const void* dY, const void* W,
                    void* dX, float* dW, vcas_stream stream);

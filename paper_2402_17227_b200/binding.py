@@ -22,7 +22,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
 
 EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
-           "vcas_linear_bwd_ex", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
+           "vcas_linear_bwd_ex", "vcas_linear_bwd_chain", "vcas_chain_parts", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
            "vcas_set_profiling", "vcas_stage_times", "vcas_score_static", "vcas_set_tuning",
            "vcas_version"]
@@ -47,6 +47,12 @@ class Config(C.Structure):
 class State(C.Structure):
     _fields_ = [("s", C.c_float), ("t", C.c_int32), ("L", C.c_int32),
                 ("rho", C.POINTER(C.c_float)), ("nu", C.POINTER(C.c_float))]
+
+
+class ChainArgs(C.Structure):
+    _fields_ = [("H", C.c_void_p), ("a_in", C.c_void_p), ("a_in_parts", C.c_int32), ("alive_in", C.c_void_p),
+                ("alive_cnt_in", C.c_void_p), ("a_out", C.c_void_p), ("kept_out", C.c_void_p),
+                ("kept_cnt_out", C.c_void_p)]
 
 
 _lib = None
@@ -142,6 +148,23 @@ class Layer:
                                       _stream())
         _check(rc, "vcas_linear_bwd_ex")
         return dX, dW
+
+    def linear_bwd_chain(self, X, dY, W, rho: float, nu: float, seed: int, dX, dW, *, H=None, a_in=None,
+                         a_in_parts: int = 1, alive_in=None, alive_cnt_in=None, a_out=None, kept_out=None,
+                         kept_cnt_out=None):
+        """vcas_linear_bwd_chain: scores handed down from the layer above (a_in, alive_in) and to the layer
+        below (a_out, kept_out); every extra is an optional device tensor."""
+        dp = lambda t: None if t is None else t.data_ptr()
+        args = ChainArgs(dp(H), dp(a_in), a_in_parts, dp(alive_in), dp(alive_cnt_in), dp(a_out), dp(kept_out),
+                         dp(kept_cnt_out))
+        _check(lib().vcas_linear_bwd_chain(self._h, _ptr(X), _ptr(dY), _ptr(W), C.c_float(rho), C.c_float(nu),
+                                           C.c_uint64(seed), C.byref(args), _ptr(dX), _ptr(dW), _stream()),
+               "vcas_linear_bwd_chain")
+
+    def chain_parts(self) -> int:
+        n = C.c_int32(0)
+        _check(lib().vcas_chain_parts(self._h, C.byref(n)), "vcas_chain_parts")
+        return n.value
 
     def linear_bwd_plain(self, X, dY, W, rho: float, nu: float, seed: int, dX, dW):
         """vcas_linear_bwd with caller-provided outputs (the call a training loop makes)."""

@@ -34,10 +34,10 @@ size_t layout(Handle* h, uint8_t* base) {
   const size_t N = d.N, R = (size_t)d.N * d.T, DW = (size_t)d.d_out * d.d_in;
   uint8_t* cur = base;
   Workspace& w = h->ws;
+  const size_t chunks = R / 32 + 2;
   w.a = carve<float>(cur, R);
-  w.b = carve<float>(cur, R);
-  w.lev = carve<float>(cur, R);
-  w.u24 = carve<uint32_t>(cur, R);
+  w.wc = carve<float>(cur, R);
+  w.uc = carve<uint32_t>(cur, R);
   w.g = carve<float>(cur, N);
   w.p = carve<float>(cur, N);
   w.w = carve<float>(cur, R);
@@ -48,9 +48,8 @@ size_t layout(Handle* h, uint8_t* base) {
   w.idxA = carve<int32_t>(cur, N);
   w.dropA = carve<int32_t>(cur, N);
   w.idxW = carve<int32_t>(cur, R);
-  w.scaleA2 = carve<float>(cur, N);
-  w.idxA2 = carve<int32_t>(cur, N);
-  w.dropA2 = carve<int32_t>(cur, N);
+  w.chunk_off = carve<int32_t>(cur, chunks);
+  w.fix = carve<float>(cur, 4);
   w.counts = carve<int32_t>(cur, 8);
   w.status = carve<int32_t>(cur, 1);
   w.acc = carve<double>(cur, 16);
@@ -75,6 +74,8 @@ size_t layout(Handle* h, uint8_t* base) {
   // second set (variance probe): see Handle::ws2
   Workspace& v = h->ws2;
   v = w;
+  v.wc = carve<float>(cur, R);
+  v.uc = carve<uint32_t>(cur, R);
   v.g = carve<float>(cur, N);
   v.p = carve<float>(cur, N);
   v.w = carve<float>(cur, R);
@@ -84,6 +85,8 @@ size_t layout(Handle* h, uint8_t* base) {
   v.idxA = carve<int32_t>(cur, N);
   v.dropA = carve<int32_t>(cur, N);
   v.idxW = carve<int32_t>(cur, R);
+  v.chunk_off = carve<int32_t>(cur, chunks);
+  v.fix = carve<float>(cur, 4);
   v.counts = carve<int32_t>(cur, 8);
   v.acc = carve<double>(cur, 16);
   v.partial = carve<double>(cur, PARTIAL_SLOTS);
@@ -114,12 +117,18 @@ int copy_out(Handle* h, float* g, float* p, float* w, float* q, int32_t* idxA, i
   return VCAS_OK;
 }
 
-// dW over the rows the sampler kept (idxW / scaleW / counts[1]) into `out`
-int sampled_dw(Handle* h, const void* X, const void* dY, float keep_hint, float* out, cudaStream_t st) {
+// SampleW, the kept-row list with its compact operands, and dW over those rows into `out`; follows SampleA
+// on the workspace set that h->ws currently names.  first_programmatic: the first kernel is launched as a
+// dependent of the kernel before it in `st` (false when its inputs arrive through an event).
+int sample_w_and_dw(Handle* h, const void* X, const void* dY, const SamplerArgs& a, bool first_programmatic,
+                    const Plan* plan, float* out, cudaStream_t st) {
+  VCAS_CUDA(launch_scores_x(h, X, a, first_programmatic, st));
+  VCAS_CUDA(launch_sample_w(h, a, st));
+  VCAS_CUDA(launch_emit_pack(h, dY, X, a, h->tensor_path, st));
   if (h->tensor_path) {
-    VCAS_CUDA(launch_pack(h, dY, X, st));
-    const int hint = (int)(keep_hint * (float)(h->desc.N * h->desc.T)) + 1;
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, nullptr, out, st));
+    const float keep = a.sample_w ? a.rho * a.nu : a.rho;
+    const int hint = (int)(keep * (float)(h->desc.N * h->desc.T)) + 1;
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, plan, out, st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, out, st));
   }
@@ -250,75 +259,91 @@ int vcas_launch_count(vcas_handle hh, uint64_t* launches) {
   return VCAS_OK;
 }
 
+namespace {
+// One sampled backward (Eq. 2).  `a` carries the ratios, the seed, the optional given probabilities and the
+// optional scores handed down from the layer above; a_out: optional row square-norms of dX for the layer below.
+int run_sampled(Handle* h, const void* X, const void* dY, const void* W, const SamplerArgs& a, const void* Hpre,
+                void* dX, float* dW, float* a_out, cudaStream_t st) {
+  const int hint = (int)(a.rho * a.nu * (float)(h->desc.N * h->desc.T)) + 1;
+  // The sampled dX grid leaves one SM free: SampleW's single-CTA kernel, which runs beside it on the side
+  // stream, needs a whole SM's shared memory.
+  const int spare = 1;
+  Plan px = {256, 1, 1}, pw = {256, 1, 1};
+  if (h->tensor_path) plan_products(h, false, a.rho, hint, spare, a_out != nullptr, &px, &pw);
+  if (!h->tensor_path || h->prof_enabled) {
+    // one stream, so that (with stage profiling) each pair of events brackets the kernels of one stage
+    mark(h, 0, st);
+    VCAS_CUDA(launch_rownorm_dy(h, dY, a, st));
+    mark(h, 1, st);
+    VCAS_CUDA(launch_sample_a(h, a, a.a_in == nullptr && !h->prof_enabled, st));
+    VCAS_CUDA(launch_scores_x(h, X, a, !h->prof_enabled, st));
+    VCAS_CUDA(launch_sample_w(h, a, st));
+    mark(h, 2, st);
+    if (h->tensor_path) {
+      VCAS_CUDA(launch_umma_dx(h, dY, W, false, a.rho, Hpre, dX, a_out, spare, &px, st));
+    } else {
+      VCAS_CUDA(launch_fma_dx(h, dY, W, h->ws.scaleA, Hpre, dX, st));
+      if (a_out != nullptr) VCAS_CUDA(launch_rownorm_out(h, dX, a_out, st));
+    }
+    mark(h, 3, st);
+    mark(h, 6, st);
+    VCAS_CUDA(launch_emit_pack(h, dY, X, a, h->tensor_path, st));
+    mark(h, 4, st);
+    if (h->tensor_path) {
+      VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, &pw, dW, st));
+    } else {
+      VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, dW, st));
+    }
+    mark(h, 5, st);
+  } else {
+    // The dX product needs SampleA only: on `st`, the row norms of dY, SampleA and the dX product follow one
+    // another as programmatic dependent launches.  Everything SampleW needs (the norms of the kept rows of X,
+    // the water-filling, the kept-row list and the compact operands) and the dW product run beside the dX
+    // product on the handle's side stream and are joined back before the call's work ends on `st`.
+    VCAS_CUDA(launch_rownorm_dy(h, dY, a, st));
+    VCAS_CUDA(launch_sample_a(h, a, a.a_in == nullptr, st));
+    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
+    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, a.rho, Hpre, dX, a_out, spare, &px, st));
+    const int rc = sample_w_and_dw(h, X, dY, a, false, &pw, dW, h->side_stream);
+    if (rc != VCAS_OK) return rc;
+    VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
+    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
+  }
+  if (h->prof_enabled && h->prof_calls < PROF_RING) h->prof_calls += 1;
+  return VCAS_OK;
+}
+}  // namespace
+
 int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void* W, float rho, float nu,
                        uint64_t seed, const float* p_in, const float* q_in, const void* Hpre, void* dX, float* dW,
                        vcas_stream stream) {
   if (hh == nullptr || X == nullptr || dY == nullptr || W == nullptr || dX == nullptr || dW == nullptr)
     return VCAS_ERR_BAD_ARG;
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
-  Handle* h = H(hh);
-  cudaStream_t st = S(stream);
-  SamplerArgs a;
-  a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = p_in; a.q_in = q_in; a.sample_w = 1; a.accumulate_vw = 0;
-  const int hint = (int)(rho * nu * (float)(h->desc.N * h->desc.T)) + 1;
-  const bool early_dx = fast_sampling(h->desc);     // dX forks right after the row norms
-  Plan px = {256, 1, 1}, pw = {256, 1, 1};
-  if (h->tensor_path) plan_products(h, false, rho, hint, early_dx ? 1 : 0, &px, &pw);
-  if (!h->tensor_path) {
-    mark(h, 0, st);
-    VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
-    mark(h, 1, st);
-    VCAS_CUDA(launch_sampler(h, a, st));
-    mark(h, 2, st);
-    VCAS_CUDA(launch_fma_dx(h, dY, W, h->ws.scaleA, Hpre, dX, st));
-    mark(h, 3, st);
-    mark(h, 6, st);
-    mark(h, 4, st);
-    VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, dW, st));
-    mark(h, 5, st);
-  } else if (h->prof_enabled) {
-    // stage profiling: everything on `st`, so that each pair of events brackets one kernel
-    mark(h, 0, st);
-    VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
-    mark(h, 1, st);
-    VCAS_CUDA(launch_sampler(h, a, st));
-    mark(h, 2, st);
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, early_dx ? 1 : 0, false, &px, st));
-    mark(h, 3, st);
-    mark(h, 6, st);
-    VCAS_CUDA(launch_pack(h, dY, X, st));
-    mark(h, 4, st);
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, &pw, dW, st));
-    mark(h, 5, st);
-  } else if (early_dx) {
-    // The dX product needs SampleA only.  On `st`, a small SampleA-only kernel and the dX product follow the
-    // row norms as programmatic dependent launches; the full sampling kernel (which draws the same SampleA
-    // masks, then SampleW), the pack and the dW product run beside them on the handle's side stream and are
-    // joined back before the call's work ends on `st`.  The dX grid leaves one SM free: the sampling kernel
-    // is a single CTA that needs a whole SM's registers.
-    VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
-    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
-    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-    VCAS_CUDA(launch_sampler(h, a, h->side_stream, true));
-    VCAS_CUDA(launch_sample_a(h, a, st));
-    VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 1, true, &px, st));
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, &pw, dW, h->side_stream));
-    VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
-    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
-  } else {
-    // large layers (generic sampling kernel): the products fork once the sampler has run
-    VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
-    VCAS_CUDA(launch_sampler(h, a, st));
-    VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
-    VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, rho, Hpre, dX, 0, false, &px, st));
-    VCAS_CUDA(launch_pack(h, dY, X, h->side_stream));
-    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, &pw, dW, h->side_stream));
-    VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
-    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
-  }
-  if (h->prof_enabled && h->prof_calls < PROF_RING) h->prof_calls += 1;
+  SamplerArgs a = sampler_args(rho, nu, seed);
+  a.p_in = p_in; a.q_in = q_in;
+  return run_sampled(H(hh), X, dY, W, a, Hpre, dX, dW, nullptr, S(stream));
+}
+
+int vcas_linear_bwd_chain(vcas_handle hh, const void* X, const void* dY, const void* W, float rho, float nu,
+                          uint64_t seed, const vcas_chain_args* c, void* dX, float* dW, vcas_stream stream) {
+  if (hh == nullptr || X == nullptr || dY == nullptr || W == nullptr || dX == nullptr || dW == nullptr || c == nullptr)
+    return VCAS_ERR_BAD_ARG;
+  if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
+  if ((c->alive_in == nullptr) != (c->alive_cnt_in == nullptr)) return VCAS_ERR_BAD_ARG;
+  if ((c->kept_out == nullptr) != (c->kept_cnt_out == nullptr)) return VCAS_ERR_BAD_ARG;
+  if (c->a_in != nullptr && c->a_in_parts < 1) return VCAS_ERR_BAD_ARG;
+  SamplerArgs a = sampler_args(rho, nu, seed);
+  a.a_in = c->a_in; a.a_parts = c->a_in != nullptr ? c->a_in_parts : 1;
+  a.alive = c->alive_in; a.alive_cnt = c->alive_cnt_in;
+  a.kept_out = c->kept_out; a.kept_cnt_out = c->kept_cnt_out;
+  return run_sampled(H(hh), X, dY, W, a, c->H, dX, dW, c->a_out, S(stream));
+}
+
+int vcas_chain_parts(vcas_handle hh, int32_t* parts) {
+  if (hh == nullptr || parts == nullptr) return VCAS_ERR_BAD_ARG;
+  *parts = a_out_parts(H(hh)->desc.d_in);
   return VCAS_OK;
 }
 
@@ -341,10 +366,10 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
     sw = h->side_stream;
   }
   Plan px = {256, 1, 1}, pw = {256, 1, 1};
-  if (h->tensor_path) plan_products(h, true, 1.0f, h->desc.N * h->desc.T, 0, &px, &pw);
+  if (h->tensor_path) plan_products(h, true, 1.0f, h->desc.N * h->desc.T, 0, false, &px, &pw);
   mark_dense(h, 0, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, 0, false, &px, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, nullptr, 0, &px, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }
@@ -367,10 +392,12 @@ int vcas_score(vcas_handle hh, const void* X, const void* dY, float rho, float n
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
-  SamplerArgs a;
-  a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 1; a.accumulate_vw = 0;
-  VCAS_CUDA(launch_rownorms(h, dY, X, seed, st));
-  VCAS_CUDA(launch_sampler(h, a, st));
+  const SamplerArgs a = sampler_args(rho, nu, seed);
+  VCAS_CUDA(launch_rownorm_dy(h, dY, a, st));
+  VCAS_CUDA(launch_sample_a(h, a, true, st));
+  VCAS_CUDA(launch_scores_x(h, X, a, true, st));
+  VCAS_CUDA(launch_sample_w(h, a, st));
+  VCAS_CUDA(launch_emit_pack(h, dY, X, a, false, st));
   return copy_out(h, g, p, w, q, idxA, cntA, idxW, cntW, st);
 }
 
@@ -406,10 +433,14 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
     int rc = dense_dw(h, X_i[i], dY_i[i], nullptr, h->ws.Gs, st);   // G_s,i
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(launch_probe_welford(h, i, st));
-    VCAS_CUDA(launch_rownorms(h, dY_i[i], X_i[i], 0, st));   // the probe draws no SampleW mask
-    // The M draws of SampleA for this batch are independent chains (sampler, pack, product, squared
-    // difference): even draws run on `st` with the first workspace set, odd draws on the side stream with
-    // the second, so that the latency-bound kernels of one chain overlap the product of the other.
+    SamplerArgs a = sampler_args(rho, nu, 0);
+    a.sample_w = 0;          // the probe draws no SampleW mask: G_act keeps every row of the kept data,
+    a.accumulate_vw = 1;     // and Eq. 3 is accumulated analytically at ratio nu
+    VCAS_CUDA(launch_rownorm_dy(h, dY_i[i], a, st));
+    // The M draws of SampleA for this batch are independent chains (SampleA, scores, SampleW's probabilities,
+    // kept rows, product, squared difference): even draws run on `st` with the first workspace set, odd draws
+    // on the side stream with the second, so that the latency-bound kernels of one chain overlap the product
+    // of the other.
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
     const Workspace first = h->ws;
@@ -417,12 +448,11 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
       const bool second = (j & 1) != 0;
       cudaStream_t sj = second ? h->side_stream : st;
       h->ws = second ? h->ws2 : first;
-      SamplerArgs a;
-      a.rho = rho; a.nu = nu; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 0; a.accumulate_vw = 1;
+      h->ws.a = first.a;
       a.seed = seed + (uint64_t)(i * M + j + 1) * 0x9E3779B97F4A7C15ull;
-      cudaError_t e = launch_sampler(h, a, sj, second);
+      cudaError_t e = launch_sample_a(h, a, !second, sj);
       if (e == cudaSuccess && j == 0) e = launch_probe_sparsity(h, s_lo, s_hi, sj);
-      if (e == cudaSuccess) rc = sampled_dw(h, X_i[i], dY_i[i], rho, h->ws.Gact, sj);   // G_act,ij (SampleA only)
+      if (e == cudaSuccess) rc = sample_w_and_dw(h, X_i[i], dY_i[i], a, true, nullptr, h->ws.Gact, sj);   // G_act,ij
       if (e == cudaSuccess && rc == VCAS_OK) e = launch_probe_sqdiff(h, sj);
       h->ws = first;
       if (e != cudaSuccess) return VCAS_ERR_CUDA;

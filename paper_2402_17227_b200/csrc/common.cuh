@@ -14,25 +14,23 @@ namespace vcas {
 // ---------------------------------------------------------------------------------------
 struct Workspace {
   // scores (Sec. 4.1, 4.2)
-  float* a;        // [R]  ||dY_r||^2
-  float* b;        // [R]  ||X_r||^2
-  float* lev;      // [R]  ||dY_r|| ||X_r||
-  uint32_t* u24;   // [R]  SampleW's 24-bit uniform of each row
+  float* a;        // [R]  ||dY_r||^2 (rows of data that may be non-zero)
+  float* wc;       // [R]  leverage scores ||G_hat_r|| ||X_r|| of the rows of kept data, compact: entry k*T + t is
+                   //      token t of the k-th kept datum
+  uint32_t* uc;    // [R]  SampleW's 24-bit uniform of those rows, same order
   float* g;        // [N]  ||G_n||_F
   float* p;        // [N]  SampleA keep probabilities
-  float* w;        // [R]  leverage scores of G_hat
-  float* q;        // [R]  SampleW keep probabilities
+  float* w;        // [R]  leverage scores by global row (0 on rows of dropped data)
+  float* q;        // [R]  SampleW keep probabilities by global row
   float* scaleA;   // [N]  1/p_n for kept data, 0 for dropped data
   float* scaleW;   // [R]  1/(p_n q_r) per compacted row
   float* sorted;   // [N]  data norms in descending order (Eq. 4)
   int32_t* idxA;   // [N]  kept data, ascending
   int32_t* dropA;  // [N]  dropped data, ascending
   int32_t* idxW;   // [R]  kept rows, ascending
-  // second set of SampleA results (launch_sample_a), read by a dX product that runs beside the sampling kernel
-  float* scaleA2;  // [N]
-  int32_t* idxA2;  // [N]
-  int32_t* dropA2; // [N]
-  int32_t* counts; // [8]  0: cntA, 1: cntW, 2: R (constant, for dense launches), 4: reduction ticket, 6: cntA of the second SampleA set
+  int32_t* chunk_off;  // [R/32 + 2] position in idxW of the first kept row of every chunk of 32 compact rows
+  float* fix;      // [4]  0: the factor c of q = min(1, c w) found by the water-filling, 1: mode (see sample_w_kernel)
+  int32_t* counts; // [8]  0: cntA, 1: cntW, 2: R (constant, for dense launches), 4: reduction ticket
   int32_t* status; // [1]  device status word
   double* acc;     // [16] probe accumulators (0: V_act, 1: V_w, 2: p_lo, 3: p_hi, 4: V_s)
   double* partial; // [PARTIAL_SLOTS] block partial sums of the probe reductions
@@ -240,7 +238,7 @@ __device__ __forceinline__ void capped_prop_warp(float (&v)[SLOTS], float budget
 // Where SampleA's results go: the workspace arrays, and optionally shared-memory copies of p and 1/p.
 struct SampleAOut {
   float* p; float* scaleA; int32_t* idxA; int32_t* dropA;
-  float* sh_p; float* sh_scaleA;
+  int32_t* idx_copy;   // optional second copy of the kept list (handed to the next layer of a chain)
 };
 
 // SampleA over N <= 32 * SLOTS data by one full warp: keep probabilities from the data norms g (or the
@@ -269,11 +267,15 @@ __device__ __forceinline__ int sample_a_warp(const float* g, int N, float rho, c
     const unsigned lower = (1u << lane) - 1u;
     if (in) {
       const float sc = keep ? 1.0f / v[j] : 0.f;
-      if (o.p != nullptr) o.p[n] = v[j];
+      o.p[n] = v[j];
       o.scaleA[n] = sc;
-      if (o.sh_p != nullptr) { o.sh_p[n] = v[j]; o.sh_scaleA[n] = sc; }
-      if (keep) o.idxA[kept_before + __popc(bk & lower)] = n;
-      else o.dropA[drop_before + __popc(bd & lower)] = n;
+      if (keep) {
+        const int pos = kept_before + __popc(bk & lower);
+        o.idxA[pos] = n;
+        if (o.idx_copy != nullptr) o.idx_copy[pos] = n;
+      } else {
+        o.dropA[drop_before + __popc(bd & lower)] = n;
+      }
     }
     kept_before += __popc(bk);
     drop_before += __popc(bd);
@@ -281,13 +283,9 @@ __device__ __forceinline__ int sample_a_warp(const float* g, int N, float rho, c
   return kept_before;
 }
 
-// The single-CTA register-resident sampling kernel, and with it the SampleA-only kernel that lets the dX
-// product start early, serve layers of at most this many data and rows.
-constexpr int FAST_MAX_N = 1024;
-constexpr int FAST_MAX_R = 16 * 1024;
-inline bool fast_sampling(const vcas_layer_desc& d) {
-  return d.N <= FAST_MAX_N && (long long)d.N * d.T <= FAST_MAX_R;
-}
+// SampleA runs inside one warp for up to this many data (32 lanes x 32 slots); larger batches take a
+// block-wide kernel.
+constexpr int WARP_MAX_N = 1024;
 
 // ---------------------------------------------------------------------------------------
 // Launchers (one per .cu file).  All enqueue on `st` and return a cudaError_t.
@@ -299,15 +297,33 @@ struct SamplerArgs {
   const float* q_in;
   int sample_w;      // 1: SampleW mask applied; 0: all rows of kept data survive (probe)
   int accumulate_vw; // 1: add Eq. 3 at ratio nu to acc[1]
+  // Scoring handed down a stack of layers (the gradient gets sparser from layer to layer, Sec. 4):
+  const float* a_in;        // row square-norms of dY made by its producer, a_r = sum of a_parts consecutive floats
+  int a_parts;              // (nullptr: computed here from dY, one float per row)
+  const int32_t* alive;     // data whose rows of dY may be non-zero (device list, ascending) and its length;
+  const int32_t* alive_cnt; // every other datum is known to be zero and is never read (nullptr: all N data)
+  int32_t* kept_out;        // optional copies of this call's kept-data list and count (device)
+  int32_t* kept_cnt_out;
 };
-// seed: the call's seed (the SampleW uniforms are drawn here, one per row)
-cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, cudaStream_t st);
-// SampleA alone (rho, p_in and seed of `a`), into the workspace's second set of SampleA arrays (idxA2, dropA2,
-// scaleA2, counts[6]): what the dX product needs, so that it can start while the full sampling kernel,
-// which draws the same masks, runs beside it on another stream.  Requires fast_sampling(desc).
-cudaError_t launch_sample_a(Handle* h, const SamplerArgs& a, cudaStream_t st);
-// after_event: launched plainly (its inputs come through an event from another stream)
-cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st, bool after_event = false);
+inline SamplerArgs sampler_args(float rho, float nu, uint64_t seed) {
+  SamplerArgs a = {};
+  a.rho = rho; a.nu = nu; a.seed = seed; a.sample_w = 1; a.a_parts = 1;
+  return a;
+}
+// a_r = ||dY_r||^2 on the rows of alive data (nothing to do when the producer supplied them)
+cudaError_t launch_rownorm_dy(Handle* h, const void* dY, const SamplerArgs& a, cudaStream_t st);
+// row square-norms of a finished dX in the layout of the product kernels' partial sums (a_out_parts floats per
+// row), for the products that do not emit them from their epilogue
+cudaError_t launch_rownorm_out(Handle* h, const void* dX, float* a_out, cudaStream_t st);
+// SampleA (Sec. 4.1): g, p, mask, kept / dropped lists, 1/p; programmatic: launched as a dependent of the
+// kernel before it in the stream
+cudaError_t launch_sample_a(Handle* h, const SamplerArgs& a, bool programmatic, cudaStream_t st);
+// ||X_r|| on the rows of kept data, the leverage scores of G_hat and SampleW's uniforms, in compact order
+cudaError_t launch_scores_x(Handle* h, const void* X, const SamplerArgs& a, bool programmatic, cudaStream_t st);
+// SampleW (Sec. 4.2): the factor c of q = min(1, c w), the masks' counts per chunk of 32 compact rows
+cudaError_t launch_sample_w(Handle* h, const SamplerArgs& a, cudaStream_t st);
+// kept-row list, 1/(p q), q and w by global row and, with pack, the compact bf16 operands of the dW product
+cudaError_t launch_emit_pack(Handle* h, const void* dY, const void* X, const SamplerArgs& a, bool pack, cudaStream_t st);
 cudaError_t launch_mask_from_probs(Handle* h, const float* p, int n, uint64_t seed, int sampler,
                                    uint8_t* keep, int32_t* idx, int32_t* cnt, cudaStream_t st);
 
@@ -319,19 +335,21 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 
 // tensor-core products
 // spare_sms: SMs the persistent grid leaves free (for a kernel of another stream that must run beside it);
-// second_set: kept / dropped data and scales from the second set of SampleA arrays (launch_sample_a);
 // pair_plan: the tiling chosen by plan_products for a call whose two products run at the same time
 // (nullptr: chosen here, for this product alone)
+// a_out: optional [R][a_out_parts(d_in)] partial row square-norms of the stored dX, written by the epilogue
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, int spare_sms, bool second_set, const Plan* pair_plan, cudaStream_t st);
-cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st);
+                           const void* H, void* dX, float* a_out, int spare_sms, const Plan* pair_plan, cudaStream_t st);
+inline int a_out_parts(int d_in) { return (d_in + 255) / 256; }
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity,
                            const int32_t* cnt, int cnt_hint, const Plan* pair_plan, float* dW, cudaStream_t st);
 // Tilings of the dX and dW products of one call, chosen together because they share the SMs (cached in the
 // handle until the expected kept counts or the tuning overrides change).
-void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spare_sms, Plan* dx, Plan* dw);
+// row_norms_out: the dX product must emit row square-norms from its epilogue (unsliced 256-wide tiles only)
+void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spare_sms, bool row_norms_out, Plan* dx,
+                   Plan* dw);
 
 // probe reductions
 cudaError_t launch_probe_reset(Handle* h, cudaStream_t st);

@@ -276,6 +276,8 @@ struct GemmParams {
   const float* scaleA;     // 1/p_n per datum
   const __nv_bfloat16* H;  // optional GELU pre-activation [R, d_in]
   __nv_bfloat16* dX;       // [R, d_in]
+  float* a_out;            // optional [R][a_parts]: square-norm of the stored row of dX, one partial sum per 256-column
+  int a_parts;             // tile (unsliced 256-wide tiles only); the layer below adds the partials in order
   int N, T;
   int dense;               // 1: every datum kept with scale 1
   int a_tx_bytes;          // bytes one A box delivers (min(T, 128) token rows of 128 B)
@@ -604,6 +606,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
           for (int j = 0; j < BN / 8; ++j)
             if (col0 + j * 8 < P.d_in) *reinterpret_cast<uint4*>(P.dX + off + j * 8) = make_uint4(0u, 0u, 0u, 0u);
+          if (P.a_out != nullptr) P.a_out[(row0 + hrow) * P.a_parts + col0 / 256] = 0.f;
         } else {
 #pragma unroll
           for (int j = 0; j < BN / 4; ++j)
@@ -674,6 +677,9 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // tensor are clipped by the tensor map, so rows of the next datum are never touched)
         constexpr int COLS = MODE == MODE_DX ? 64 : 32;             // columns per 128-byte staged row
         int nbuf = 0;
+        float rowsq[MH];                                            // square-norm of this thread's row(s), as stored
+#pragma unroll
+        for (int hh = 0; hh < MH; ++hh) rowsq[hh] = 0.f;
 #pragma unroll 1
         for (int hj = 0; hj < MH * (BN / COLS); ++hj, ++nbuf) {
           const int hh = hj / (BN / COLS), j = hj % (BN / COLS);    // 128-row half of the tile, column chunk
@@ -708,6 +714,19 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 o.x = pack_bf16(r[0], r[1]); o.y = pack_bf16(r[2], r[3]);
                 o.z = pack_bf16(r[4], r[5]); o.w = pack_bf16(r[6], r[7]);
                 myrow[(uint32_t)(half * 4 + g8) ^ swz] = o;
+                if (P.a_out != nullptr) {
+                  const uint32_t ou[4] = {o.x, o.y, o.z, o.w};
+                  float sq = 0.f;
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    const float lo = __uint_as_float(ou[e] << 16), hi = __uint_as_float(ou[e] & 0xffff0000u);
+                    sq = fmaf(lo, lo, sq);
+                    sq = fmaf(hi, hi, sq);
+                  }
+#pragma unroll
+                  for (int h2 = 0; h2 < MH; ++h2)
+                    if (h2 == hh) rowsq[h2] += sq;
+                }
               }
             }
           } else {
@@ -727,6 +746,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         tc_fence_before();
         mbar_arrive(&s.tmem_empty[buf]);
+        if (MODE == MODE_DX && P.a_out != nullptr) {
+#pragma unroll
+          for (int hh = 0; hh < MH; ++hh)
+            if (hh * BM + row < rows_valid) P.a_out[(row0 + hh * BM + row) * P.a_parts + col0 / 256] = rowsq[hh];
+        }
         if (lane == 0) bulk_wait_all();        // staging buffers are reused by the next unit
         __syncwarp();
         continue;
@@ -804,44 +828,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
-}
-
-// ---------------------------------------------------------------------------- pack kernel
-// Compact operands of the weight-gradient product: row k of packG = scaleW[k] * dY[idxW[k]]
-// (G_tilde of Sec. 4.2, rounded to bf16), row k of packX = X[idxW[k]]; rows up to the next
-// multiple of 64 are zero so that the last k-block of the product contributes nothing.
-__global__ void __launch_bounds__(256) pack_kernel(const __nv_bfloat16* __restrict__ dY, const __nv_bfloat16* __restrict__ X,
-                                                   const int32_t* __restrict__ idxW, const float* __restrict__ scaleW,
-                                                   const int32_t* __restrict__ counts, __nv_bfloat16* __restrict__ packG,
-                                                   __nv_bfloat16* __restrict__ packX, int d_out, int d_in) {
-  pdl_wait();      // the kept rows come from the sampling kernel before this one
-  pdl_trigger();   // the dW product kernel may set itself up; it waits for this grid before loading
-  const int cnt = counts[1];
-  const int padded = (cnt + BK - 1) / BK * BK;
-  const int vo = d_out / 8, vi = d_in / 8;
-  for (int k = blockIdx.x; k < padded; k += gridDim.x) {
-    uint4* og = reinterpret_cast<uint4*>(packG + (size_t)k * d_out);
-    uint4* ox = reinterpret_cast<uint4*>(packX + (size_t)k * d_in);
-    if (k < cnt) {
-      const int r = idxW[k];
-      const float sc = scaleW[k];
-      const uint4* ig = reinterpret_cast<const uint4*>(dY + (size_t)r * d_out);
-      const uint4* ix = reinterpret_cast<const uint4*>(X + (size_t)r * d_in);
-      for (int i = threadIdx.x; i < vo; i += blockDim.x) {
-        const uint4 v = __ldg(ig + i);
-        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-        uint32_t o[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          o[e] = pack_bf16(sc * __uint_as_float(u[e] << 16), sc * __uint_as_float(u[e] & 0xffff0000u));
-        og[i] = make_uint4(o[0], o[1], o[2], o[3]);
-      }
-      for (int i = threadIdx.x; i < vi; i += blockDim.x) ox[i] = __ldg(ix + i);
-    } else {
-      for (int i = threadIdx.x; i < vo; i += blockDim.x) og[i] = make_uint4(0u, 0u, 0u, 0u);
-      for (int i = threadIdx.x; i < vi; i += blockDim.x) ox[i] = make_uint4(0u, 0u, 0u, 0u);
-    }
-  }
 }
 
 // ------------------------------------------------------------------------------ host side
@@ -1076,19 +1062,23 @@ bool dw_remainder_ok(const Handle* h) {
 }
 }  // namespace
 
-void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spare_sms, Plan* dx, Plan* dw) {
+void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spare_sms, bool row_norms_out, Plan* dx,
+                   Plan* dw) {
   const vcas_layer_desc& d = h->desc;
   const DxShape g = dx_shape(h, dense, rho_hint);
   const int kb_w = (cnt_hint + BK - 1) / BK;
-  const int key[PLAN_KEY_INTS] = {dense ? 1 : 0, (int)g.row_tiles128, kb_w, spare_sms, h->tune_dx_tile_n,
-                                  h->tune_dw_tile_n, h->tune_dx_split_k, h->tune_dw_split_k, h->tune_tile_m};
+  const int key[PLAN_KEY_INTS] = {(dense ? 1 : 0) | (row_norms_out ? 2 : 0), (int)g.row_tiles128, kb_w, spare_sms,
+                                  h->tune_dx_tile_n, h->tune_dw_tile_n, h->tune_dx_split_k, h->tune_dw_split_k,
+                                  h->tune_tile_m};
   bool hit = h->plan_valid;
   for (int i = 0; i < PLAN_KEY_INTS && hit; ++i) hit = h->plan_key[i] == key[i];
   if (!hit) {
     const int ctas = h->num_sms - spare_sms > 1 ? h->num_sms - spare_sms : 1;
     Cand cx[MAX_CANDS], cw[MAX_CANDS];
+    // the epilogue emits row square-norms of dX only from unsliced 256-wide tiles (one partial sum per tile)
     const int nx = enumerate_plans(g.row_tiles128, g.row_tiles256, d.d_in, g.kblocks, ctas, h->max_units,
-                                   h->tune_dx_tile_n, h->tune_dx_split_k, g.rem_ok, cx);
+                                   row_norms_out ? 256 : h->tune_dx_tile_n, row_norms_out ? 1 : h->tune_dx_split_k,
+                                   g.rem_ok && !row_norms_out, cx);
     const bool rem_w = dw_remainder_ok(h);
     const int nw = enumerate_plans((d.d_out + BM - 1) / BM, (d.d_out + 2 * BM - 1) / (2 * BM), d.d_in, kb_w, h->num_sms,
                                    h->max_units, h->tune_dw_tile_n, h->tune_dw_split_k, rem_w, cw);
@@ -1098,7 +1088,7 @@ void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spar
     const double offset = dense ? 0.0 : 10.5;
     Plan px, pw;
     best_pair(cx, nx, ctas, cw, nw, h->num_sms, h->num_sms, offset, &px, &pw);
-    h->plan_dx = apply_tile_m(h, px, g.rem_ok);
+    h->plan_dx = apply_tile_m(h, px, g.rem_ok && !row_norms_out);
     h->plan_dw = apply_tile_m(h, pw, rem_w);
     for (int i = 0; i < PLAN_KEY_INTS; ++i) h->plan_key[i] = key[i];
     h->plan_valid = true;
@@ -1108,7 +1098,7 @@ void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spar
 }
 
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint, const void* H,
-                           void* dX, int spare_sms, bool second_set, const Plan* pair_plan, cudaStream_t st) {
+                           void* dX, float* a_out, int spare_sms, const Plan* pair_plan, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -1132,7 +1122,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   GemmParams P;
   common_params(h, P, 0);
   P.idxA = h->ws.idxA; P.dropA = h->ws.dropA; P.counts = h->ws.counts; P.scaleA = h->ws.scaleA;
-  if (second_set) { P.idxA = h->ws.idxA2; P.dropA = h->ws.dropA2; P.counts = h->ws.counts + 6; P.scaleA = h->ws.scaleA2; }
+  P.a_out = a_out; P.a_parts = a_out_parts(d.d_in);
   P.H = (const __nv_bfloat16*)H; P.dX = (__nv_bfloat16*)dX;
   P.N = d.N; P.T = d.T; P.dense = dense ? 1 : 0;
   P.a_tx_bytes = (d.T < BM ? d.T : BM) * BK * 2;
@@ -1144,25 +1134,15 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   } else {
     DxShape g = dx_shape(h, dense, rho_hint);
     Cand cands[MAX_CANDS];
+    const bool rn = a_out != nullptr;
     const int n = enumerate_plans(g.row_tiles128, g.row_tiles256, d.d_in, g.kblocks, ctas, h->max_units,
-                                  h->tune_dx_tile_n, h->tune_dx_split_k, g.rem_ok, cands);
-    plan = apply_tile_m(h, best_alone(cands, n), g.rem_ok);
+                                  rn ? 256 : h->tune_dx_tile_n, rn ? 1 : h->tune_dx_split_k, g.rem_ok && !rn, cands);
+    plan = apply_tile_m(h, best_alone(cands, n), g.rem_ok && !rn);
   }
   P.split_k = plan.split;
   // upper bound of work items: every datum kept and split, or every datum a zero tile
   const long max_items = (long)d.N * (plan.mh >= 2 ? chunks2 : chunks) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
   return run_gemm_bn<MODE_DX>(h, plan, tmA, tmB, tmC, P, max_items, ctas, true, st);
-}
-
-cudaError_t launch_pack(Handle* h, const void* dY, const void* X, cudaStream_t st) {
-  const vcas_layer_desc& d = h->desc;
-  int blocks = h->num_sms * 8;
-  if (blocks > h->R_pad) blocks = h->R_pad;
-  const cudaError_t e = launch_after(pack_kernel, dim3(blocks), dim3(256), 0, st, (const __nv_bfloat16*)dY,
-                                     (const __nv_bfloat16*)X, h->ws.idxW, h->ws.scaleW, h->ws.counts, h->ws.packG,
-                                     h->ws.packX, d.d_out, d.d_in);
-  h->launches += 1;
-  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity, const int32_t* cnt,

@@ -1,14 +1,21 @@
 // Keep probabilities, Philox Bernoulli masks and compaction for SampleA and SampleW
-// (Sec. 4.1, 4.2).  The arrays involved are tiny (N and R = N*T floats), so the whole stage is
-// one CTA: latency-bound, not bandwidth-bound.  Everything stays on the device: the kept
-// counts are written to the workspace and read by the product kernels.
+// (Sec. 4.1, 4.2).  Everything stays on the device: the kept counts are written to the workspace
+// and read by the product kernels.  The stage is a chain of small kernels:
+//   sample_a_kernel   one CTA: ||G_n||_F, p_n, mask, kept / dropped data (the dX product can start here);
+//   scores_x_kernel   (score.cu) many CTAs: leverage scores and uniforms of the rows of kept data;
+//   sample_w_kernel   one CTA, scores in shared memory: the water-filling for q = min(1, c w) - a handful
+//                     of block-wide sums - then the masks' counts per chunk of 32 rows and their prefix sums;
+//   emit_pack_kernel  many CTAs: kept-row list, 1/(p q), and the compact operands of the dW product.
+// Only the scalar fixed point and a scan over R/32 counts run on a single SM.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace vcas {
 namespace {
 
 constexpr int SAMPLER_THREADS = 1024;
-static_assert(FAST_MAX_N <= SAMPLER_THREADS && FAST_MAX_R == 16 * SAMPLER_THREADS, "fast sampling limits");
+constexpr int WATER_ROUNDS = 128;     // rounds of the water-filling before it is reported as not converged
 
 struct Scratch {
   double d[32];
@@ -41,8 +48,8 @@ __device__ void block_sum(double& s, int& c, Scratch* sc) {
 // Keep probabilities proportional to v, capped at 1, summing to `budget` (the minimiser of
 // sum (1-p)/p v^2 under that budget): p = min(1, c v).  The saturated set is grown from
 // empty; c only increases, so the iteration reaches the least fixed point, which is the
-// unique solution.
-__device__ void capped_prop_block(const float* v, int n, double budget, float* p, Scratch* sc) {
+// unique solution.  Returns false if it has not converged after WATER_ROUNDS rounds.
+__device__ bool capped_prop_block(const float* v, int n, double budget, float* p, Scratch* sc) {
   const int tid = threadIdx.x, nt = blockDim.x;
   double S = 0.0;
   int nz = 0;
@@ -53,15 +60,16 @@ __device__ void capped_prop_block(const float* v, int n, double budget, float* p
   block_sum(S, nz, sc);
   if (nz == 0 || budget <= 0.0) {
     for (int i = tid; i < n; i += nt) p[i] = 0.f;
-    return;
+    return true;
   }
   if ((double)nz <= budget) {
     for (int i = tid; i < n; i += nt) p[i] = v[i] > 0.f ? 1.f : 0.f;
-    return;
+    return true;
   }
   double c = budget / S;
   int k = 0;
-  for (int iter = 0; iter < 128; ++iter) {
+  bool converged = false;
+  for (int iter = 0; iter < WATER_ROUNDS; ++iter) {
     double Su = 0.0;
     int ks = 0;
     for (int i = tid; i < n; i += nt) {
@@ -71,7 +79,7 @@ __device__ void capped_prop_block(const float* v, int n, double budget, float* p
       }
     }
     block_sum(Su, ks, sc);
-    if (ks == k) break;
+    if (ks == k) { converged = true; break; }
     k = ks;
     if (Su > 0.0) {
       const double cn = (budget - (double)k) / Su;
@@ -87,6 +95,7 @@ __device__ void capped_prop_block(const float* v, int n, double budget, float* p
     }
     p[i] = r;
   }
+  return converged;
 }
 
 // Ordered compaction of the indices i < n with keep(i): emit(i, position).  Returns the count.
@@ -120,39 +129,72 @@ __device__ int block_compact(int n, KeepFn keep, EmitFn emit, Scratch* sc) {
   return base;
 }
 
-struct SamplerParams {
-  const float* a; const float* b;
-  const float* lev; const uint32_t* u24;   // per-row leverage ||dY_r|| ||X_r|| and SampleW uniform (row-norm kernel)
-  float* g; float* p; float* w; float* q;
-  float* scaleA; float* scaleW;
-  int32_t* idxA; int32_t* dropA; int32_t* idxW; int32_t* counts;
-  double* acc;
-  const float* p_in; const float* q_in;
+// ------------------------------------------------------------------------------ SampleA
+struct SampleAParams {
+  const float* a; int a_parts;
+  const int32_t* alive; const int32_t* alive_cnt;
   int N, T;
-  float rho, nu;
+  float rho;
+  const float* p_in;
   uint64_t seed;
-  int sample_w, accumulate_vw;
+  float* g; float* p; float* scaleA;
+  int32_t* idxA; int32_t* dropA; int32_t* counts;
+  int32_t* kept_out; int32_t* kept_cnt_out;
+  int32_t* status;
 };
 
-__global__ void __launch_bounds__(SAMPLER_THREADS) sampler_kernel(SamplerParams P) {
-  __shared__ Scratch sc;
+// SampleA (Sec. 4.1) for N <= 32 * SLOTS data: one warp per datum sums its T row square-norms (only the alive
+// data are read; the others have norm 0), then warp 0 finds p, draws the masks and writes the lists.
+constexpr int SAMPLE_A_THREADS = 512;
+template <int SLOTS>
+__global__ void __launch_bounds__(SAMPLE_A_THREADS) sample_a_kernel(SampleAParams P) {
+  __shared__ float s_g[32 * SLOTS];
   pdl_wait();      // the row norms come from the kernel before this one
-  pdl_trigger();   // the product kernel may set itself up meanwhile
-  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
-  const int N = P.N, T = P.T, R = N * T;
+  pdl_trigger();   // the dX product kernel may set itself up meanwhile
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int n = threadIdx.x; n < 32 * SLOTS; n += SAMPLE_A_THREADS) s_g[n] = 0.f;
+  __syncthreads();
+  const int nd = P.alive != nullptr ? *P.alive_cnt : P.N;
+  const int len = P.T * P.a_parts;
+  for (int k = warp; k < nd; k += SAMPLE_A_THREADS / 32) {
+    const int n = P.alive != nullptr ? P.alive[k] : k;
+    const float s = datum_sqnorm_warp(P.a + (size_t)n * len, len, lane);
+    if (lane == 0) s_g[n] = sqrtf(s);
+  }
+  __syncthreads();
+  for (int n = threadIdx.x; n < P.N; n += SAMPLE_A_THREADS) P.g[n] = s_g[n];
+  if (warp == 0) {
+    SampleAOut o;
+    o.p = P.p; o.scaleA = P.scaleA; o.idxA = P.idxA; o.dropA = P.dropA; o.idx_copy = P.kept_out;
+    const int kept = sample_a_warp<SLOTS>(s_g, P.N, P.rho, P.p_in, P.seed, o, lane);
+    if (lane == 0) {
+      P.counts[0] = kept;
+      if (P.kept_cnt_out != nullptr) *P.kept_cnt_out = kept;
+    }
+  }
+}
 
-  // ---- SampleA: ||G_n||_F, p_n, mask, kept / dropped data lists (Sec. 4.1)
-  for (int n = warp; n < N; n += nw) {
-    double s = 0.0;
-    for (int t = lane; t < T; t += 32) s += (double)P.a[(size_t)n * T + t];
-    s = warp_sum(s);
-    if (lane == 0) P.g[n] = (float)sqrt(s);
+// The same for batches of more than 1024 data: one CTA over global memory.
+__global__ void __launch_bounds__(SAMPLER_THREADS) sample_a_big_kernel(SampleAParams P) {
+  __shared__ Scratch sc;
+  pdl_wait();
+  pdl_trigger();
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+  const int N = P.N;
+  for (int n = tid; n < N; n += nt) P.g[n] = 0.f;
+  __syncthreads();
+  const int nd = P.alive != nullptr ? *P.alive_cnt : N;
+  const int len = P.T * P.a_parts;
+  for (int k = warp; k < nd; k += nw) {
+    const int n = P.alive != nullptr ? P.alive[k] : k;
+    const float s = datum_sqnorm_warp(P.a + (size_t)n * len, len, lane);
+    if (lane == 0) P.g[n] = sqrtf(s);
   }
   __syncthreads();
   if (P.p_in != nullptr) {
     for (int n = tid; n < N; n += nt) P.p[n] = P.p_in[n];
-  } else {
-    capped_prop_block(P.g, N, (double)N * (double)P.rho, P.p, &sc);
+  } else if (!capped_prop_block(P.g, N, (double)N * (double)P.rho, P.p, &sc)) {
+    if (tid == 0) atomicExch(P.status, (int32_t)VCAS_ERR_INTERNAL);
   }
   __syncthreads();
   for (int n = tid; n < N; n += nt) {
@@ -161,70 +203,61 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sampler_kernel(SamplerParams 
   }
   __syncthreads();
   const int cntA = block_compact(N, [&](int n) { return P.scaleA[n] > 0.f; },
-                                 [&](int n, int pos) { P.idxA[pos] = n; }, &sc);
-  block_compact(N, [&](int n) { return !(P.scaleA[n] > 0.f); },
-                [&](int n, int pos) { P.dropA[pos] = n; }, &sc);
-
-  // ---- SampleW: leverage scores of G_hat, q_r, mask, kept rows (Sec. 4.2, Eq. 3)
-  for (int r = tid; r < R; r += nt) {
-    const int n = r / T;
-    float wr = 0.f;
-    if (P.scaleA[n] > 0.f) wr = (float)(sqrt((double)P.a[r] * (double)P.b[r]) / (double)P.p[n]);
-    P.w[r] = wr;
+                                 [&](int n, int pos) { P.idxA[pos] = n; if (P.kept_out != nullptr) P.kept_out[pos] = n; },
+                                 &sc);
+  block_compact(N, [&](int n) { return !(P.scaleA[n] > 0.f); }, [&](int n, int pos) { P.dropA[pos] = n; }, &sc);
+  if (tid == 0) {
+    P.counts[0] = cntA;
+    if (P.kept_cnt_out != nullptr) *P.kept_cnt_out = cntA;
   }
-  __syncthreads();
-  if (P.q_in != nullptr) {
-    for (int r = tid; r < R; r += nt) P.q[r] = P.scaleA[r / T] > 0.f ? P.q_in[r] : 0.f;
-  } else {
-    capped_prop_block(P.w, R, (double)P.nu * (double)T * (double)cntA, P.q, &sc);
-  }
-  __syncthreads();
-  if (P.accumulate_vw) {
-    double vw = 0.0;
-    int dummy = 0;
-    for (int r = tid; r < R; r += nt) {
-      const double qr = (double)P.q[r];
-      if (qr > 0.0) {
-        const double wr = (double)P.w[r];
-        vw += (1.0 - qr) / qr * wr * wr;
-      }
-    }
-    block_sum(vw, dummy, &sc);
-    if (tid == 0) P.acc[1] += vw;
-  }
-  int cntW;
-  if (P.sample_w) {
-    cntW = block_compact(R,
-        [&](int r) { const float qr = P.q[r]; return qr > 0.f && bernoulli_keep(qr, P.seed, 1u, (uint64_t)r); },
-        [&](int r, int pos) { P.idxW[pos] = r; P.scaleW[pos] = P.scaleA[r / T] / P.q[r]; }, &sc);
-  } else {
-    cntW = block_compact(R, [&](int r) { return P.scaleA[r / T] > 0.f; },
-        [&](int r, int pos) { P.idxW[pos] = r; P.scaleW[pos] = P.scaleA[r / T]; }, &sc);
-  }
-  if (tid == 0) { P.counts[0] = cntA; P.counts[1] = cntW; }
 }
 
-// ---------------------------------------------------------------------------------------
-// Fast path for R <= 16 * 1024 rows and N <= 1024 data: every thread keeps its E consecutive
-// rows in registers, SampleA runs inside warp 0 with shuffles only, and each water-filling
-// iteration over the rows costs two block barriers.
-// ---------------------------------------------------------------------------------------
-struct FastShared {
+// ------------------------------------------------------------------------------ SampleW
+// How q follows from a row's score once sample_w_kernel has run: fix[1] = mode, fix[0] = c.
+constexpr int Q_ZERO = 0;     // nothing to keep (no score is positive, or the budget is 0)
+constexpr int Q_ONES = 1;     // the budget covers every positive score: q = [w > 0]
+constexpr int Q_CAPPED = 2;   // q = min(1, c w)
+constexpr int Q_GIVEN = 3;    // q is read from the caller's q_in
+
+__device__ __forceinline__ float q_of(int mode, float c, float w, const float* q_in, int r) {
+  if (mode == Q_CAPPED) {
+    if (!(w > 0.f)) return 0.f;
+    const float cx = c * w;
+    return cx >= 1.0f ? 1.f : cx;
+  }
+  if (mode == Q_ONES) return w > 0.f ? 1.f : 0.f;
+  if (mode == Q_GIVEN) return q_in[r];
+  return 0.f;
+}
+__device__ __forceinline__ bool row_kept(int sample_w, float q, uint32_t u) {
+  return sample_w ? (q > 0.f && u < (uint32_t)floorf(q * 16777216.0f)) : true;
+}
+
+struct SampleWParams {
+  const float* wc; const uint32_t* uc;     // compact scores and uniforms of the rows of kept data
+  const float* q_in;
+  const int32_t* idxA;
+  int32_t* counts; int32_t* chunk_off; float* fix;
+  double* acc; int32_t* status;
+  int T;
+  float nu;
+  int sample_w, accumulate_vw;
+  int smem_rows;                            // scores that fit the kernel's shared memory
+};
+
+struct WShared {
   float part_f[2][32];
   int part_i[2][32];
-  int warp_tot[32];
-  float scaleA[1024];
-  float pA[1024];
-  int cntA;
+  int scan[33];
 };
 
 // Block-wide sum of one float and one int in a fixed order (lanes by shuffle tree, then the 32
 // warp totals by the same tree, which every warp runs for itself so that one barrier suffices; the
 // buffers alternate with `parity`, and a buffer is rewritten only after a later barrier).  fp32 on
 // purpose: this is a single-CTA kernel, and double-precision arithmetic concentrated on one SM was
-// measured to dominate its run time; a tree sum of <= 16384 non-negative fp32 terms is accurate to
-// about 1e-6, inside the 1e-5 the probabilities are specified to.
-__device__ __forceinline__ void fast_sum(float& s, int& c, FastShared* sh, int parity) {
+// measured to dominate its run time; a tree sum of non-negative fp32 terms is accurate to about
+// 1e-6, inside the 2e-5 the probabilities are specified to.
+__device__ __forceinline__ void fast_sum(float& s, int& c, WShared* sh, int parity) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   s = warp_sum(s);
   c = __reduce_add_sync(0xffffffffu, c);
@@ -234,265 +267,240 @@ __device__ __forceinline__ void fast_sum(float& s, int& c, FastShared* sh, int p
   c = __reduce_add_sync(0xffffffffu, sh->part_i[parity][lane]);
 }
 
-template <int E, int SLOTS>
-__global__ void __launch_bounds__(SAMPLER_THREADS) sampler_fast_kernel(SamplerParams P) {
-  __shared__ FastShared sh;
-  pdl_wait();      // the row norms come from the kernel before this one
-  pdl_trigger();   // the product kernel may set itself up meanwhile
+// SampleW's single-CTA part (Sec. 4.2, Eq. 3).  The n = T * (#kept data) scores sit in shared memory (in
+// global memory beyond smem_rows: same code, slower loads).  1. c with sum_r min(1, c w_r) = nu * n by
+// water-filling: every round is one pass over the scores and one block-wide sum.  2. Eq. 3 at these
+// probabilities (probe only).  3. The number of kept rows in every chunk of 32 rows, and the exclusive
+// prefix sums of these counts: emit_pack_kernel then places every chunk's rows without looking at others.
+__global__ void __launch_bounds__(SAMPLER_THREADS) sample_w_kernel(SampleWParams P) {
+  extern __shared__ __align__(16) float s_w[];
+  __shared__ WShared sh;
+  pdl_wait();      // the scores come from the kernel before this one
+  pdl_trigger();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int N = P.N, T = P.T, R = N * T;
-  // Element e of this thread is row (e / 4) * 4096 + tid * 4 + (e % 4): four consecutive rows per
-  // thread and group, so that every 16-byte load or store of a warp covers 512 contiguous bytes.
-  auto row_of = [&](int e) { return (e >> 2) * (4 * SAMPLER_THREADS) + tid * 4 + (e & 3); };
+  const int cntA = P.counts[0];
+  const int T = P.T;
+  const int n = cntA * T;
+  const bool in_smem = n <= P.smem_rows;
+  if (in_smem) {
+    const int n4 = n >> 2;
+    for (int i = tid; i < n4; i += SAMPLER_THREADS)
+      reinterpret_cast<float4*>(s_w)[i] = reinterpret_cast<const float4*>(P.wc)[i];
+    for (int i = (n4 << 2) + tid; i < n; i += SAMPLER_THREADS) s_w[i] = P.wc[i];
+    __syncthreads();
+  }
+  const float* w = in_smem ? s_w : P.wc;
 
-  // this thread's rows: the unscaled leverage score and the SampleW uniform, both made per row by
-  // the row-norm kernel
-  float ab[E];
-#pragma unroll
-  for (int e = 0; e < E; e += 4) {
-    const int rb = row_of(e);
-    if (rb + 3 < R) {
-      const float4 v = *reinterpret_cast<const float4*>(P.lev + rb);
-      ab[e] = v.x; ab[e + 1] = v.y; ab[e + 2] = v.z; ab[e + 3] = v.w;
-    } else {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) ab[e + i] = rb + i < R ? P.lev[rb + i] : 0.f;
-    }
-  }
-  // The rows' SampleW uniforms: requested now, together with the scores, when the registers allow it
-  // (E <= 8); with E = 16 they are loaded just before the masks are drawn.
-  constexpr bool EARLY_U = E <= 8;
-  uint32_t ue[EARLY_U ? E : 4];
-  if (EARLY_U) {
-#pragma unroll
-    for (int e = 0; e < (EARLY_U ? E : 4); e += 4) {
-      const int rb = row_of(e);
-      ue[e] = ue[e + 1] = ue[e + 2] = ue[e + 3] = 0xffffffffu;
-      if (P.sample_w) {
-        if (rb + 3 < R) {
-          const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + rb);
-          ue[e] = u.x; ue[e + 1] = u.y; ue[e + 2] = u.z; ue[e + 3] = u.w;
-        } else {
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            if (rb + i < R) ue[e + i] = P.u24[rb + i];
-        }
-      }
-    }
-  }
-  // Datum of each of this thread's rows, one division per group of four rows, kept as one word per
-  // group (registers are scarce at 1024 threads): the first row's datum and three 2-bit increments.
-  int ncode[E / 4];
-#pragma unroll
-  for (int e = 0; e < E; e += 4) {
-    const int rb = row_of(e);
-    const int n0 = rb / T;
-    int n = n0, rem = rb - n0 * T, code = n0;
-#pragma unroll
-    for (int i = 1; i < 4; ++i) {
-      if (++rem == T) { rem = 0; ++n; }
-      code |= (n - n0) << (14 + 2 * i);
-    }
-    ncode[e >> 2] = code;
-  }
-  auto datum_of = [&](int e) {
-    const int code = ncode[e >> 2];
-    const int n = (code & 0xffff) + ((e & 3) ? ((code >> (14 + 2 * (e & 3))) & 3) : 0);
-    return n < N ? n : N - 1;
-  };
-
-  // ---- ||G_n||_F: one warp per datum, fixed order
-  for (int n = warp; n < N; n += 32) {
-    const float s = datum_sqnorm_warp(P.a + (size_t)n * T, T, lane);
-    if (lane == 0) { const float g = sqrtf(s); P.g[n] = g; sh.pA[n] = g; }
-  }
-  __syncthreads();
-  // ---- SampleA inside warp 0 (Sec. 4.1): p_n, mask, kept / dropped lists
-  if (warp == 0) {
-    SampleAOut o;
-    o.p = P.p; o.scaleA = P.scaleA; o.idxA = P.idxA; o.dropA = P.dropA;
-    o.sh_p = sh.pA; o.sh_scaleA = sh.scaleA;
-    const int kept = sample_a_warp<SLOTS>(sh.pA, N, P.rho, P.p_in, P.seed, o, lane);
-    if (lane == 0) sh.cntA = kept;
-  }
-  __syncthreads();
-  const int cntA = sh.cntA;
-
-  // ---- SampleW (Sec. 4.2, Eq. 3): leverage scores of G_hat in registers
-  float w[E];
-#pragma unroll
-  for (int e = 0; e < E; ++e) {
-    const int n = datum_of(e);
-    w[e] = (row_of(e) < R && sh.scaleA[n] > 0.f) ? ab[e] / sh.pA[n] : 0.f;
-  }
-#pragma unroll
-  for (int e = 0; e < E; e += 4) {
-    const int rb = row_of(e);
-    if (rb + 3 < R) {
-      *reinterpret_cast<float4*>(P.w + rb) = make_float4(w[e], w[e + 1], w[e + 2], w[e + 3]);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (rb + i < R) P.w[rb + i] = w[e + i];
-    }
-  }
-  float q[E];
-  if (P.q_in != nullptr) {
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-      const int r = row_of(e);
-      q[e] = (r < R && sh.scaleA[datum_of(e)] > 0.f) ? P.q_in[r] : 0.f;
-    }
-  } else {
+  int mode = Q_GIVEN;
+  float c = 0.f;
+  if (P.q_in == nullptr) {
     const float budget = P.nu * (float)T * (float)cntA;
     float S = 0.f;
     int nz = 0;
-#pragma unroll
-    for (int e = 0; e < E; ++e)
-      if (w[e] > 0.f) { S += w[e]; ++nz; }
+    for (int i = tid; i < n; i += SAMPLER_THREADS) {
+      const float x = w[i];
+      if (x > 0.f) { S += x; ++nz; }
+    }
     int parity = 0;
     fast_sum(S, nz, &sh, parity); parity ^= 1;
     if (nz == 0 || budget <= 0.f) {
-#pragma unroll
-      for (int e = 0; e < E; ++e) q[e] = 0.f;
+      mode = Q_ZERO;
     } else if ((float)nz <= budget) {
-#pragma unroll
-      for (int e = 0; e < E; ++e) q[e] = w[e] > 0.f ? 1.f : 0.f;
+      mode = Q_ONES;
     } else {
-      float c = budget / S;
+      mode = Q_CAPPED;
+      c = budget / S;
       int k = 0;
-      for (int iter = 0; iter < 128; ++iter) {
+      bool converged = false;
+      for (int iter = 0; iter < WATER_ROUNDS; ++iter) {
         float Su = 0.f;
         int ks = 0;
-#pragma unroll
-        for (int e = 0; e < E; ++e)
-          if (w[e] > 0.f) {
-            if (c * w[e] >= 1.0f) ++ks; else Su += w[e];
+        for (int i = tid; i < n; i += SAMPLER_THREADS) {
+          const float x = w[i];
+          if (x > 0.f) {
+            if (c * x >= 1.0f) ++ks; else Su += x;
           }
+        }
         fast_sum(Su, ks, &sh, parity); parity ^= 1;
-        if (ks == k) break;
+        if (ks == k) { converged = true; break; }
         k = ks;
         if (Su > 0.f) {
           const float cn = (budget - (float)k) / Su;
           c = cn > c ? cn : c;
         }
       }
-#pragma unroll
-      for (int e = 0; e < E; ++e) {
-        float r = 0.f;
-        if (w[e] > 0.f) {
-          const float cx = c * w[e];
-          r = cx >= 1.0f ? 1.f : cx;
-        }
-        q[e] = r;
-      }
+      if (!converged && tid == 0) atomicExch(P.status, (int32_t)VCAS_ERR_INTERNAL);
     }
   }
-#pragma unroll
-  for (int e = 0; e < E; e += 4) {
-    const int rb = row_of(e);
-    if (rb + 3 < R) {
-      *reinterpret_cast<float4*>(P.q + rb) = make_float4(q[e], q[e + 1], q[e + 2], q[e + 3]);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (rb + i < R) P.q[rb + i] = q[e + i];
-    }
-  }
+  __syncthreads();      // the reduction buffers are free again
 
-  if (P.accumulate_vw) {      // Eq. 3 at these probabilities (probe only)
+  if (P.accumulate_vw) {      // Eq. 3 at these probabilities
     float vw = 0.f;
     int dummy = 0;
-#pragma unroll
-    for (int e = 0; e < E; ++e)
-      if (q[e] > 0.f) vw += (1.0f - q[e]) / q[e] * w[e] * w[e];
+    for (int i = tid; i < n; i += SAMPLER_THREADS) {
+      const int k = i / T;
+      const float x = w[i];
+      const float q = q_of(mode, c, x, P.q_in, P.q_in != nullptr ? P.idxA[k] * T + (i - k * T) : 0);
+      if (q > 0.f) vw += (1.0f - q) / q * x * x;
+    }
     fast_sum(vw, dummy, &sh, 0);
     if (tid == 0) P.acc[1] += (double)vw;
-  }
-
-  // ---- mask and ordered compaction: rows ascend with (group, thread, k), so each group of 4096 rows
-  // gets its own block-wide exclusive scan of the per-thread counts, on top of the groups before it
-  unsigned keepbits = 0;
-#pragma unroll
-  for (int e = 0; e < E; e += 4) {
-    const int rb = row_of(e);
-    uint32_t ur[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};   // the rows' SampleW uniforms
-    if (EARLY_U) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) ur[i] = ue[(EARLY_U ? e : 0) + i];
-    } else if (P.sample_w) {
-      if (rb + 3 < R) {
-        const uint4 u = *reinterpret_cast<const uint4*>(P.u24 + rb);
-        ur[0] = u.x; ur[1] = u.y; ur[2] = u.z; ur[3] = u.w;
-      } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          if (rb + i < R) ur[i] = P.u24[rb + i];
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      bool k = false;
-      if (rb + i < R) {
-        if (P.sample_w) k = q[e + i] > 0.f && ur[i] < (uint32_t)floorf(q[e + i] * 16777216.0f);
-        else k = sh.scaleA[datum_of(e + i)] > 0.f;
-      }
-      keepbits |= (k ? 1u : 0u) << (e + i);
-    }
-  }
-  int total = 0;
-#pragma unroll
-  for (int g4 = 0; g4 < E / 4; ++g4) {
-    const unsigned bits = (keepbits >> (g4 * 4)) & 0xfu;
-    const int mine = __popc(bits);
-    int incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += t;
-    }
-    __syncthreads();                       // warp_tot of the previous group has been read by everyone
-    if (lane == 31) sh.warp_tot[warp] = incl;
     __syncthreads();
-    const int wt = sh.warp_tot[lane];
-    const int base0 = total + incl - mine + __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0);
-    total += __reduce_add_sync(0xffffffffu, wt);
-    int base = base0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-      if (bits & (1u << i)) {
-        const int e = g4 * 4 + i;
-        P.idxW[base] = row_of(e);
-        P.scaleW[base] = P.sample_w ? sh.scaleA[datum_of(e)] / q[e] : sh.scaleA[datum_of(e)];
-        ++base;
-      }
   }
-  if (tid == 0) { P.counts[0] = cntA; P.counts[1] = total; }
-}
 
-// SampleA alone (Sec. 4.1), for the dX product: the same warp-level code as in the sampling kernels, so the
-// masks are identical; results go to arrays of their own because the full sampling kernel runs at the
-// same time on another stream.
-constexpr int SAMPLE_A_THREADS = 512;
-template <int SLOTS>
-__global__ void __launch_bounds__(SAMPLE_A_THREADS)
-sample_a_kernel(const float* __restrict__ a, int N, int T, float rho, const float* __restrict__ p_in, uint64_t seed,
-                float* scaleA, int32_t* idxA, int32_t* dropA, int32_t* cnt) {
-  __shared__ float s_g[32 * SLOTS];
-  pdl_wait();      // the row norms come from the kernel before this one
-  pdl_trigger();   // the dX product kernel may set itself up meanwhile
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int n = warp; n < N; n += SAMPLE_A_THREADS / 32) {
-    const float s = datum_sqnorm_warp(a + (size_t)n * T, T, lane);
-    if (lane == 0) s_g[n] = sqrtf(s);
+  // kept rows per chunk of 32 compact rows: chunk_off[ch] = count for now
+  const int nchunks = (n + 31) >> 5;
+  for (int ch = warp; ch < nchunks; ch += SAMPLER_THREADS / 32) {
+    const int i = (ch << 5) + lane;
+    bool keep = false;
+    if (i < n) {
+      const int k = i / T;
+      const float q = q_of(mode, c, w[i], P.q_in, P.q_in != nullptr ? P.idxA[k] * T + (i - k * T) : 0);
+      keep = row_kept(P.sample_w, q, P.sample_w ? P.uc[i] : 0u);
+    }
+    const unsigned b = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0) P.chunk_off[ch] = __popc(b);
   }
   __syncthreads();
-  if (warp == 0) {
-    SampleAOut o;
-    o.p = nullptr; o.scaleA = scaleA; o.idxA = idxA; o.dropA = dropA;
-    o.sh_p = nullptr; o.sh_scaleA = nullptr;
-    const int kept = sample_a_warp<SLOTS>(s_g, N, rho, p_in, seed, o, lane);
-    if (lane == 0) *cnt = kept;
+  // exclusive prefix sums over the chunk counts: every thread owns a contiguous segment
+  const int seg = (nchunks + SAMPLER_THREADS - 1) / SAMPLER_THREADS;
+  const int lo = tid * seg, hi = min(nchunks, lo + seg);
+  int mine = 0;
+  for (int ch = lo; ch < hi; ++ch) mine += P.chunk_off[ch];
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) sh.scan[warp] = incl;
+  __syncthreads();
+  const int wt = sh.scan[lane];
+  int base = incl - mine + __reduce_add_sync(0xffffffffu, lane < warp ? wt : 0);
+  const int total = __reduce_add_sync(0xffffffffu, wt);
+  for (int ch = lo; ch < hi; ++ch) {
+    const int cnt = P.chunk_off[ch];
+    P.chunk_off[ch] = base;
+    base += cnt;
+  }
+  if (tid == 0) {
+    P.counts[1] = total;
+    P.fix[0] = c;
+    P.fix[1] = (float)mode;
+  }
+}
+
+struct EmitParams {
+  const float* wc; const uint32_t* uc;
+  const float* q_in;
+  const float* scaleA;
+  const int32_t* idxA; const int32_t* dropA;
+  const int32_t* counts; const int32_t* chunk_off; const float* fix;
+  float* w; float* q; float* scaleW; int32_t* idxW;
+  const __nv_bfloat16* dY; const __nv_bfloat16* X;       // operands to pack (nullptr: that one is not packed)
+  __nv_bfloat16* packG; __nv_bfloat16* packX;
+  int N, T, d_in, d_out;
+  int sample_w;
+};
+
+// Row k of packG = scaleW[k] * dY[idxW[k]] (G_tilde of Sec. 4.2, rounded to bf16), row k of packX = X[idxW[k]].
+__device__ __forceinline__ void pack_row(const __nv_bfloat16* src, __nv_bfloat16* dst, int d, float sc, bool scaled) {
+  const uint4* in = reinterpret_cast<const uint4*>(src);
+  uint4* out = reinterpret_cast<uint4*>(dst);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
+    const uint4 v = __ldg(in + i);
+    if (scaled) {
+      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+      uint32_t o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 t = __floats2bfloat162_rn(sc * __uint_as_float(u[e] << 16),
+                                                       sc * __uint_as_float(u[e] & 0xffff0000u));
+        o[e] = *reinterpret_cast<const uint32_t*>(&t);
+      }
+      out[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    } else {
+      out[i] = v;
+    }
+  }
+}
+
+// One CTA per chunk of 32 compact rows (grid-strided): the chunk's kept rows go to positions chunk_off[ch]...
+// of the ascending kept-row list with their rescale factors 1/(p_n q_r); q and w are written by global row;
+// the rows' operands are packed for the dW product.  The rows of dropped data get w = q = 0, and the compact
+// operands are padded with zero rows to a multiple of 64 (the product's last k-block then adds nothing).
+constexpr int EMIT_THREADS = 128;
+__global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
+  __shared__ int s_r[32], s_pos[32], s_cnt;
+  __shared__ float s_sc[32];
+  pdl_wait();      // c and the chunk offsets come from the kernel before this one
+  pdl_trigger();   // the dW product kernel may set itself up; it waits for this grid before loading
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cntA = P.counts[0], cntW = P.counts[1];
+  const int T = P.T;
+  const int n = cntA * T;
+  const float c = P.fix[0];
+  const int mode = (int)P.fix[1];
+  const int nchunks = (n + 31) >> 5;
+  const bool pack = P.packG != nullptr || P.packX != nullptr;
+  for (int ch = blockIdx.x; ch < nchunks; ch += gridDim.x) {
+    if (warp == 0) {
+      const int i = (ch << 5) + lane;
+      bool keep = false;
+      float q = 0.f, wv = 0.f, sa = 0.f;
+      int r = 0;
+      if (i < n) {
+        const int k = i / T;
+        const int nd = P.idxA[k];
+        r = nd * T + (i - k * T);
+        wv = P.wc[i];
+        q = q_of(mode, c, wv, P.q_in, r);
+        keep = row_kept(P.sample_w, q, P.sample_w ? P.uc[i] : 0u);
+        sa = P.scaleA[nd];
+        P.w[r] = wv;
+        P.q[r] = q;
+      }
+      const unsigned b = __ballot_sync(0xffffffffu, keep);
+      if (keep) {
+        const int j = __popc(b & ((1u << lane) - 1u));
+        const int pos = P.chunk_off[ch] + j;
+        const float sc = P.sample_w ? sa / q : sa;
+        P.idxW[pos] = r;
+        P.scaleW[pos] = sc;
+        s_r[j] = r; s_pos[j] = pos; s_sc[j] = sc;
+      }
+      if (lane == 0) s_cnt = __popc(b);
+    }
+    if (pack) {
+      __syncthreads();
+      const int m = s_cnt;
+      for (int j = 0; j < m; ++j) {
+        const size_t r = (size_t)s_r[j], pos = (size_t)s_pos[j];
+        if (P.packG != nullptr) pack_row(P.dY + r * P.d_out, P.packG + pos * P.d_out, P.d_out, s_sc[j], true);
+        if (P.packX != nullptr) pack_row(P.X + r * P.d_in, P.packX + pos * P.d_in, P.d_in, 1.f, false);
+      }
+      __syncthreads();
+    }
+  }
+  // rows of dropped data
+  const int ndrop_rows = (P.N - cntA) * T;
+  for (int i = blockIdx.x * EMIT_THREADS + tid; i < ndrop_rows; i += gridDim.x * EMIT_THREADS) {
+    const int k = i / T;
+    const int r = P.dropA[k] * T + (i - k * T);
+    P.w[r] = 0.f;
+    P.q[r] = 0.f;
+  }
+  // zero rows up to the next multiple of 64
+  if (pack) {
+    const int padded = (cntW + 63) / 64 * 64;
+    for (int k = cntW + (int)blockIdx.x; k < padded; k += gridDim.x) {
+      if (P.packG != nullptr)
+        for (int i = tid; i < P.d_out / 8; i += EMIT_THREADS)
+          reinterpret_cast<uint4*>(P.packG + (size_t)k * P.d_out)[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (P.packX != nullptr)
+        for (int i = tid; i < P.d_in / 8; i += EMIT_THREADS)
+          reinterpret_cast<uint4*>(P.packX + (size_t)k * P.d_in)[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
   }
 }
 
@@ -510,50 +518,81 @@ mask_kernel(const float* __restrict__ p, int n, uint64_t seed, int sampler, uint
   if (threadIdx.x == 0 && cnt != nullptr) *cnt = c;
 }
 
+constexpr int SAMPLE_W_SMEM_ROWS = 56 * 1024;     // 224 KB of scores
+
 }  // namespace
 
-cudaError_t launch_sampler(Handle* h, const SamplerArgs& a, cudaStream_t st, bool after_event) {
+cudaError_t launch_sample_a(Handle* h, const SamplerArgs& a, bool programmatic, cudaStream_t st) {
   const Workspace& ws = h->ws;
-  SamplerParams P;
-  P.a = ws.a; P.b = ws.b; P.lev = ws.lev; P.u24 = ws.u24; P.g = ws.g; P.p = ws.p; P.w = ws.w; P.q = ws.q;
-  P.scaleA = ws.scaleA; P.scaleW = ws.scaleW;
-  P.idxA = ws.idxA; P.dropA = ws.dropA; P.idxW = ws.idxW; P.counts = ws.counts;
-  P.acc = ws.acc;
-  P.p_in = a.p_in; P.q_in = a.q_in;
-  P.N = h->desc.N; P.T = h->desc.T;
-  P.rho = a.rho; P.nu = a.nu; P.seed = a.seed;
-  P.sample_w = a.sample_w; P.accumulate_vw = a.accumulate_vw;
-  const int R = P.N * P.T;
-  cudaError_t e = cudaSuccess;
-  // after_event: the kernel before this one in the stream is not the producer of its inputs (those
-  // arrive through an event from another stream), so it is launched without the programmatic attribute
-  auto go = [&](void (*k)(SamplerParams)) {
-    if (after_event) { k<<<1, SAMPLER_THREADS, 0, st>>>(P); return cudaSuccess; }
-    return launch_after(k, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
-  };
-  if (fast_sampling(h->desc)) {
-    const bool wide = P.N > 32;       // SampleA slots per lane of warp 0
-    if (R <= 4 * SAMPLER_THREADS) e = go(wide ? sampler_fast_kernel<4, 32> : sampler_fast_kernel<4, 1>);
-    else if (R <= 8 * SAMPLER_THREADS) e = go(wide ? sampler_fast_kernel<8, 32> : sampler_fast_kernel<8, 1>);
-    else e = go(wide ? sampler_fast_kernel<16, 32> : sampler_fast_kernel<16, 1>);
-  } else {
-    e = go(sampler_kernel);
-  }
+  const vcas_layer_desc& d = h->desc;
+  SampleAParams P;
+  P.a = a.a_in != nullptr ? a.a_in : ws.a;
+  P.a_parts = a.a_in != nullptr ? a.a_parts : 1;
+  P.alive = a.alive; P.alive_cnt = a.alive_cnt;
+  P.N = d.N; P.T = d.T; P.rho = a.rho; P.p_in = a.p_in; P.seed = a.seed;
+  P.g = ws.g; P.p = ws.p; P.scaleA = ws.scaleA; P.idxA = ws.idxA; P.dropA = ws.dropA; P.counts = ws.counts;
+  P.kept_out = a.kept_out; P.kept_cnt_out = a.kept_cnt_out;
+  P.status = ws.status;
+  cudaError_t e;
+  if (d.N <= 32)
+    e = launch_maybe_after(programmatic, sample_a_kernel<1>, dim3(1), dim3(SAMPLE_A_THREADS), 0, st, P);
+  else if (d.N <= WARP_MAX_N)
+    e = launch_maybe_after(programmatic, sample_a_kernel<32>, dim3(1), dim3(SAMPLE_A_THREADS), 0, st, P);
+  else
+    e = launch_maybe_after(programmatic, sample_a_big_kernel, dim3(1), dim3(SAMPLER_THREADS), 0, st, P);
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t launch_sample_a(Handle* h, const SamplerArgs& a, cudaStream_t st) {
+cudaError_t launch_sample_w(Handle* h, const SamplerArgs& a, cudaStream_t st) {
+  static std::atomic<bool> attr_set[64];
   const Workspace& ws = h->ws;
   const vcas_layer_desc& d = h->desc;
-  if (!fast_sampling(d)) return cudaErrorInvalidValue;
-  cudaError_t e;
-  if (d.N <= 32)
-    e = launch_after(sample_a_kernel<1>, dim3(1), dim3(SAMPLE_A_THREADS), 0, st, (const float*)ws.a, d.N, d.T, a.rho,
-                     a.p_in, a.seed, ws.scaleA2, ws.idxA2, ws.dropA2, ws.counts + 6);
-  else
-    e = launch_after(sample_a_kernel<32>, dim3(1), dim3(SAMPLE_A_THREADS), 0, st, (const float*)ws.a, d.N, d.T, a.rho,
-                     a.p_in, a.seed, ws.scaleA2, ws.idxA2, ws.dropA2, ws.counts + 6);
+  const long R = (long)d.N * d.T;
+  // shared memory for the scores: enough for every row when that fits, else the kernel reads global memory
+  // whenever the kept rows exceed it
+  int rows = (int)(R < SAMPLE_W_SMEM_ROWS ? R : SAMPLE_W_SMEM_ROWS);
+  rows = (rows + 3) & ~3;
+  const size_t smem = (size_t)rows * sizeof(float);
+  if (smem > 48 * 1024) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev].load(std::memory_order_acquire)) {
+      e = cudaFuncSetAttribute(sample_w_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               SAMPLE_W_SMEM_ROWS * (int)sizeof(float));
+      if (e != cudaSuccess) return e;
+      attr_set[dev].store(true, std::memory_order_release);
+    }
+  }
+  SampleWParams P;
+  P.wc = ws.wc; P.uc = ws.uc; P.q_in = a.q_in; P.idxA = ws.idxA;
+  P.counts = ws.counts; P.chunk_off = ws.chunk_off; P.fix = ws.fix; P.acc = ws.acc; P.status = ws.status;
+  P.T = d.T; P.nu = a.nu; P.sample_w = a.sample_w; P.accumulate_vw = a.accumulate_vw;
+  P.smem_rows = rows;
+  const cudaError_t e = launch_after(sample_w_kernel, dim3(1), dim3(SAMPLER_THREADS), smem, st, P);
+  h->launches += 1;
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_emit_pack(Handle* h, const void* dY, const void* X, const SamplerArgs& a, bool pack, cudaStream_t st) {
+  const Workspace& ws = h->ws;
+  const vcas_layer_desc& d = h->desc;
+  EmitParams P;
+  P.wc = ws.wc; P.uc = ws.uc; P.q_in = a.q_in; P.scaleA = ws.scaleA; P.idxA = ws.idxA; P.dropA = ws.dropA;
+  P.counts = ws.counts; P.chunk_off = ws.chunk_off; P.fix = ws.fix;
+  P.w = ws.w; P.q = ws.q; P.scaleW = ws.scaleW; P.idxW = ws.idxW;
+  P.dY = (const __nv_bfloat16*)dY; P.X = (const __nv_bfloat16*)X;
+  P.packG = pack ? ws.packG : nullptr;
+  P.packX = pack ? ws.packX : nullptr;
+  P.N = d.N; P.T = d.T; P.d_in = d.d_in; P.d_out = d.d_out;
+  P.sample_w = a.sample_w;
+  const long R = (long)d.N * d.T;
+  long blocks = (R + 31) / 32;
+  const long cap = (long)(h->num_sms > 0 ? h->num_sms : 148) * 8;
+  if (blocks > cap) blocks = cap;
+  const cudaError_t e = launch_after(emit_pack_kernel, dim3((unsigned)blocks), dim3(EMIT_THREADS), 0, st, P);
   h->launches += 1;
   return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -1,6 +1,7 @@
 // Row square-norms of dY and X (Sec. 4.1: ||G_n||_F is built from them; Sec. 4.2: the
-// leverage scores ||G_hat_r|| ||X_r||).  HBM-bound: every input byte is read exactly once,
-// with 128-bit loads, one warp per row, fp32 accumulation and a shuffle reduction.
+// leverage scores ||G_hat_r|| ||X_r||).  HBM-bound: 128-bit loads, one warp per row, fp32
+// accumulation and a shuffle reduction.  Two passes: every row of dY that can be non-zero is read
+// once, before SampleA; of X only the rows of the data SampleA kept are read, after it.
 #include "common.cuh"
 
 namespace vcas {
@@ -68,64 +69,116 @@ __device__ __forceinline__ float row_partial(const T* __restrict__ src, int d, i
   return (acc0 + acc1) + (acc2 + acc3);
 }
 
-// One warp per row r: a[r] = ||dY_r||^2, b[r] = ||X_r||^2, and two per-row values the sampling
-// stage would otherwise compute on its single SM: lev[r] = ||dY_r|| ||X_r|| (the leverage score of
-// Sec. 4.2 before the 1/p_n rescale) and u24[r], the 24-bit Philox uniform of SampleW for this row.
+// One warp per row: a[r] = ||dY_r||^2.  With a list of alive data only their rows are read (the rows of every
+// other datum are known to be zero: they were dropped by a layer above).
+// The result of row r goes to a[r * stride], followed by stride - 1 zeros (the layout of a producer's partial sums).
 template <typename T>
-__global__ void __launch_bounds__(256) rownorm_kernel(const T* __restrict__ dY, const T* __restrict__ X,
-                                                      int R, int d_out, int d_in, uint64_t seed,
-                                                      float* __restrict__ a, float* __restrict__ b,
-                                                      float* __restrict__ lev, uint32_t* __restrict__ u24) {
+__global__ void __launch_bounds__(256) rownorm_dy_kernel(const T* __restrict__ dY, int R, int Tn, int d_out,
+                                                         const int32_t* __restrict__ alive,
+                                                         const int32_t* __restrict__ alive_cnt, float* __restrict__ a,
+                                                         int stride) {
   pdl_trigger();   // the next kernel may be scheduled now; it waits for this grid before reading
   const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= R) return;
-  // the first four vectors per lane of the X row are requested before the dY row is touched
-  using V = typename Vec<T>::type;
-  constexpr int VN = Vec<T>::N;
-  const T* xrow = X + (size_t)row * d_in;
-  const bool xvec = (d_in % VN) == 0;
-  const int nvx = xvec ? d_in / VN : 0;
-  V xv[4];
-#pragma unroll
-  for (int k = 0; k < 4; ++k)
-    if (lane + 32 * k < nvx) xv[k] = __ldg(reinterpret_cast<const V*>(xrow) + lane + 32 * k);
-  const float pa = row_partial<T>(dY + (size_t)row * d_out, d_out, lane);
-  float pb = 0.f;
-  if (xvec) {
-#pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if (lane + 32 * k < nvx) pb += Vec<T>::sq(xv[k]);
-    for (int i = lane + 128; i < nvx; i += 32) pb += Vec<T>::sq(__ldg(reinterpret_cast<const V*>(xrow) + i));
-  } else {
-    pb = row_partial<T>(xrow, d_in, lane);
+  const int wpb = blockDim.x >> 5;
+  const int rows = alive != nullptr ? *alive_cnt * Tn : R;
+  for (int c = blockIdx.x * wpb + (threadIdx.x >> 5); c < rows; c += gridDim.x * wpb) {
+    int r = c;
+    if (alive != nullptr) { const int k = c / Tn; r = alive[k] * Tn + (c - k * Tn); }
+    const float sa = warp_sum(row_partial<T>(dY + (size_t)r * d_out, d_out, lane));
+    if (lane == 0) a[(size_t)r * stride] = sa;
+    else if (lane < stride) a[(size_t)r * stride + lane] = 0.f;
   }
-  const float sa = warp_sum(pa), sb = warp_sum(pb);
-  if (lane == 0) {
-    a[row] = sa;
-    b[row] = sb;
-    lev[row] = sqrtf(sa) * sqrtf(sb);
-    u24[row] = philox_word0((uint32_t)row, 0u, 1u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32)) >> 8;
+}
+
+// One warp per row of a kept datum, in compact order (entry c = k*T + t is token t of the k-th kept datum):
+// ||X_r||^2, then the leverage score of the rescaled gradient, w = ||dY_r|| ||X_r|| / p_n (Sec. 4.2, Eq. 3),
+// and the row's 24-bit Philox uniform of SampleW, so that the single-CTA stage that follows has no per-row
+// transcendental or Philox work.  a_r is the sum of a_parts consecutive floats (partial sums of a producer).
+template <typename T>
+__global__ void __launch_bounds__(256) scores_x_kernel(const T* __restrict__ X, int Tn, int d_in,
+                                                       const float* __restrict__ a, int a_parts,
+                                                       const float* __restrict__ p, const int32_t* __restrict__ idxA,
+                                                       const int32_t* __restrict__ counts, uint64_t seed, int sample_w,
+                                                       float* __restrict__ wc, uint32_t* __restrict__ uc) {
+  pdl_wait();      // the kept data come from the SampleA kernel
+  pdl_trigger();
+  const int lane = threadIdx.x & 31;
+  const int wpb = blockDim.x >> 5;
+  const int rows = counts[0] * Tn;
+  for (int c = blockIdx.x * wpb + (threadIdx.x >> 5); c < rows; c += gridDim.x * wpb) {
+    const int k = c / Tn;
+    const int n = idxA[k];
+    const int r = n * Tn + (c - k * Tn);
+    const float sb = warp_sum(row_partial<T>(X + (size_t)r * d_in, d_in, lane));
+    if (lane == 0) {
+      float sa = 0.f;
+      for (int j = 0; j < a_parts; ++j) sa += a[(size_t)r * a_parts + j];
+      wc[c] = sqrtf(sa) * sqrtf(sb) / p[n];
+      uc[c] = sample_w ? philox_word0((uint32_t)r, 0u, 1u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32)) >> 8 : 0u;
+    }
   }
+}
+
+int row_grid(const Handle* h, long rows) {
+  long blocks = (rows + 7) / 8;
+  const long cap = (long)(h->num_sms > 0 ? h->num_sms : 148) * 8;     // eight resident CTAs of 256 threads per SM
+  if (blocks > cap) blocks = cap;
+  return (int)(blocks < 1 ? 1 : blocks);
 }
 
 }  // namespace
 
-cudaError_t launch_rownorms(Handle* h, const void* dY, const void* X, uint64_t seed, cudaStream_t st) {
+cudaError_t launch_rownorm_dy(Handle* h, const void* dY, const SamplerArgs& s, cudaStream_t st) {
+  if (s.a_in != nullptr) return cudaSuccess;     // the producer of dY supplied its row norms
   const vcas_layer_desc& d = h->desc;
   const int R = d.N * d.T;
-  const int warps_per_block = 8;
-  const int blocks = (R + warps_per_block - 1) / warps_per_block;
+  const int blocks = row_grid(h, R);
   if (d.dtype == VCAS_DTYPE_BF16) {
-    rownorm_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dY, (const __nv_bfloat16*)X, R,
-                                                          d.d_out, d.d_in, seed, h->ws.a, h->ws.b, h->ws.lev,
-                                                          h->ws.u24);
+    rownorm_dy_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dY, R, d.T, d.d_out, s.alive,
+                                                             s.alive_cnt, h->ws.a, 1);
   } else {
-    rownorm_kernel<float><<<blocks, 256, 0, st>>>((const float*)dY, (const float*)X, R, d.d_out, d.d_in, seed,
-                                                  h->ws.a, h->ws.b, h->ws.lev, h->ws.u24);
+    rownorm_dy_kernel<float><<<blocks, 256, 0, st>>>((const float*)dY, R, d.T, d.d_out, s.alive, s.alive_cnt, h->ws.a, 1);
   }
   h->launches += 1;
   return cudaGetLastError();
+}
+
+cudaError_t launch_rownorm_out(Handle* h, const void* dX, float* a_out, cudaStream_t st) {
+  const vcas_layer_desc& d = h->desc;
+  const int R = d.N * d.T;
+  const int blocks = row_grid(h, R);
+  const int parts = a_out_parts(d.d_in);
+  if (d.dtype == VCAS_DTYPE_BF16)
+    rownorm_dy_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dX, R, d.T, d.d_in, nullptr, nullptr,
+                                                             a_out, parts);
+  else
+    rownorm_dy_kernel<float><<<blocks, 256, 0, st>>>((const float*)dX, R, d.T, d.d_in, nullptr, nullptr, a_out, parts);
+  h->launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scores_x(Handle* h, const void* X, const SamplerArgs& s, bool programmatic, cudaStream_t st) {
+  const vcas_layer_desc& d = h->desc;
+  const Workspace& ws = h->ws;
+  // the number of kept rows is only known on the device: the grid is sized for the expected share of rows
+  // (at least a quarter) and strides over what there is
+  double share = (double)s.rho * 1.5;
+  if (share < 0.25) share = 0.25;
+  if (share > 1.0) share = 1.0;
+  const int blocks = row_grid(h, (long)(share * (double)d.N * d.T) + 8);
+  const float* a = s.a_in != nullptr ? s.a_in : ws.a;
+  const int parts = s.a_in != nullptr ? s.a_parts : 1;
+  cudaError_t e;
+  if (d.dtype == VCAS_DTYPE_BF16)
+    e = launch_maybe_after(programmatic, scores_x_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st,
+                           (const __nv_bfloat16*)X, d.T, d.d_in, a, parts, (const float*)ws.p, (const int32_t*)ws.idxA,
+                           (const int32_t*)ws.counts, s.seed, s.sample_w, ws.wc, ws.uc);
+  else
+    e = launch_maybe_after(programmatic, scores_x_kernel<float>, dim3(blocks), dim3(256), 0, st, (const float*)X, d.T,
+                           d.d_in, a, parts, (const float*)ws.p, (const int32_t*)ws.idxA, (const int32_t*)ws.counts,
+                           s.seed, s.sample_w, ws.wc, ws.uc);
+  h->launches += 1;
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace vcas

@@ -11,9 +11,9 @@ namespace {
 
 constexpr int STATIC_MAX_R = 16384;   // rows (N*T) the fixed scratch can serve
 constexpr int STATIC_MAX_N = 4096;    // data
-constexpr size_t kRowArrays = 8;      // a, b, w, q, scaleW, lev (float), idxW (int32), u24 (uint32), each [STATIC_MAX_R]
+constexpr size_t kRowArrays = 8;      // a, wc, w, q, scaleW (float), idxW, chunk_off (int32), uc (uint32), each [STATIC_MAX_R]
 constexpr size_t kDatumArrays = 6;    // g, p, scaleA, sorted (float) and idxA, dropA (int32), each [STATIC_MAX_N]
-constexpr size_t kTailBytes = 512;    // counts [8] int32 and acc [16] double, 256-byte slots
+constexpr size_t kTailBytes = 768;    // counts [8] int32, acc [16] double, fix [4] float + status word, 256-byte slots
 constexpr size_t kScratchBytes = kRowArrays * STATIC_MAX_R * 4 + kDatumArrays * STATIC_MAX_N * 4 + kTailBytes;
 
 // Lives in every GPU that loads the library until the process exits (about 0.6 MB).  In host
@@ -63,13 +63,13 @@ extern "C" int vcas_score_static(int32_t N, int32_t T, int32_t d_in, int32_t d_o
   float* fr = reinterpret_cast<float*>(base);
   Workspace& ws = h.ws;
   ws.a = fr + 0 * STATIC_MAX_R;
-  ws.b = fr + 1 * STATIC_MAX_R;
+  ws.wc = fr + 1 * STATIC_MAX_R;
   ws.w = fr + 2 * STATIC_MAX_R;
   ws.q = fr + 3 * STATIC_MAX_R;
   ws.scaleW = fr + 4 * STATIC_MAX_R;
   ws.idxW = reinterpret_cast<int32_t*>(fr + 5 * STATIC_MAX_R);
-  ws.lev = fr + 6 * STATIC_MAX_R;
-  ws.u24 = reinterpret_cast<uint32_t*>(fr + 7 * STATIC_MAX_R);
+  ws.chunk_off = reinterpret_cast<int32_t*>(fr + 6 * STATIC_MAX_R);
+  ws.uc = reinterpret_cast<uint32_t*>(fr + 7 * STATIC_MAX_R);
   float* fn = fr + kRowArrays * STATIC_MAX_R;
   ws.g = fn + 0 * STATIC_MAX_N;
   ws.p = fn + 1 * STATIC_MAX_N;
@@ -80,13 +80,17 @@ extern "C" int vcas_score_static(int32_t N, int32_t T, int32_t d_in, int32_t d_o
   unsigned char* tail = reinterpret_cast<unsigned char*>(fn + kDatumArrays * STATIC_MAX_N);
   ws.counts = reinterpret_cast<int32_t*>(tail);
   ws.acc = reinterpret_cast<double*>(tail + 256);
+  ws.fix = reinterpret_cast<float*>(tail + 512);
+  ws.status = reinterpret_cast<int32_t*>(tail + 512 + 64);
 
   // The array keeps the previous call's contents: the counters and accumulators start at zero.
   if (cudaMemsetAsync(tail, 0, kTailBytes, st) != cudaSuccess) return VCAS_ERR_CUDA;
-  SamplerArgs a;
-  a.rho = rho; a.nu = nu; a.seed = seed; a.p_in = nullptr; a.q_in = nullptr; a.sample_w = 1; a.accumulate_vw = 0;
-  if (launch_rownorms(&h, dY, X, seed, st) != cudaSuccess) return VCAS_ERR_CUDA;
-  if (launch_sampler(&h, a, st) != cudaSuccess) return VCAS_ERR_CUDA;
+  const SamplerArgs a = sampler_args(rho, nu, seed);
+  if (launch_rownorm_dy(&h, dY, a, st) != cudaSuccess) return VCAS_ERR_CUDA;
+  if (launch_sample_a(&h, a, true, st) != cudaSuccess) return VCAS_ERR_CUDA;
+  if (launch_scores_x(&h, X, a, true, st) != cudaSuccess) return VCAS_ERR_CUDA;
+  if (launch_sample_w(&h, a, st) != cudaSuccess) return VCAS_ERR_CUDA;
+  if (launch_emit_pack(&h, dY, X, a, false, st) != cudaSuccess) return VCAS_ERR_CUDA;
 
   const size_t R = (size_t)N * T;
   const cudaMemcpyKind k = cudaMemcpyDeviceToDevice;
