@@ -465,6 +465,8 @@ def main():
     ap.add_argument("--impl", default="vcas", choices=["vcas", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the workloads reported under other_workloads")
+    ap.add_argument("--sweep", default="grid", choices=["grid", "diag"],
+                    help="ratio sweep on the headline layer: the 5 x 5 grid of (rho, nu), or its diagonal only")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -612,7 +614,7 @@ def main():
     extra = None
     if world == 1 and not args.no_extra:
         sweep_seeds = list(range(20))
-        grid = [(r, n) for r in SWEEP for n in SWEEP]
+        grid = [(r, n) for r in SWEEP for n in SWEEP if args.sweep == "grid" or r == n]
         extra = {
             # BASELINE configs[4]: the 5 x 5 grid of keep ratios on the headline layer, 20 seeds per point
             "llm_mlp_up_ratio_sweep": measure_layer(case, vb, inputs, torch, dev, pk, grid, sweep_seeds,

@@ -397,39 +397,52 @@ struct EmitParams {
   const int32_t* idxA; const int32_t* dropA;
   const int32_t* counts; const int32_t* chunk_off; const float* fix;
   float* w; float* q; float* scaleW; int32_t* idxW;
-  const __nv_bfloat16* dY; const __nv_bfloat16* X;       // operands to pack (nullptr: that one is not packed)
-  __nv_bfloat16* packG; __nv_bfloat16* packX;
-  int N, T, d_in, d_out;
+  const __nv_bfloat16* src;  // the operand to pack, [R, d] (the narrower of dY and X), or nullptr
+  __nv_bfloat16* dst;        // [R_pad, d]: row k = src[idxW[k]] / (p q), rounded to bf16
+  int d;
+  int N, T;
   int sample_w;
+  int parts;                                             // CTAs that share the packing of one chunk's rows
 };
 
-// Row k of packG = scaleW[k] * dY[idxW[k]] (G_tilde of Sec. 4.2, rounded to bf16), row k of packX = X[idxW[k]].
-__device__ __forceinline__ void pack_row(const __nv_bfloat16* src, __nv_bfloat16* dst, int d, float sc, bool scaled) {
-  const uint4* in = reinterpret_cast<const uint4*>(src);
-  uint4* out = reinterpret_cast<uint4*>(dst);
-  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) {
-    const uint4 v = __ldg(in + i);
-    if (scaled) {
-      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-      uint32_t o[4];
+// Row k of the compact operand = scaleW[k] * src[idxW[k]], rounded to bf16: the factor 1/(p q) of G_tilde
+// (Sec. 4.2) sits on the contraction axis of G_tilde^T X, so it may scale either operand's row; it scales the
+// narrower one, and the other is read in place.  Four independent 16-byte loads per thread are in flight.
+__device__ __forceinline__ uint4 scale8(const uint4& v, float sc) {
+  const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+  uint32_t o[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const __nv_bfloat162 t = __floats2bfloat162_rn(sc * __uint_as_float(u[e] << 16),
-                                                       sc * __uint_as_float(u[e] & 0xffff0000u));
-        o[e] = *reinterpret_cast<const uint32_t*>(&t);
-      }
-      out[i] = make_uint4(o[0], o[1], o[2], o[3]);
-    } else {
-      out[i] = v;
-    }
+  for (int e = 0; e < 4; ++e) {
+    const __nv_bfloat162 t = __floats2bfloat162_rn(sc * __uint_as_float(u[e] << 16), sc * __uint_as_float(u[e] & 0xffff0000u));
+    o[e] = *reinterpret_cast<const uint32_t*>(&t);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+__device__ __forceinline__ void pack_row(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int d,
+                                         float sc) {
+  constexpr bool scaled = true;
+  const uint4* __restrict__ in = reinterpret_cast<const uint4*>(src);
+  uint4* __restrict__ out = reinterpret_cast<uint4*>(dst);
+  const int nv = d / 8, nt = blockDim.x;
+  int i = threadIdx.x;
+  for (; i + 3 * nt < nv; i += 4 * nt) {
+    uint4 v0 = __ldg(in + i), v1 = __ldg(in + i + nt), v2 = __ldg(in + i + 2 * nt), v3 = __ldg(in + i + 3 * nt);
+    if (scaled) { v0 = scale8(v0, sc); v1 = scale8(v1, sc); v2 = scale8(v2, sc); v3 = scale8(v3, sc); }
+    out[i] = v0; out[i + nt] = v1; out[i + 2 * nt] = v2; out[i + 3 * nt] = v3;
+  }
+  for (; i < nv; i += nt) {
+    uint4 v = __ldg(in + i);
+    if (scaled) v = scale8(v, sc);
+    out[i] = v;
   }
 }
 
-// One CTA per chunk of 32 compact rows (grid-strided): the chunk's kept rows go to positions chunk_off[ch]...
-// of the ascending kept-row list with their rescale factors 1/(p_n q_r); q and w are written by global row;
-// the rows' operands are packed for the dW product.  The rows of dropped data get w = q = 0, and the compact
-// operands are padded with zero rows to a multiple of 64 (the product's last k-block then adds nothing).
-constexpr int EMIT_THREADS = 128;
+// One CTA per (chunk of 32 compact rows, part) (grid-strided): the chunk's kept rows go to positions
+// chunk_off[ch]... of the ascending kept-row list with their rescale factors 1/(p_n q_r); q and w are written by
+// global row (by part 0); the operands of the chunk's kept rows j with j % parts == part are packed for the dW
+// product.  The rows of dropped data get w = q = 0, and the compact operands are padded with zero rows to a
+// multiple of 64 (the product's last k-block then adds nothing).
+constexpr int EMIT_THREADS = 256;
 __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
   __shared__ int s_r[32], s_pos[32], s_cnt;
   __shared__ float s_sc[32];
@@ -442,8 +455,10 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
   const float c = P.fix[0];
   const int mode = (int)P.fix[1];
   const int nchunks = (n + 31) >> 5;
-  const bool pack = P.packG != nullptr || P.packX != nullptr;
-  for (int ch = blockIdx.x; ch < nchunks; ch += gridDim.x) {
+  const bool pack = P.dst != nullptr;
+  const int parts = pack ? P.parts : 1;
+  for (int u = blockIdx.x; u < nchunks * parts; u += gridDim.x) {
+    const int ch = u / parts, part = u - ch * parts;
     if (warp == 0) {
       const int i = (ch << 5) + lane;
       bool keep = false;
@@ -457,16 +472,14 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
         q = q_of(mode, c, wv, P.q_in, r);
         keep = row_kept(P.sample_w, q, P.sample_w ? P.uc[i] : 0u);
         sa = P.scaleA[nd];
-        P.w[r] = wv;
-        P.q[r] = q;
+        if (part == 0) { P.w[r] = wv; P.q[r] = q; }
       }
       const unsigned b = __ballot_sync(0xffffffffu, keep);
       if (keep) {
         const int j = __popc(b & ((1u << lane) - 1u));
         const int pos = P.chunk_off[ch] + j;
         const float sc = P.sample_w ? sa / q : sa;
-        P.idxW[pos] = r;
-        P.scaleW[pos] = sc;
+        if (part == 0) { P.idxW[pos] = r; P.scaleW[pos] = sc; }
         s_r[j] = r; s_pos[j] = pos; s_sc[j] = sc;
       }
       if (lane == 0) s_cnt = __popc(b);
@@ -474,10 +487,9 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
     if (pack) {
       __syncthreads();
       const int m = s_cnt;
-      for (int j = 0; j < m; ++j) {
+      for (int j = part; j < m; j += parts) {
         const size_t r = (size_t)s_r[j], pos = (size_t)s_pos[j];
-        if (P.packG != nullptr) pack_row(P.dY + r * P.d_out, P.packG + pos * P.d_out, P.d_out, s_sc[j], true);
-        if (P.packX != nullptr) pack_row(P.X + r * P.d_in, P.packX + pos * P.d_in, P.d_in, 1.f, false);
+        pack_row(P.src + r * P.d, P.dst + pos * P.d, P.d, s_sc[j]);
       }
       __syncthreads();
     }
@@ -490,16 +502,14 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
     P.w[r] = 0.f;
     P.q[r] = 0.f;
   }
-  // zero rows up to the next multiple of 64
+  // up to the next multiple of 64: zero rows in the compact operand, and in the list a row that is read anyway
+  // (the first row of a kept datum), so that the product's last k-block adds nothing
   if (pack) {
     const int padded = (cntW + 63) / 64 * 64;
     for (int k = cntW + (int)blockIdx.x; k < padded; k += gridDim.x) {
-      if (P.packG != nullptr)
-        for (int i = tid; i < P.d_out / 8; i += EMIT_THREADS)
-          reinterpret_cast<uint4*>(P.packG + (size_t)k * P.d_out)[i] = make_uint4(0u, 0u, 0u, 0u);
-      if (P.packX != nullptr)
-        for (int i = tid; i < P.d_in / 8; i += EMIT_THREADS)
-          reinterpret_cast<uint4*>(P.packX + (size_t)k * P.d_in)[i] = make_uint4(0u, 0u, 0u, 0u);
+      for (int i = tid; i < P.d / 8; i += EMIT_THREADS)
+        reinterpret_cast<uint4*>(P.dst + (size_t)k * P.d)[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (tid == 0) P.idxW[k] = P.idxA[0] * T;
     }
   }
 }
@@ -583,14 +593,22 @@ cudaError_t launch_emit_pack(Handle* h, const void* dY, const void* X, const Sam
   P.wc = ws.wc; P.uc = ws.uc; P.q_in = a.q_in; P.scaleA = ws.scaleA; P.idxA = ws.idxA; P.dropA = ws.dropA;
   P.counts = ws.counts; P.chunk_off = ws.chunk_off; P.fix = ws.fix;
   P.w = ws.w; P.q = ws.q; P.scaleW = ws.scaleW; P.idxW = ws.idxW;
-  P.dY = (const __nv_bfloat16*)dY; P.X = (const __nv_bfloat16*)X;
-  P.packG = pack ? ws.packG : nullptr;
-  P.packX = pack ? ws.packX : nullptr;
-  P.N = d.N; P.T = d.T; P.d_in = d.d_in; P.d_out = d.d_out;
+  const bool pack_x = h->gather == 1;
+  P.src = pack ? (const __nv_bfloat16*)(pack_x ? X : dY) : nullptr;
+  P.dst = pack ? ws.pack : nullptr;
+  P.d = pack_x ? d.d_in : d.d_out;
+  P.N = d.N; P.T = d.T;
   P.sample_w = a.sample_w;
+  // The number of chunks with kept rows is only known on the device.  With packing, the grid has eight CTAs per
+  // SM and the rows of a chunk are shared among as many CTAs as the expected number of chunks leaves room for.
   const long R = (long)d.N * d.T;
-  long blocks = (R + 31) / 32;
   const long cap = (long)(h->num_sms > 0 ? h->num_sms : 148) * 8;
+  long expected = (long)((double)a.rho * (double)R / 32.0) + 1;
+  long parts = pack ? cap / expected : 1;
+  if (parts < 1) parts = 1;
+  if (parts > 16) parts = 16;
+  P.parts = (int)parts;
+  long blocks = ((R + 31) / 32) * parts;
   if (blocks > cap) blocks = cap;
   const cudaError_t e = launch_after(emit_pack_kernel, dim3((unsigned)blocks), dim3(EMIT_THREADS), 0, st, P);
   h->launches += 1;

@@ -119,10 +119,13 @@ __global__ void __launch_bounds__(256) scores_x_kernel(const T* __restrict__ X, 
   }
 }
 
-int row_grid(const Handle* h, long rows) {
+// One warp per row, eight rows per CTA (the kernels stride over whatever the grid does not cover).  Not a
+// persistent grid: the register count of these kernels leaves room for six or seven CTAs per SM, and a grid of
+// whole waves at an assumed occupancy was measured slower than letting the hardware schedule one CTA per
+// eight rows.
+int row_grid(long rows) {
   long blocks = (rows + 7) / 8;
-  const long cap = (long)(h->num_sms > 0 ? h->num_sms : 148) * 8;     // eight resident CTAs of 256 threads per SM
-  if (blocks > cap) blocks = cap;
+  if (blocks > (1l << 20)) blocks = 1l << 20;
   return (int)(blocks < 1 ? 1 : blocks);
 }
 
@@ -132,7 +135,7 @@ cudaError_t launch_rownorm_dy(Handle* h, const void* dY, const SamplerArgs& s, c
   if (s.a_in != nullptr) return cudaSuccess;     // the producer of dY supplied its row norms
   const vcas_layer_desc& d = h->desc;
   const int R = d.N * d.T;
-  const int blocks = row_grid(h, R);
+  const int blocks = row_grid(R);
   if (d.dtype == VCAS_DTYPE_BF16) {
     rownorm_dy_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dY, R, d.T, d.d_out, s.alive,
                                                              s.alive_cnt, h->ws.a, 1);
@@ -146,7 +149,7 @@ cudaError_t launch_rownorm_dy(Handle* h, const void* dY, const SamplerArgs& s, c
 cudaError_t launch_rownorm_out(Handle* h, const void* dX, float* a_out, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   const int R = d.N * d.T;
-  const int blocks = row_grid(h, R);
+  const int blocks = row_grid(R);
   const int parts = a_out_parts(d.d_in);
   if (d.dtype == VCAS_DTYPE_BF16)
     rownorm_dy_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)dX, R, d.T, d.d_in, nullptr, nullptr,
@@ -165,7 +168,7 @@ cudaError_t launch_scores_x(Handle* h, const void* X, const SamplerArgs& s, bool
   double share = (double)s.rho * 1.5;
   if (share < 0.25) share = 0.25;
   if (share > 1.0) share = 1.0;
-  const int blocks = row_grid(h, (long)(share * (double)d.N * d.T) + 8);
+  const int blocks = row_grid((long)(share * (double)d.N * d.T) + 8);
   const float* a = s.a_in != nullptr ? s.a_in : ws.a;
   const int parts = s.a_in != nullptr ? s.a_parts : 1;
   cudaError_t e;
