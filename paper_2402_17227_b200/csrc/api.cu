@@ -47,7 +47,7 @@ size_t layout(Handle* h, uint8_t* base) {
   w.sorted = carve<float>(cur, N);
   w.idxA = carve<int32_t>(cur, N);
   w.dropA = carve<int32_t>(cur, N);
-  w.idxW = carve<int32_t>(cur, R + 64);
+  w.idxW = carve<int32_t>(cur, R);
   w.chunk_off = carve<int32_t>(cur, chunks);
   w.fix = carve<float>(cur, 4);
   w.counts = carve<int32_t>(cur, 8);
@@ -55,12 +55,14 @@ size_t layout(Handle* h, uint8_t* base) {
   w.acc = carve<double>(cur, 16);
   w.partial = carve<double>(cur, PARTIAL_SLOTS);
   if (h->tensor_path) {
-    w.pack = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * (d.d_in < d.d_out ? d.d_in : d.d_out));
+    w.packG = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_out);
+    w.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
     w.partial_tiles = carve<float>(cur, 3 * (size_t)h->max_units * 128 * 256);
     w.tickets = carve<int32_t>(cur, 6 * (size_t)h->max_units);
     w.sched = carve<int32_t>(cur, 8);
   } else {
-    w.pack = nullptr;
+    w.packG = nullptr;
+    w.packX = nullptr;
     w.partial_tiles = nullptr;
     w.tickets = nullptr;
     w.sched = nullptr;
@@ -82,14 +84,15 @@ size_t layout(Handle* h, uint8_t* base) {
   v.scaleW = carve<float>(cur, R);
   v.idxA = carve<int32_t>(cur, N);
   v.dropA = carve<int32_t>(cur, N);
-  v.idxW = carve<int32_t>(cur, R + 64);
+  v.idxW = carve<int32_t>(cur, R);
   v.chunk_off = carve<int32_t>(cur, chunks);
   v.fix = carve<float>(cur, 4);
   v.counts = carve<int32_t>(cur, 8);
   v.acc = carve<double>(cur, 16);
   v.partial = carve<double>(cur, PARTIAL_SLOTS);
   if (h->tensor_path) {
-    v.pack = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * (d.d_in < d.d_out ? d.d_in : d.d_out));
+    v.packG = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_out);
+    v.packX = carve<__nv_bfloat16>(cur, (size_t)h->R_pad * d.d_in);
     v.partial_tiles = w.partial_tiles + (size_t)h->max_units * 128 * 256;   // dW slot of this set = third slot
     v.tickets = w.tickets + 2 * (size_t)h->max_units;
     v.sched = w.sched + 2;
@@ -114,15 +117,6 @@ int copy_out(Handle* h, float* g, float* p, float* w, float* q, int32_t* idxA, i
   return VCAS_OK;
 }
 
-// dW over the kept rows of the current workspace set: the wider operand's rows are fetched in place by row
-// index, the narrower one is the compact array made by emit_pack_kernel
-cudaError_t launch_sampled_umma_dw(Handle* h, const void* X, const void* dY, int hint, const Plan* plan, float* out,
-                                   cudaStream_t st) {
-  const void* A = h->gather == 1 ? dY : (const void*)h->ws.pack;
-  const void* B = h->gather == 1 ? (const void*)h->ws.pack : X;
-  return launch_umma_dw(h, A, B, h->R_pad, h->ws.idxW, h->gather, h->ws.counts + 1, hint, plan, out, st);
-}
-
 // SampleW, the kept-row list with its compact operands, and dW over those rows into `out`; follows SampleA
 // on the workspace set that h->ws currently names.  first_programmatic: the first kernel is launched as a
 // dependent of the kernel before it in `st` (false when its inputs arrive through an event).
@@ -134,7 +128,7 @@ int sample_w_and_dw(Handle* h, const void* X, const void* dY, const SamplerArgs&
   if (h->tensor_path) {
     const float keep = a.sample_w ? a.rho * a.nu : a.rho;
     const int hint = (int)(keep * (float)(h->desc.N * h->desc.T)) + 1;
-    VCAS_CUDA(launch_sampled_umma_dw(h, X, dY, hint, plan, out, st));
+    VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, plan, out, st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, out, st));
   }
@@ -152,8 +146,7 @@ inline void mark_dense(Handle* h, int k, cudaStream_t st) {
 // plan: the tiling made for a call whose dX product runs beside it (nullptr: planned alone)
 int dense_dw(Handle* h, const void* X, const void* dY, const Plan* plan, float* out, cudaStream_t st) {
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, nullptr, 0, h->ws.counts + 2, h->desc.N * h->desc.T, plan, out,
-                             st));
+    VCAS_CUDA(launch_umma_dw(h, dY, X, h->desc.N * h->desc.T, h->ws.counts + 2, h->desc.N * h->desc.T, plan, out, st));
   } else {
     VCAS_CUDA(launch_fma_dw(h, dY, X, nullptr, nullptr, h->ws.counts + 2, out, st));
   }
@@ -195,7 +188,6 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   if (cfg != nullptr) h->cfg = *cfg; else vcas_default_config(&h->cfg);
   h->tensor_path = tensor_ok && desc->gemm_path != VCAS_GEMM_FMA;
   h->R_pad = (desc->N * desc->T + 63) / 64 * 64;
-  h->gather = desc->d_out >= desc->d_in ? 1 : 2;
   h->launches = 0;
   h->prof_enabled = false;
   h->ev = nullptr;
@@ -298,7 +290,7 @@ int run_sampled(Handle* h, const void* X, const void* dY, const void* W, const S
     VCAS_CUDA(launch_emit_pack(h, dY, X, a, h->tensor_path, st));
     mark(h, 4, st);
     if (h->tensor_path) {
-      VCAS_CUDA(launch_sampled_umma_dw(h, X, dY, hint, &pw, dW, st));
+      VCAS_CUDA(launch_umma_dw(h, h->ws.packG, h->ws.packX, h->R_pad, h->ws.counts + 1, hint, &pw, dW, st));
     } else {
       VCAS_CUDA(launch_fma_dw(h, dY, X, h->ws.idxW, h->ws.scaleW, h->ws.counts + 1, dW, st));
     }

@@ -27,7 +27,7 @@ struct Workspace {
   float* sorted;   // [N]  data norms in descending order (Eq. 4)
   int32_t* idxA;   // [N]  kept data, ascending
   int32_t* dropA;  // [N]  dropped data, ascending
-  int32_t* idxW;   // [R_pad]  kept rows, ascending, padded to a multiple of 64 with a kept datum's first row
+  int32_t* idxW;   // [R]  kept rows, ascending
   int32_t* chunk_off;  // [R/32 + 2] position in idxW of the first kept row of every chunk of 32 compact rows
   float* fix;      // [4]  0: the factor c of q = min(1, c w) found by the water-filling, 1: mode (see sample_w_kernel)
   int32_t* counts; // [8]  0: cntA, 1: cntW, 2: R (constant, for dense launches), 4: reduction ticket
@@ -35,7 +35,8 @@ struct Workspace {
   double* acc;     // [16] probe accumulators (0: V_act, 1: V_w, 2: p_lo, 3: p_hi, 4: V_s)
   double* partial; // [PARTIAL_SLOTS] block partial sums of the probe reductions
   // compact operands of the weight-gradient product (tensor path)
-  __nv_bfloat16* pack;   // [R_pad, min(d_in, d_out)] the narrower operand's kept rows times 1/(p q), compact
+  __nv_bfloat16* packG;  // [R_pad, d_out]
+  __nv_bfloat16* packX;  // [R_pad, d_in]
   float* partial_tiles;  // [3][max_units][128 * 256] fp32 partial tiles of a split contraction: dX, dW, and the dW
                          // of the workspace's second set (see Handle::ws2)
   int32_t* tickets;      // [3][2 * max_units]: slices stored, slices finished, per tile
@@ -61,7 +62,6 @@ struct Handle {
   int num_sms;
   bool tensor_path;
   int R_pad;
-  int gather;      // sampled dW product: 1 = dY rows fetched by TMA gather and X packed (d_out >= d_in), 2 = the reverse
   int max_units;   // capacity of the split-contraction workspace, in (tile, slice) units
   void* base;
   size_t bytes;
@@ -323,7 +323,7 @@ cudaError_t launch_scores_x(Handle* h, const void* X, const SamplerArgs& a, bool
 // SampleW (Sec. 4.2): the factor c of q = min(1, c w), the masks' counts per chunk of 32 compact rows
 cudaError_t launch_sample_w(Handle* h, const SamplerArgs& a, cudaStream_t st);
 // kept-row list, 1/(p q), q and w by global row and, with pack, the compact bf16 operands of the dW product
-cudaError_t launch_emit_pack(Handle* h, const void* dY, const void* X, const SamplerArgs& a, bool pack, cudaStream_t st);   // pack: the narrower of dY / X
+cudaError_t launch_emit_pack(Handle* h, const void* dY, const void* X, const SamplerArgs& a, bool pack, cudaStream_t st);
 cudaError_t launch_mask_from_probs(Handle* h, const float* p, int n, uint64_t seed, int sampler,
                                    uint8_t* keep, int32_t* idx, int32_t* cnt, cudaStream_t st);
 
@@ -341,12 +341,10 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
                            const void* H, void* dX, float* a_out, int spare_sms, const Plan* pair_plan, cudaStream_t st);
 inline int a_out_parts(int d_in) { return (d_in + 255) / 256; }
-// dW = A_rows^T B_rows over *cnt rows (bf16).  gather = 0: A_rows [rows_capacity, d_out] and B_rows
-// [rows_capacity, d_in] are compact; gather = 1 / 2: A_rows / B_rows is the original [R, .] tensor and row k of
-// the contraction is its row gidx[k] (the other operand is compact and carries the rescale factors).
+// dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling
-cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity, const int32_t* gidx,
-                           int gather, const int32_t* cnt, int cnt_hint, const Plan* pair_plan, float* dW, cudaStream_t st);
+cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity,
+                           const int32_t* cnt, int cnt_hint, const Plan* pair_plan, float* dW, cudaStream_t st);
 // Tilings of the dX and dW products of one call, chosen together because they share the SMs (cached in the
 // handle until the expected kept counts or the tuning overrides change).
 // row_norms_out: the dX product must emit row square-norms from its epilogue (unsliced 256-wide tiles only)

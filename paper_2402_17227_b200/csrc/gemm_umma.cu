@@ -101,16 +101,6 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, i
       ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
 }
 
-// Four rows of a 2-D tensor, given by their row indices, 64 columns (128 bytes) each, land as four consecutive
-// 128-byte rows at dst (the tensor map's box is one row high; the 128-byte swizzle follows the shared-memory
-// address, so pieces placed 512 bytes apart compose the same layout as one tiled load of the rows).
-__device__ __forceinline__ void tma_gather4(void* dst, const CUtensorMap* map, int col, const int4& rows, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(col), "r"(rows.x), "r"(rows.y), "r"(rows.z), "r"(rows.w), "r"(smem_u32(bar))
-      : "memory");
-}
-
 // ---- asynchronous bulk stores (shared -> global), tracked in per-thread bulk groups
 __device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, uint32_t bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(ssrc)), "r"(bytes) : "memory");
@@ -291,11 +281,7 @@ struct GemmParams {
   int N, T;
   int dense;               // 1: every datum kept with scale 1
   int a_tx_bytes;          // bytes one A box delivers (min(T, 128) token rows of 128 B)
-  // dW: A = rows x d_out, B = rows x d_in (both MN-major).  gather = 0: both operands are compact arrays of
-  // rows; 1 / 2: the A / B operand is the original tensor, whose kept rows gidx[k] are fetched by TMA gather,
-  // and the other operand is a compact array that carries the rescale factors.
-  const int32_t* gidx;     // kept rows (ascending), padded to a multiple of 64 with a valid row
-  int gather;
+  // dW: A = rows x d_out, B = rows x d_in (both MN-major, gathered along k by the pack step)
   const int32_t* cnt;      // number of valid rows (the contraction length)
   float* dW;               // [d_out, d_in]
 };
@@ -413,88 +399,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const Decomp D = decompose<MODE, BN, MH, LEAN>(P);
   const int total_items = D.units + D.zero_tiles;     // unsliced instances: product tiles, then zero tiles
 
-  if (warp == 4 && MODE == MODE_DW && P.gather != 0) {
-    // ------------------------------------------- TMA producer, one operand gathered by row index (whole warp)
-    // Lane 0 waits for the stage, posts the expected bytes and loads the compact operand; then every lane
-    // issues gathers of four rows each for the other operand: lane l fetches rows 4 (l % 16) ... + 3 of the
-    // k-block for the 64-column chunks l / 16, l / 16 + 2, ...  The row indices of the next k-block are
-    // requested while this one is issued.
-    int stage = 0; uint32_t phase = 0;
-    bool ok = true;
-    int qi = 0; uint32_t qph = 0;
-    auto next_unit = [&](int prev) -> int {
-      int t = -1;
-      if (lane == 0) {
-        if constexpr (DYN) {
-          if (!mbar_wait(&s.q_empty[qi], qph ^ 1u, abort_flag, P.status)) {
-            ok = false;
-          } else {
-            t = atomicAdd(P.sched, 1);
-            if (t >= D.units + D.zero_tiles) t = -1;
-            *(volatile int*)&s.tile_q[qi] = t;
-            mbar_arrive(&s.q_full[qi]);
-          }
-        } else if constexpr (LEAN) {
-          const int u = prev < 0 ? (int)blockIdx.x : prev + (int)gridDim.x;
-          t = u < total_items ? u : -1;
-        } else {
-          const int u = prev < 0 ? (int)blockIdx.x : prev + D.upi;
-          t = ((int)blockIdx.x < D.upi && u < D.units) ? u : -1;
-        }
-      }
-      if constexpr (DYN) { if (++qi == QD) { qi = 0; qph ^= 1u; } }
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      return __shfl_sync(0xffffffffu, t, 0);
-    };
-    const int g4 = lane & 15, jh = lane >> 4;
-    const int4* gi = reinterpret_cast<const int4*>(P.gidx);
-    for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
-      if (LEAN && u >= D.units) continue;    // a zero tile: nothing to load
-      const int tile = u / D.S, slice = u % D.S;
-      const int kb0 = slice * D.kb_per;
-      const int kb1 = min(D.kblocks, kb0 + D.kb_per);
-      int k, c0, c1;
-      tile_coords<MODE>(P, D, tile, k, c0, c1);
-      int4 rows = kb0 < kb1 ? __ldg(gi + kb0 * 16 + g4) : make_int4(0, 0, 0, 0);
-      for (int kb = kb0; kb < kb1; ++kb) {
-        const int4 rows_next = kb + 1 < kb1 ? __ldg(gi + (kb + 1) * 16 + g4) : rows;
-        uint8_t* sa = s.stages + stage * C::STAGE_BYTES;
-        int okl = 1;
-        if (lane == 0) {
-          okl = mbar_wait(&s.empty[stage], phase ^ 1u, abort_flag, P.status) ? 1 : 0;
-          if (okl) {
-            mbar_expect_tx(&s.full[stage], C::STAGE_BYTES);
-            if (P.gather == 1) {
-#pragma unroll
-              for (int j = 0; j < BN / 64; ++j)
-                tma_load_2d(sa + C::AT_BYTES + j * CHUNK_BYTES, &tmB, c1 * BN + j * 64, kb * BK, &s.full[stage]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < BMT / 64; ++j)
-                tma_load_2d(sa + j * CHUNK_BYTES, &tmA, c0 * BMT + j * 64, kb * BK, &s.full[stage]);
-            }
-          }
-        }
-        ok = __shfl_sync(0xffffffffu, okl, 0) != 0;
-        if (!ok) break;
-        if (P.gather == 1) {
-          for (int j = jh; j < BMT / 64; j += 2)
-            tma_gather4(sa + j * CHUNK_BYTES + g4 * 512, &tmA, c0 * BMT + j * 64, rows, &s.full[stage]);
-        } else {
-          for (int j = jh; j < BN / 64; j += 2)
-            tma_gather4(sa + C::AT_BYTES + j * CHUNK_BYTES + g4 * 512, &tmB, c1 * BN + j * 64, rows, &s.full[stage]);
-        }
-        rows = rows_next;
-        if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
-      }
-    }
-    if constexpr (DYN) {
-      if (ok && lane == 0) {        // the last CTA to run out of work re-arms the counters for the next launch
-        __threadfence();
-        if (atomicAdd(P.sched + 1, 1) == (int)gridDim.x - 1) { P.sched[0] = 0; P.sched[1] = 0; }
-      }
-    }
-  } else if (warp == 4) {
+  if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
@@ -1240,24 +1145,20 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   return run_gemm_bn<MODE_DX>(h, plan, tmA, tmB, tmC, P, max_items, ctas, true, st);
 }
 
-cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity, const int32_t* gidx,
-                           int gather, const int32_t* cnt, int cnt_hint, const Plan* pair_plan, float* dW, cudaStream_t st) {
+cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity, const int32_t* cnt,
+                           int cnt_hint, const Plan* pair_plan, float* dW, cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
-  const int R = d.N * d.T;
   {
-    // gathered: the original [R, d_out] tensor, one row of 64 columns per box (four rows per gather)
-    const bool g = gather == 1;
-    const uint64_t dims[2] = {(uint64_t)d.d_out, (uint64_t)(g ? R : rows_capacity)};
+    const uint64_t dims[2] = {(uint64_t)d.d_out, (uint64_t)rows_capacity};
     const uint64_t strides[1] = {(uint64_t)d.d_out * 2};
-    const uint32_t box[2] = {64, (uint32_t)(g ? 1 : BK)};
+    const uint32_t box[2] = {64, BK};
     if (!make_map(&tmA, A_rows, 2, dims, strides, box)) return cudaErrorInvalidValue;
   }
   {
-    const bool g = gather == 2;
-    const uint64_t dims[2] = {(uint64_t)d.d_in, (uint64_t)(g ? R : rows_capacity)};
+    const uint64_t dims[2] = {(uint64_t)d.d_in, (uint64_t)rows_capacity};
     const uint64_t strides[1] = {(uint64_t)d.d_in * 2};
-    const uint32_t box[2] = {64, (uint32_t)(g ? 1 : BK)};
+    const uint32_t box[2] = {64, BK};
     if (!make_map(&tmB, B_rows, 2, dims, strides, box)) return cudaErrorInvalidValue;
   }
   {
@@ -1269,7 +1170,6 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
   GemmParams P;
   common_params(h, P, 1);
   P.cnt = cnt; P.dW = dW;
-  P.gidx = gidx; P.gather = gidx != nullptr ? gather : 0;
   const long mtiles = (d.d_out + BM - 1) / BM, mtiles2 = (d.d_out + 2 * BM - 1) / (2 * BM);
   Plan plan;
   if (pair_plan != nullptr) {

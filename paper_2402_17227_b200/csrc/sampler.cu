@@ -397,17 +397,15 @@ struct EmitParams {
   const int32_t* idxA; const int32_t* dropA;
   const int32_t* counts; const int32_t* chunk_off; const float* fix;
   float* w; float* q; float* scaleW; int32_t* idxW;
-  const __nv_bfloat16* src;  // the operand to pack, [R, d] (the narrower of dY and X), or nullptr
-  __nv_bfloat16* dst;        // [R_pad, d]: row k = src[idxW[k]] / (p q), rounded to bf16
-  int d;
-  int N, T;
+  const __nv_bfloat16* dY; const __nv_bfloat16* X;       // operands to pack
+  __nv_bfloat16* packG; __nv_bfloat16* packX;            // compact operands (nullptr: no packing)
+  int N, T, d_in, d_out;
   int sample_w;
   int parts;                                             // CTAs that share the packing of one chunk's rows
 };
 
-// Row k of the compact operand = scaleW[k] * src[idxW[k]], rounded to bf16: the factor 1/(p q) of G_tilde
-// (Sec. 4.2) sits on the contraction axis of G_tilde^T X, so it may scale either operand's row; it scales the
-// narrower one, and the other is read in place.  Four independent 16-byte loads per thread are in flight.
+// Row k of packG = scaleW[k] * dY[idxW[k]] (G_tilde of Sec. 4.2, rounded to bf16), row k of packX = X[idxW[k]].
+// Four independent 16-byte loads per thread are in flight.
 __device__ __forceinline__ uint4 scale8(const uint4& v, float sc) {
   const uint32_t u[4] = {v.x, v.y, v.z, v.w};
   uint32_t o[4];
@@ -419,8 +417,7 @@ __device__ __forceinline__ uint4 scale8(const uint4& v, float sc) {
   return make_uint4(o[0], o[1], o[2], o[3]);
 }
 __device__ __forceinline__ void pack_row(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int d,
-                                         float sc) {
-  constexpr bool scaled = true;
+                                         float sc, bool scaled) {
   const uint4* __restrict__ in = reinterpret_cast<const uint4*>(src);
   uint4* __restrict__ out = reinterpret_cast<uint4*>(dst);
   const int nv = d / 8, nt = blockDim.x;
@@ -455,7 +452,7 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
   const float c = P.fix[0];
   const int mode = (int)P.fix[1];
   const int nchunks = (n + 31) >> 5;
-  const bool pack = P.dst != nullptr;
+  const bool pack = P.packG != nullptr;
   const int parts = pack ? P.parts : 1;
   for (int u = blockIdx.x; u < nchunks * parts; u += gridDim.x) {
     const int ch = u / parts, part = u - ch * parts;
@@ -489,7 +486,8 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
       const int m = s_cnt;
       for (int j = part; j < m; j += parts) {
         const size_t r = (size_t)s_r[j], pos = (size_t)s_pos[j];
-        pack_row(P.src + r * P.d, P.dst + pos * P.d, P.d, s_sc[j]);
+        pack_row(P.dY + r * P.d_out, P.packG + pos * P.d_out, P.d_out, s_sc[j], true);
+        pack_row(P.X + r * P.d_in, P.packX + pos * P.d_in, P.d_in, 1.f, false);
       }
       __syncthreads();
     }
@@ -502,14 +500,14 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
     P.w[r] = 0.f;
     P.q[r] = 0.f;
   }
-  // up to the next multiple of 64: zero rows in the compact operand, and in the list a row that is read anyway
-  // (the first row of a kept datum), so that the product's last k-block adds nothing
+  // zero rows up to the next multiple of 64
   if (pack) {
     const int padded = (cntW + 63) / 64 * 64;
     for (int k = cntW + (int)blockIdx.x; k < padded; k += gridDim.x) {
-      for (int i = tid; i < P.d / 8; i += EMIT_THREADS)
-        reinterpret_cast<uint4*>(P.dst + (size_t)k * P.d)[i] = make_uint4(0u, 0u, 0u, 0u);
-      if (tid == 0) P.idxW[k] = P.idxA[0] * T;
+      for (int i = tid; i < P.d_out / 8; i += EMIT_THREADS)
+        reinterpret_cast<uint4*>(P.packG + (size_t)k * P.d_out)[i] = make_uint4(0u, 0u, 0u, 0u);
+      for (int i = tid; i < P.d_in / 8; i += EMIT_THREADS)
+        reinterpret_cast<uint4*>(P.packX + (size_t)k * P.d_in)[i] = make_uint4(0u, 0u, 0u, 0u);
     }
   }
 }
@@ -593,11 +591,10 @@ cudaError_t launch_emit_pack(Handle* h, const void* dY, const void* X, const Sam
   P.wc = ws.wc; P.uc = ws.uc; P.q_in = a.q_in; P.scaleA = ws.scaleA; P.idxA = ws.idxA; P.dropA = ws.dropA;
   P.counts = ws.counts; P.chunk_off = ws.chunk_off; P.fix = ws.fix;
   P.w = ws.w; P.q = ws.q; P.scaleW = ws.scaleW; P.idxW = ws.idxW;
-  const bool pack_x = h->gather == 1;
-  P.src = pack ? (const __nv_bfloat16*)(pack_x ? X : dY) : nullptr;
-  P.dst = pack ? ws.pack : nullptr;
-  P.d = pack_x ? d.d_in : d.d_out;
-  P.N = d.N; P.T = d.T;
+  P.dY = (const __nv_bfloat16*)dY; P.X = (const __nv_bfloat16*)X;
+  P.packG = pack ? ws.packG : nullptr;
+  P.packX = pack ? ws.packX : nullptr;
+  P.N = d.N; P.T = d.T; P.d_in = d.d_in; P.d_out = d.d_out;
   P.sample_w = a.sample_w;
   // The number of chunks with kept rows is only known on the device.  With packing, the grid has eight CTAs per
   // SM and the rows of a chunk are shared among as many CTAs as the expected number of chunks leaves room for.
