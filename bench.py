@@ -256,7 +256,7 @@ def point_report(case, rho, nu, kA, kW, t_s, t_d, per, pk):
     """One (rho, nu) point in the layout of the report: kept rows, times, achieved rates and fractions."""
     R, d_in, d_out = case.R, case.d_in, case.d_out
     b = 4 if str(case.dtype).endswith("float32") else 2
-    score_bytes = R * (d_in + d_out) * b
+    score_bytes = R * d_out * b                 # the first pass reads every row of dY once (X: kept rows only, later)
     flops_ratio = 2.0 * R / max(1.0, kA + kW)
     rate = lambda work, ms: (work / ms / 1e9) if ms and ms > 0 else None
     out = {
@@ -281,8 +281,10 @@ def point_report(case, rho, nu, kA, kW, t_s, t_d, per, pk):
     return out
 
 
-def measure_layer(case, vb, inputs, torch, dev, pk, ratios, seeds, profile=True, tensors=None, layer=None):
-    """Sampled and dense backward of one layer at several (rho, nu): per call and per stage."""
+def measure_layer(case, vb, inputs, torch, dev, pk, ratios, seeds, profile=True, tensors=None, layer=None,
+                  graph=False):
+    """Sampled and dense backward of one layer at several (rho, nu): per call and per stage.  graph: the timed
+    calls are replayed from a CUDA graph (for layers so small that the host's launch cost would bound them)."""
     N, T, d_in, d_out, R = case.N, case.T, case.d_in, case.d_out, case.R
     if tensors is None:
         tensors = [t.to(dev) for t in inputs.make_layer(case)]
@@ -295,27 +297,29 @@ def measure_layer(case, vb, inputs, torch, dev, pk, ratios, seeds, profile=True,
     out = {"N": N, "T": T, "d_in": d_in, "d_out": d_out, "seeds_per_point": len(seeds),
            "workspace_bytes": layer.workspace_bytes(), "points": []}
     n = len(seeds)
-    for _ in range(3):
-        layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
-    torch.cuda.synchronize()
-    e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    e[0].record()
-    for _ in seeds:
-        layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
-    e[1].record()
-    torch.cuda.synchronize()
-    t_d = e[0].elapsed_time(e[1]) / n
-    for rho, nu in ratios:
+
+    def time_calls(fn):
+        """ms per call of fn(seed) over the seeds (eager launches, or one CUDA graph of all of them replayed)."""
         for sd in seeds[:3]:
-            layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
+            fn(sd)
+        torch.cuda.synchronize()
+        run = lambda: [fn(sd) for sd in seeds]
+        if graph:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                run()
+            run = g.replay
+            run()
         torch.cuda.synchronize()
         e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
         e[0].record()
-        for sd in seeds:
-            layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW)
+        run()
         e[1].record()
         torch.cuda.synchronize()
-        t_s = e[0].elapsed_time(e[1]) / n
+        return e[0].elapsed_time(e[1]) / n
+    t_d = time_calls(lambda sd: layer.dense_bwd(X, dY, W, dX=dX, dW=dW))
+    for rho, nu in ratios:
+        t_s = time_calls(lambda sd: layer.linear_bwd_plain(X, dY, W, rho, nu, sd, dX, dW))
         per = None
         if profile:
             def cs():
@@ -396,7 +400,7 @@ def measure_bert_base_with_probe(vb, inputs, torch, dev, pk):
     t_calls = ms_of(g_calls.replay, 10)
     t_dense = ms_of(g_dense.replay, 10)
     pt = measure_layer(case, vb, inputs, torch, dev, pk, [(case.rho, case.nu)], list(range(16)),
-                       tensors=(Xs[0], dYs[0], W), layer=layer)
+                       tensors=(Xs[0], dYs[0], W), layer=layer, graph=True)
     pt.update({"ms_per_layer_with_probe_every_100_calls": t_period / F, "sampled_call_ms_graph_replay": t_calls / F,
                "dense_call_ms_graph_replay": t_dense / F, "probe_M": M,
                "speedup_vs_dense_graph_replay": t_dense / t_calls})
@@ -457,6 +461,186 @@ def measure_vit_block(vb, inputs, torch, dev, pk):
             "note": "dense block: exact products of both linears, without the GELU Jacobian"}
 
 
+def measure_bert_large_stack(vb, inputs, torch, dev, steps=200, F=50, M=2):
+    """The 96 linears of a 24-block BERT-large-shaped stack (N=32, T=512, d=1024: QKV 1024->3072, attention output
+    1024->1024, FFN 1024->4096->1024 with the GELU Jacobian fused), backward from the top layer down with the
+    chain entry point: every layer receives the list of data the layer above kept, the FFN pair hands its row
+    norms down from the dX epilogue.  Keep ratios start at rho_l = 0.8 (top) ... 0.2 (bottom), nu = 0.3; every F
+    steps Alg. 1 probes every layer (M batches) and updates (s, rho_l, nu_l); the passes of a period are replayed from
+    a CUDA graph.  QKV and the attention output have
+    no attention between them here, so each linear has its own synthetic incoming gradient; all blocks share one
+    pool of activations and gradients per shape (two variants), with their own random weights."""
+    import numpy as np
+    from paper_2402_17227_b200.stack import LinearStack, StackLayer
+    N, T, d, ffn, qkv, blocks = 32, 512, 1024, 4096, 3072, 24
+    bf = torch.bfloat16
+    cfg = vb.default_config()
+    cfg.F, cfg.M = F, M
+    cfg.rho_min, cfg.nu_min = 1.0 / N, 1e-3
+    specs = [("ffn_down", ffn, d, True, False), ("ffn_up", d, ffn, False, True), ("attn_out", d, d, False, False),
+             ("qkv", d, qkv, False, False)]
+    pool = {}
+    for k, (name, d_in, d_out, gelu, chained) in enumerate(specs):
+        c = inputs.LayerCase(name, N, T, d_in, d_out, bf, 1.0, 0.5, 0.5, 0.3, data_seed=4000 + k)
+        batches = [inputs.make_layer(c, batch=b, device=dev) for b in range(M)]
+        Xs, H = [b[0] for b in batches], None
+        if gelu:
+            H = [inputs.make_preactivation(c, batch=b, width=d_in, device=dev) for b in range(M)]
+            Xs = [torch.nn.functional.gelu(h.float()).to(bf) for h in H]
+        pool[name] = (Xs, [b[1] for b in batches], H)
+    gw = torch.Generator(dev).manual_seed(99)
+    layers = []
+    for blk in range(blocks - 1, -1, -1):
+        for name, d_in, d_out, gelu, chained in specs:
+            W = (torch.randn(d_out, d_in, generator=gw, device=dev, dtype=torch.float32) * 0.02).to(bf)
+            Xs, dYs, H = pool[name]
+            layers.append(StackLayer(f"b{blk}.{name}", d_in, d_out, W, Xs, dYs, H=H, chained=chained))
+    stack = LinearStack(layers, N, T, config=cfg)
+    L = len(layers)
+    # Alg. 1's state in layer order (index 0 = lowest layer); the stack runs in backward order (top first)
+    state = dict(s=0.75, rho=list(np.linspace(0.2, 0.8, L)), nu=[0.3] * L)
+    traj = []
+
+    def adapt(t):
+        V = stack.probe(state["rho"][::-1], state["nu"][::-1], state["s"], seed=31 * t).cpu().numpy()[::-1]
+        s, rho, nu = vb.update_ratios(state["s"], state["rho"], state["nu"], V[:, 0], V[:, 1], V[:, 2], V[:, 3],
+                                      V[:, 4], cfg)
+        state.update(s=s, rho=rho, nu=nu)
+        traj.append({"t": t, "s": s, "rho_bottom": rho[0], "rho_top": rho[-1], "nu_min": min(nu), "nu_max": max(nu)})
+
+    PASSES = 5          # passes (with their own seeds and batch variants) captured into one CUDA graph
+
+    def capture(t0):
+        # The ratios only change when Alg. 1 adapts them, so the passes of a period are captured once into a CUDA
+        # graph (the library neither synchronises nor allocates) and replayed: the host's launch cost of 96 calls
+        # of about eight kernels each would otherwise bound the step.
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for k in range(PASSES):
+                stack.backward(state["rho"][::-1], state["nu"][::-1], seed=t0 + k, variant=t0 + k)
+        return g
+
+    def run_period(t0, n):
+        adapt(t0)
+        g = capture(t0)
+        for _ in range(n // PASSES):
+            g.replay()
+        return g
+    for t in range(3):                          # warm-up at the initial ratios
+        stack.backward(state["rho"][::-1], state["nu"][::-1], seed=t, variant=t)
+    stack.dense_backward()
+    torch.cuda.synchronize()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+    e[0].record()
+    g_last = None
+    for t0 in range(0, steps, F):
+        g_last = run_period(t0, F)
+    e[1].record()
+    torch.cuda.synchronize()
+    ms_step = e[0].elapsed_time(e[1]) / steps
+    # at the final ratios: sampled passes alone (graph replay and eager launches), dense passes (graph replay)
+    g_dense = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_dense):
+        for k in range(PASSES):
+            stack.dense_backward(variant=k)
+    torch.cuda.synchronize()
+    reps = 4
+    e[1].record()
+    for _ in range(reps):
+        g_last.replay()
+    e[2].record()
+    for _ in range(reps):
+        g_dense.replay()
+    e[3].record()
+    for t in range(PASSES):
+        stack.backward(state["rho"][::-1], state["nu"][::-1], seed=10_000 + t, variant=t)
+    e[4].record()
+    torch.cuda.synchronize()
+    ms_sampled = e[1].elapsed_time(e[2]) / (reps * PASSES)
+    ms_dense = e[2].elapsed_time(e[3]) / (reps * PASSES)
+    ms_sampled_eager = e[3].elapsed_time(e[4]) / PASSES
+    ev, kept = [], []
+
+    def hook(i, lay, after):
+        x = torch.cuda.Event(enable_timing=True)
+        x.record()
+        ev.append(x)
+        if after:
+            smp = lay.handle.last_sampling()
+            kept.append((lay.name.split(".")[1], smp.cntA * T, smp.cntW, lay.d_in * lay.d_out))
+    by_type, dense_by_type = {}, {}
+    for rep in range(3):
+        ev.clear()
+        stack.backward(state["rho"][::-1], state["nu"][::-1], seed=20_000 + rep, variant=rep, hook=hook)
+        torch.cuda.synchronize()
+        for i, lay in enumerate(layers):
+            k = lay.name.split(".")[1]
+            by_type[k] = by_type.get(k, 0.0) + ev[2 * i].elapsed_time(ev[2 * i + 1]) / 3
+    ev2 = []
+
+    def hook2(i, lay, after):
+        x = torch.cuda.Event(enable_timing=True)
+        x.record()
+        ev2.append(x)
+    stack.dense_backward(hook=hook2)
+    torch.cuda.synchronize()
+    for i, lay in enumerate(layers):
+        k = lay.name.split(".")[1]
+        dense_by_type[k] = dense_by_type.get(k, 0.0) + ev2[2 * i].elapsed_time(ev2[2 * i + 1])
+    flops_dense = sum(2.0 * 2.0 * N * T * lay.d_in * lay.d_out for lay in layers)
+    flops_sampled = sum(2.0 * (a + w) * dd for _, a, w, dd in kept) / 3
+    out = {
+        "N": N, "T": T, "d": d, "blocks": blocks, "linears": L, "steps": steps, "F": F, "M": M,
+        "ms_per_step_with_probes": ms_step, "ms_per_step_sampled_at_final_ratios": ms_sampled,
+        "ms_per_step_sampled_eager_launches": ms_sampled_eager,
+        "ms_per_step_dense": ms_dense, "speedup_vs_dense": ms_dense / ms_sampled,
+        "speedup_vs_dense_with_probes": ms_dense / ms_step,
+        "flops_reduction_ratio": flops_dense / max(1.0, flops_sampled),
+        "speedup_over_flops_ratio": (ms_dense / ms_sampled) / (flops_dense / max(1.0, flops_sampled)),
+        "dense_tflops": flops_dense / ms_dense / 1e9,
+        "ms_per_step_by_layer_type_sampled": by_type, "ms_per_step_by_layer_type_dense": dense_by_type,
+        "kept_rows_mean_by_type": {k: {"kept_A": float(np.mean([a for n_, a, w, _ in kept if n_ == k])),
+                                       "kept_W": float(np.mean([w for n_, a, w, _ in kept if n_ == k]))}
+                                   for k in by_type},
+        "initial": {"s": 0.75, "rho_top": 0.8, "rho_bottom": 0.2, "nu": 0.3},
+        "trajectory": traj, "final": {"s": state["s"], "rho": [round(float(x), 4) for x in state["rho"]],
+                                      "nu": [round(float(x), 4) for x in state["nu"]]},
+        "workspace_bytes": stack.workspace_bytes(), "handles": len(stack.handles),
+    }
+    assert stack.device_status() == 0
+    stack.close()
+    return out
+
+
+def kernel_run(args):
+    """A small run for profilers: `--kernel-run WORKLOAD` makes 2 warm-up + `--calls` sampled backward calls and as
+    many dense ones of one workload at (--rho, --nu), inputs drawn on the device, and prints one JSON line."""
+    import torch
+    from paper_2402_17227_b200 import binding as vb
+    from paper_2402_17227_b200 import build as vbuild
+    from paper_2402_17227_b200 import inputs
+    vbuild.build()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    case = inputs.CASES[args.kernel_run]
+    X, dY, W = inputs.make_layer(case, device=dev)
+    layer = vb.Layer(case.N, case.T, case.d_in, case.d_out, case.dtype)
+    dX = torch.empty(case.R, case.d_in, dtype=case.dtype, device=dev)
+    dW = torch.empty(case.d_out, case.d_in, dtype=torch.float32, device=dev)
+    for k in range(2 + args.calls):
+        layer.linear_bwd_plain(X, dY, W, args.rho, args.nu, k, dX, dW)
+    torch.cuda.synchronize()
+    l0 = layer.launch_count()
+    for k in range(args.calls):
+        layer.dense_bwd(X, dY, W, dX=dX, dW=dW)
+    torch.cuda.synchronize()
+    smp = layer.last_sampling()
+    print(json.dumps({"workload": case.name, "rho": args.rho, "nu": args.nu, "calls": args.calls,
+                      "kept_A": smp.cntA * case.T, "kept_W": smp.cntW, "launches_sampled": l0,
+                      "status": layer.device_status()}))
+    layer.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -467,7 +651,14 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the workloads reported under other_workloads")
     ap.add_argument("--sweep", default="grid", choices=["grid", "diag"],
                     help="ratio sweep on the headline layer: the 5 x 5 grid of (rho, nu), or its diagonal only")
+    ap.add_argument("--kernel-run", default=None, metavar="WORKLOAD",
+                    help="profiling aid: a few sampled and dense calls of one workload, nothing else")
+    ap.add_argument("--rho", type=float, default=RHO)
+    ap.add_argument("--nu", type=float, default=NU)
+    ap.add_argument("--calls", type=int, default=2)
     args = ap.parse_args()
+    if args.kernel_run is not None:
+        return kernel_run(args)
     if args.impl == "reference":
         return run_reference(args)
     args.warmup = max(args.warmup, 3)
@@ -623,9 +814,12 @@ def main():
         del Xs, dYs, host
         torch.cuda.empty_cache()
         extra["fp32_small"] = measure_layer(inputs.CASES["fp32_small"], vb, inputs, torch, dev, pk, [(0.5, 0.5)],
-                                            list(range(50)))
+                                            list(range(50)), graph=True)
         extra["bert_base_ffn_up"] = measure_bert_base_with_probe(vb, inputs, torch, dev, pk)
         extra["vit_base_mlp_block"] = measure_vit_block(vb, inputs, torch, dev, pk)
+        torch.cuda.empty_cache()
+        extra["bert_large_stack"] = measure_bert_large_stack(vb, inputs, torch, dev)
+        torch.cuda.empty_cache()
         # a BERT-large FFN linear at the keep ratios of a top, a middle and a bottom layer
         extra["bert_large_ffn_up"] = measure_layer(inputs.CASES["bert_large_ffn_up"], vb, inputs, torch, dev, pk,
                                                    [(0.8, 0.3), (0.5, 0.3), (0.2, 0.3)], list(range(20)))
@@ -636,7 +830,7 @@ def main():
         return
 
     names = ["rownorm_kernel", "sampler_kernel", "umma_dx_kernel", "pack_kernel", "umma_dw_kernel"]
-    bytes_score = (R * d_out + R * d_in) * 2                      # every input byte read once
+    bytes_score = R * d_out * 2                                   # the scoring pass reads every row of dY once
     flops_dx = 2.0 * kept_A * d_in * d_out
     flops_dw = 2.0 * kept_W * d_in * d_out
     stages = {
@@ -646,14 +840,20 @@ def main():
         "pack_kernel": dict(ms=per[3], bound="hbm"),
         "umma_dw_kernel": dict(ms=per[4], bound="tensor", achieved=flops_dw / per[4] / 1e9 if per[4] else None),
     }
+    # The stage times come from 40 calls back to back behind a timed region of seconds: the GPU sits at its power
+    # cap (see `clocks`), so tensor-bound stages are held against the sustained bf16 peak, not the burst one.
     for k, v in stages.items():
         if v.get("achieved"):
-            v["frac"] = v["achieved"] / (pk["hbm"] if v["bound"] == "hbm" else pk["tc_burst"])
+            v["frac"] = v["achieved"] / (pk["hbm"] if v["bound"] == "hbm" else pk["tc_sustained"])
+            if v["bound"] == "tensor":
+                v["frac_of_burst_peak"] = v["achieved"] / pk["tc_burst"]
     dom = max(range(5), key=lambda i: per[i])
     dname = names[dom]
     if stages[dname]["bound"] == "tensor":
-        roof = dict(bound="tensor", kernel=dname, achieved=stages[dname]["achieved"], peak=pk["tc_burst"],
-                    unit="TFLOP/s", traffic=ncu_traffic(dname, WORKLOAD), peak_source=pk["source"] + " bf16 burst")
+        roof = dict(bound="tensor", kernel=dname, achieved=stages[dname]["achieved"], peak=pk["tc_sustained"],
+                    unit="TFLOP/s", traffic=ncu_traffic(dname, WORKLOAD),
+                    peak_source=pk["source"] + " bf16 sustained (kernel timed inside a long, power-capped run)",
+                    frac_of_burst_peak=stages[dname]["achieved"] / pk["tc_burst"])
     else:
         if dname != "rownorm_kernel":   # the small latency-bound stages are reported under the scoring pass
             dname = "rownorm_kernel"

@@ -232,8 +232,17 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
 /* Synchronises the device and returns the handle's device status word in *status
  * (VCAS_OK or VCAS_ERR_TIMEOUT / VCAS_ERR_INTERNAL); the word is then cleared.  After an
  * error the outputs of the calls since the last check are undefined; the workspace counters
- * that a kernel which gave up may have left behind are reset, so the handle stays usable. */
+ * that a kernel which gave up may have left behind are reset, so the handle stays usable.  No kernel of the
+ * library waits for another kernel or for another CTA; the only waits are those of vcas_set_wait_limit. */
 int vcas_last_device_status(vcas_handle h, int32_t* status);
+
+/* Failure detection (the paper has no counterpart).  Every wait inside the product kernels (on a TMA arrival,
+ * on the tensor pipe, on a work item) is bounded: when it lasts longer than limit_ns (default 2 s) the CTA
+ * records VCAS_ERR_TIMEOUT in the status word, all its roles leave their loops, its TMEM is released and the
+ * kernel returns.  Test hook: with stall_once != 0 the first CTA of every product launch leaves out the loads
+ * of its first k-block, so that one wait is certain to run out (nothing faults: the loads are simply not
+ * issued); with a limit of about a millisecond this exercises the give-up path.  limit_ns = 0 is rejected. */
+int vcas_set_wait_limit(vcas_handle h, uint64_t limit_ns, int32_t stall_once);
 
 /* Tuning overrides for the tensor-core products (the paper has no counterpart): output tile
  * width of the dX and dW kernels (64, 128 or 256), the number of slices each contraction is

@@ -196,6 +196,8 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->tune_dx_tile_n = h->tune_dw_tile_n = h->tune_dx_split_k = h->tune_dw_split_k = 0;
   h->tune_tile_m = 0;
   h->plan_valid = false;
+  h->wait_limit_ns = 2000000000ull;
+  h->stall_once = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&h->device) != cudaSuccess || cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
     delete h;
@@ -511,6 +513,13 @@ int vcas_set_tuning(vcas_handle hh, int32_t dx_tile_n, int32_t dw_tile_n, int32_
   h->tune_dx_split_k = dx_split_k;
   h->tune_dw_split_k = dw_split_k;
   h->tune_tile_m = tile_m;
+  return VCAS_OK;
+}
+
+int vcas_set_wait_limit(vcas_handle hh, uint64_t limit_ns, int32_t stall_once) {
+  if (hh == nullptr || limit_ns == 0) return VCAS_ERR_BAD_ARG;
+  H(hh)->wait_limit_ns = limit_ns;
+  H(hh)->stall_once = stall_once != 0 ? 1 : 0;
   return VCAS_OK;
 }
 

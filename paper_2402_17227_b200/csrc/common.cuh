@@ -85,6 +85,8 @@ struct Handle {
   bool plan_valid;
   int plan_key[PLAN_KEY_INTS];
   Plan plan_dx, plan_dw;
+  unsigned long long wait_limit_ns;   // bound of every device-side wait (default 2 s)
+  int stall_once;    // test hook, see vcas_set_wait_limit
   int tune_tile_m;   // 0 auto, 1: 128-row tiles only, 2: 256-row tiles whenever the width is 256, 3: 256-row tiles for
                      // whole waves of CTAs and 128-row tiles, their contraction sliced, for the rest
 };

@@ -27,7 +27,6 @@ constexpr int A_BYTES = BM * BK * 2;
 constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN chunk of an MN-major operand
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 constexpr int EPI_WARP_BYTES = 32 * 128;                // one staging buffer: 32 rows of 128 bytes, 128B-swizzled
 constexpr int EPI_BYTES = 4 * 2 * EPI_WARP_BYTES;       // two buffers for each of the four epilogue warps
 
@@ -69,9 +68,10 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Waits for the phase with the given parity; gives up after WAIT_LIMIT_NS or when another
-// role of this CTA has given up.  Returns false in that case.
+// Waits for the phase with the given parity; gives up after the wait limit (the 64-bit word 20 bytes after abort_flag, nanoseconds,
+// put there at set-up) or when another role of this CTA has given up.  Returns false in that case.
 __device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  const unsigned long long limit = *reinterpret_cast<volatile unsigned long long*>(abort_flag + 5);
   unsigned long long t0 = 0;
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
@@ -80,7 +80,7 @@ __device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile 
       const unsigned long long now = global_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > WAIT_LIMIT_NS) {
+      } else if (now - t0 > limit) {
         *abort_flag = 1;
         atomicExch(status, (int32_t)VCAS_ERR_TIMEOUT);
         return false;
@@ -215,7 +215,8 @@ __device__ __forceinline__ SmemLayout carve(uint8_t* raw) {
 }
 
 template <int BN, int MH>
-__device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid, bool with_queue) {
+__device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid, bool with_queue,
+                                          unsigned long long wait_limit_ns) {
   using C = TileCfg<BN, MH>;
   if (tid == 0) {
     for (int i = 0; i < C::STAGES; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
@@ -223,6 +224,7 @@ __device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid
     if (with_queue)
       for (int i = 0; i < QD; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 129); }
     *s.abort_flag = 0;
+    *reinterpret_cast<unsigned long long*>(s.abort_flag + 5) = wait_limit_ns;   // read by mbar_wait
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -233,10 +235,18 @@ __device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid
   return *(volatile uint32_t*)s.tmem_holder;
 }
 
-__device__ __noinline__ float gelu_prime(float x) {   // one copy: rarely run, and the product kernels are sensitive to code size
-  const float Phi = 0.5f * (1.0f + erff(x * 0.70710678118654752f));
-  const float phi = 0.39894228040143268f * expf(-0.5f * x * x);
-  return fmaf(x, phi, Phi);
+// GELU'(x) = Phi(x) + x phi(x) (erf form).  Both terms share E = exp(-x^2 / 2): phi = E / sqrt(2 pi), and
+// erf(|x| / sqrt 2) = 1 - (a1 t + ... + a5 t^5) E with t = 1 / (1 + p |x| / sqrt 2) (Abramowitz & Stegun 7.1.26,
+// absolute error below 1.5e-7, far inside the bf16 rounding of the result).  One exponential and one reciprocal
+// per element: the epilogue has only four warps per SM, so this arithmetic is on the critical path of the tile.
+__device__ __forceinline__ float gelu_prime(float x) {
+  const float ax = fabsf(x);
+  const float E = __expf(-0.5f * x * x);
+  const float t = __frcp_rn(fmaf(0.3275911f * 0.70710678118654752f, ax, 1.0f));
+  const float poly = t * fmaf(t, fmaf(t, fmaf(t, fmaf(t, 1.061405429f, -1.453152027f), 1.421413741f), -0.284496736f), 0.254829592f);
+  const float erf_abs = fmaf(-poly, E, 1.0f);
+  const float Phi = 0.5f * (1.0f + copysignf(erf_abs, x));
+  return fmaf(x, 0.39894228040143268f * E, Phi);
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -249,7 +259,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Work decomposition (all derived on the device from the kept counts): `gemm_tiles` output
 // tiles, each cut along the contraction into S slices of kb_per k-blocks -> units; a unit is
 // (tile, slice).  With S > 1 every unit stores its fp32 partial tile to the workspace and takes a
-// ticket on its tile; when all S tickets are in, each of the S units adds the S partials of its
+// ticket on its tile; the unit that takes the last of the S tickets adds the S partials of the
 // share of the tile's rows in slice order (a fixed order: results do not depend on timing) and
 // writes that share of the output.
 constexpr int MODE_DX = 0, MODE_DW = 1;
@@ -262,6 +272,8 @@ struct GemmParams {
   int32_t* sched;          // [2]: next work item, CTAs that have finished (unsliced instance); zero between launches
   int split_k;             // slices requested by the host
   int max_units;
+  unsigned long long wait_limit_ns;   // every mbarrier wait gives up after this long
+  int stall_once;          // test hook: CTA 0 leaves out the loads of its first k-block, so that a wait runs out
   // Whole waves and remainder (256-wide tiles): part 1 is the launch with 256-row tiles, which takes only as
   // many tiles as fill its head_ctas CTAs a whole number of times (when the rest is at most half a wave);
   // part 2 is a second launch with 128-row tiles that covers the remaining 256-row tiles, two tiles each,
@@ -391,7 +403,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   extern __shared__ uint8_t smem_raw[];
   const SmemLayout s = carve<BN, MH>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t tmem_base = setup<BN, MH>(s, warp, tid, KIND == KIND_DYNAMIC);
+  const uint32_t tmem_base = setup<BN, MH>(s, warp, tid, KIND == KIND_DYNAMIC, P.wait_limit_ns);
   volatile int* abort_flag = s.abort_flag;
   pdl_wait();      // barriers and TMEM are set up; the counts and operands come from earlier kernels
   constexpr bool LEAN = KIND != KIND_SLICED;
@@ -403,7 +415,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      bool ok = true;
+      bool ok = true, stalled = false;
       int qi = 0; uint32_t qph = 0;
       // next unit of this CTA, or -1 (see KIND above)
       auto next_unit = [&](int prev) -> int {
@@ -438,6 +450,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           ok = mbar_wait(&s.empty[stage], phase ^ 1u, abort_flag, P.status);
           if (!ok) break;
           uint8_t* sa = s.stages + stage * C::STAGE_BYTES;
+          if (P.stall_once != 0 && blockIdx.x == 0 && !stalled) {
+            stalled = true;                    // nothing will ever arrive for this stage: the MMA role's wait runs out
+            if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           if (MODE == MODE_DX) {
             mbar_expect_tx(&s.full[stage], (uint32_t)(MH * P.a_tx_bytes + C::B_BYTES));
 #pragma unroll
@@ -621,16 +638,27 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(tile, true, row0, rows_valid, col0, sc, n_out, t_out);
       const int buf = lt_now % NACC; const uint32_t use = (uint32_t)(lt_now / NACC) & 1u;
-      if (!mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status)) break;
+      bool got = mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status);
+      if constexpr (!LEAN) {
+        // the 128 epilogue threads meet at barriers further down: they give up together or not at all
+        uint32_t all;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.u32 p, %1, 0;\n\t"
+            "bar.red.and.pred q, 1, 128, p;\n\t"
+            "selp.u32 %0, 1, 0, q;\n\t}"
+            : "=r"(all) : "r"(got ? 1u : 0u) : "memory");
+        got = all != 0;
+      }
+      if (!got) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * BN);
       // Adds the slices of this unit's share of the tile's rows in slice order and writes that share of the
       // output.  A partial tile is laid out [32-column chunk][row][32 floats] with the eight 16-byte slots of
       // a row swizzled by (row & 7); load4(slice, float offset) fetches one slot of one slice.
-      auto reduce_share = [&](auto load4) {
-        const int rows_per = (BM + D.S - 1) / D.S;
-        const int r_begin = slice * rows_per;
-        const int r_end = min(min(BM, r_begin + rows_per), rows_valid);
+      auto reduce_tile = [&](auto load4) {
+        const int r_begin = 0;
+        const int r_end = min(BM, rows_valid);
         const int c8n = min(BN, P.d_in - col0) / 8;               // 8-column groups per row inside the tensor
         const int n_items = max(0, r_end - r_begin) * c8n;
         auto slot_off = [&](int r, int c8, int half) {
@@ -680,12 +708,34 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         float rowsq[MH];                                            // square-norm of this thread's row(s), as stored
 #pragma unroll
         for (int hh = 0; hh < MH; ++hh) rowsq[hh] = 0.f;
+        // GELU' epilogue: this thread's 64 pre-activations of a chunk (eight 16-byte loads, its own row) are
+        // requested one chunk ahead, so that their latency hides behind the chunk before (a load per use was
+        // measured to double the time of the whole product)
+        uint4 hq[8], hn[8];
+        auto load_h = [&](int hj2, uint4 (&dst)[8]) {
+          const int hh2 = hj2 / (BN / COLS), j2 = hj2 % (BN / COLS);
+          const int hrow2 = hh2 * BM + row;
+          const bool okh = hj2 < MH * (BN / COLS) && hrow2 < rows_valid && col0 + j2 * COLS < P.d_in;
+          if (okh) {
+            const uint4* src = reinterpret_cast<const uint4*>(P.H + (row0 + hrow2) * ld + col0 + j2 * COLS);
+#pragma unroll
+            for (int k8 = 0; k8 < 8; ++k8) dst[k8] = __ldg(src + k8);
+          }
+        };
+        if (MODE == MODE_DX && P.H != nullptr) load_h(0, hq);
 #pragma unroll 1
         for (int hj = 0; hj < MH * (BN / COLS); ++hj, ++nbuf) {
           const int hh = hj / (BN / COLS), j = hj % (BN / COLS);    // 128-row half of the tile, column chunk
           const int hrow = hh * BM + row;
           const bool valid = hrow < rows_valid;
           const uint32_t taddr_h = taddr + (uint32_t)(hh * BN);
+          if (MODE == MODE_DX && P.H != nullptr) {
+            if (hj > 0) {
+#pragma unroll
+              for (int k8 = 0; k8 < 8; ++k8) hq[k8] = hn[k8];
+            }
+            load_h(hj + 1, hn);
+          }
           if (col0 + j * COLS >= P.d_in) { --nbuf; continue; }      // warp-uniform
           uint8_t* buf8 = stage0 + (nbuf & 1) * EPI_WARP_BYTES;
           if (nbuf >= 2) { if (lane == 0) bulk_wait_read_1(); __syncwarp(); }
@@ -701,8 +751,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int e = 0; e < 8; ++e) r[e] = sc * __uint_as_float(v[g8 * 8 + e]);
                 if (P.H != nullptr && valid) {
-                  const size_t off = (row0 + hrow) * ld + col0 + j * 64 + half * 32 + g8 * 8;
-                  const uint4 hv = *reinterpret_cast<const uint4*>(P.H + off);
+                  const uint4 hv = hq[half * 4 + g8];
                   const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
 #pragma unroll
                   for (int e = 0; e < 4; ++e) {
@@ -782,41 +831,27 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       mbar_arrive(&s.tmem_empty[buf]);          // the accumulator is free again
       if (lane == 0) bulk_wait_all();           // this warp's part of the partial tile is in global memory
       __syncwarp();
-      // ... announce it, wait (bounded) until all S slices of the tile are stored ...
+      // ... announce it.  The unit that finds the other S - 1 slices of its tile already announced adds the S
+      // partial tiles in slice order (a fixed order: results do not depend on which unit comes last) and writes
+      // the output; the others are done.  No unit waits for another one, so the S units of a tile need not be
+      // resident at the same time.
       __threadfence();
       epi_bar();
       if (tid == 0) {
-        atomicAdd(&P.tickets[tile], 1);
-        unsigned long long t0 = 0; uint32_t spins = 0; int good = 1;
-        while (*(volatile int32_t*)&P.tickets[tile] < D.S) {
-          if ((++spins & 0xffu) == 0) {
-            if (*abort_flag) { good = 0; break; }
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; atomicExch(P.status, (int32_t)VCAS_ERR_TIMEOUT); good = 0; break; }
-          }
-        }
-        *s.flag = good;
+        const int arrived = atomicAdd(&P.tickets[tile], 1);
+        const int last = arrived == D.S - 1 ? 1 : 0;
+        if (last) P.tickets[tile] = 0;            // all S have arrived: re-armed for the next launch
+        *s.flag = last;
       }
       epi_bar();
-      ok = *(volatile int*)s.flag != 0;
-      if (!ok) break;
-      __threadfence();
-      // ... then add the S partials of this unit's share of the rows, in slice order, and write the output.
-      {
+      if (*(volatile int*)s.flag != 0) {
+        __threadfence();
         const float* tile_part = P.partial + (size_t)(tile * D.S) * (BM * BN);
-        reduce_share([&](int sl, size_t off) {
+        reduce_tile([&](int sl, size_t off) {
           return __ldcg(reinterpret_cast<const float4*>(tile_part + (size_t)sl * (BM * BN) + off));
         });
       }
-      epi_bar();
-      if (tid == 0) {
-        __threadfence();
-        if (atomicAdd(&P.tickets[P.max_units + tile], 1) == D.S - 1) {   // last slice done: reset for the next launch
-          P.tickets[tile] = 0;
-          P.tickets[P.max_units + tile] = 0;
-        }
-      }
+      epi_bar();                                  // s.flag is rewritten by the next unit
       }  // !LEAN
     }
     // sliced instance: zero tiles are taken from the far end of the grid first, where CTAs have no product units
@@ -865,7 +900,8 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
 // in-kernel timestamps: a k-block costs about 0.5 / 0.45 / 0.43 us for 256 / 128 / 64 wide tiles
 // (the shared-memory fill rate of one SM bounds it, so narrow tiles only pay off when they fill
 // more SMs); a unit costs about 4 us of set-up, pipeline fill and output store; a sliced unit
-// about 7 us more (partial store, wait for its siblings, reduction); a 256 x 256 tile (mh = 2) costs
+// about 3 us more for its partial store, and the unit that comes last adds the S partial tiles of the whole
+// tile (about 2.5 us per slice); a 256 x 256 tile (mh = 2) costs
 // about 0.62 us per k-block for twice the work, and 7 us per tile.
 struct Cand {
   Plan plan;
@@ -895,7 +931,7 @@ int enumerate_plans(long row_tiles128, long row_tiles256, int n_extent, int kblo
       if (sp > 1 && force_split == 0 && kblocks / sp < 4) continue;   // slices too short to pay off
       const long units = tiles * sp;
       const double waves = (double)((units + num_sms - 1) / num_sms);
-      const double unit = (double)((kblocks + sp - 1) / sp) * c_kb[i] + (sp > 1 ? 11.0 + 0.25 * sp : 4.0);
+      const double unit = (double)((kblocks + sp - 1) / sp) * c_kb[i] + (sp > 1 ? 7.0 + 2.5 * sp : 4.0);
       if (n < MAX_CANDS) out[n++] = {{widths[i], sp, 1}, units, unit, waves * unit};
     }
     if (widths[i] == 256 && force_split <= 1) {                        // 256 x 256 tiles, never sliced
@@ -908,7 +944,7 @@ int enumerate_plans(long row_tiles128, long row_tiles256, int n_extent, int kblo
         if (sp > 8) sp = 8;
         if (sp > kblocks / 4) sp = kblocks / 4;
         if (sp < 1) sp = 1;
-        const double tail = (double)((kblocks + sp - 1) / sp) * 0.50 + (sp > 1 ? 11.0 + 0.25 * sp : 4.0) + 4.0;
+        const double tail = (double)((kblocks + sp - 1) / sp) * 0.50 + (sp > 1 ? 7.0 + 2.5 * (double)sp : 4.0) + 4.0;
         if (n < MAX_CANDS) out[n++] = {{256, 1, 3}, units, wave, (double)(units / num_sms) * wave + tail};
       }
     }
@@ -1035,6 +1071,8 @@ void common_params(Handle* h, GemmParams& P, int which) {
   P.tickets = h->ws.tickets + (size_t)which * 2 * h->max_units;
   P.sched = h->ws.sched + which * 2;
   P.max_units = h->max_units;
+  P.wait_limit_ns = h->wait_limit_ns;
+  P.stall_once = h->stall_once;
   P.d_in = h->desc.d_in;
   P.d_out = h->desc.d_out;
 }

@@ -52,8 +52,11 @@ CASES = {
 }
 
 
-def make_layer(case: LayerCase, batch: int = 0, *, N=None, T=None, d_in=None, d_out=None):
-    """Draw (X [R, d_in], dY [R, d_out], W [d_out, d_in]) for `case` on the CPU.
+def make_layer(case: LayerCase, batch: int = 0, *, N=None, T=None, d_in=None, d_out=None, device="cpu"):
+    """Draw (X [R, d_in], dY [R, d_out], W [d_out, d_in]) for `case`, by default on the CPU.
+
+    With a CUDA `device` the same recipe runs on that device's generator (same distributions and seeds, other
+    values than the CPU's): for benchmarks that need many large tensors and no host copy of them.
 
     `batch` selects an independent mini-batch (same W, fresh X and dY), as the probe's
     Monte-Carlo batches need.  Shape overrides give reduced copies of a workload with the
@@ -64,24 +67,25 @@ def make_layer(case: LayerCase, batch: int = 0, *, N=None, T=None, d_in=None, d_
     d_in = case.d_in if d_in is None else d_in
     d_out = case.d_out if d_out is None else d_out
     R = N * T
-    gw = torch.Generator().manual_seed(case.data_seed)
-    W = (torch.randn(d_out, d_in, generator=gw, dtype=torch.float32) * 0.02).to(case.dtype)
-    gb = torch.Generator().manual_seed(case.data_seed * 1000003 + 7919 * (batch + 1))
-    X = torch.randn(R, d_in, generator=gb, dtype=torch.float32).to(case.dtype)
-    A = torch.exp(case.sigma_A * torch.randn(N, generator=gb, dtype=torch.float32))
-    B = torch.exp(case.sigma_B * torch.randn(N, T, generator=gb, dtype=torch.float32))
+    kw = dict(dtype=torch.float32, device=device)
+    gw = torch.Generator(device).manual_seed(case.data_seed)
+    W = (torch.randn(d_out, d_in, generator=gw, **kw) * 0.02).to(case.dtype)
+    gb = torch.Generator(device).manual_seed(case.data_seed * 1000003 + 7919 * (batch + 1))
+    X = torch.randn(R, d_in, generator=gb, **kw).to(case.dtype)
+    A = torch.exp(case.sigma_A * torch.randn(N, generator=gb, **kw))
+    B = torch.exp(case.sigma_B * torch.randn(N, T, generator=gb, **kw))
     if case.zero_fraction > 0.0:
-        dead = torch.rand(N, generator=gb) < case.zero_fraction
+        dead = torch.rand(N, generator=gb, device=device) < case.zero_fraction
         A = torch.where(dead, torch.zeros_like(A), A)
-    dY = torch.randn(R, d_out, generator=gb, dtype=torch.float32)
+    dY = torch.randn(R, d_out, generator=gb, **kw)
     dY = (dY * (A[:, None] * B).reshape(R, 1)).to(case.dtype)
     return X, dY, W
 
 
-def make_preactivation(case: LayerCase, batch: int = 0, *, N=None, T=None, width=None):
+def make_preactivation(case: LayerCase, batch: int = 0, *, N=None, T=None, width=None, device="cpu"):
     """Pre-activation H ~ N(0, 1) of shape [R, width] saved by a GELU between two linears."""
     N = case.N if N is None else N
     T = case.T if T is None else T
     width = case.d_in if width is None else width
-    g = torch.Generator().manual_seed(case.data_seed * 7 + 13 * (batch + 1))
-    return torch.randn(N * T, width, generator=g, dtype=torch.float32).to(case.dtype)
+    g = torch.Generator(device).manual_seed(case.data_seed * 7 + 13 * (batch + 1))
+    return torch.randn(N * T, width, generator=g, dtype=torch.float32, device=device).to(case.dtype)

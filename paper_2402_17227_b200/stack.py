@@ -70,8 +70,9 @@ class LinearStack:
                     self._scratch[L.d_in] = torch.empty(self.R, L.d_in, dtype=dtype, device=dev)
                 L.dX = self._scratch[L.d_in]
 
-    def backward(self, rho, nu, seed: int, variant: int = 0) -> None:
-        """One sampled backward pass, top layer first.  rho, nu: per-layer keep ratios in backward order."""
+    def backward(self, rho, nu, seed: int, variant: int = 0, hook=None) -> None:
+        """One sampled backward pass, top layer first.  rho, nu: per-layer keep ratios in backward order.
+        hook(i, layer, after): optional callback before (after=False) and after every layer's call."""
         prev = None
         for i, L in enumerate(self.layers):
             v = variant % len(L.X)
@@ -84,17 +85,25 @@ class LinearStack:
             else:
                 dY = L.dY[v]
             H = L.H[v % len(L.H)] if L.H is not None else None
+            if hook is not None:
+                hook(i, L, False)
             L.handle.linear_bwd_chain(L.X[v], dY, L.W, float(rho[i]), float(nu[i]), seed * len(self.layers) + i,
                                       L.dX, L.dW, H=H, a_out=L.a_out, kept_out=L.kept, kept_cnt_out=L.kept_cnt, **kw)
+            if hook is not None:
+                hook(i, L, True)
             prev = L
 
-    def dense_backward(self, variant: int = 0) -> None:
+    def dense_backward(self, variant: int = 0, hook=None) -> None:
         """The exact backward of the same layers (no sampling, no Jacobian factor): the dense comparison."""
         prev = None
-        for L in self.layers:
+        for i, L in enumerate(self.layers):
             v = variant % len(L.X)
             dY = prev.dX if L.chained else L.dY[v]
+            if hook is not None:
+                hook(i, L, False)
             L.handle.dense_bwd(L.X[v], dY, L.W, dX=L.dX, dW=L.dW)
+            if hook is not None:
+                hook(i, L, True)
             prev = L
 
     def probe(self, rho, nu, s: float, seed: int):
