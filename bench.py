@@ -495,7 +495,7 @@ def measure_bert_large_stack(vb, inputs, torch, dev, steps=200, F=50, M=2):
             W = (torch.randn(d_out, d_in, generator=gw, device=dev, dtype=torch.float32) * 0.02).to(bf)
             Xs, dYs, H = pool[name]
             layers.append(StackLayer(f"b{blk}.{name}", d_in, d_out, W, Xs, dYs, H=H, chained=chained))
-    stack = LinearStack(layers, N, T, config=cfg)
+    stack = LinearStack(layers, N, T, config=cfg, skip_dropped_rows=True)    # every consumer takes the kept-data list
     L = len(layers)
     # Alg. 1's state in layer order (index 0 = lowest layer); the stack runs in backward order (top first)
     state = dict(s=0.75, rho=list(np.linspace(0.2, 0.8, L)), nu=[0.3] * L)

@@ -130,8 +130,13 @@ int vcas_linear_bwd_ex(vcas_handle h, const void* X, const void* dY, const void*
  *                its rows of dY and a_in are never read, it is never kept, its rows of dX are zero;
  *   a_out        [R][vcas_chain_parts] fp32: partial sums of the square-norm of every row of dX as stored
  *                (after the GELU' factor and the rounding to the layer dtype), written by the dX product;
- *   kept_out     [N] int32: ascending list of the data this call kept, kept_cnt_out [1] its length.
- * alive_in / alive_cnt_in and kept_out / kept_cnt_out come in pairs; the lists must not alias.
+ *   kept_out     [N] int32: ascending list of the data this call kept, kept_cnt_out [1] its length;
+ *   skip_dropped_rows  non-zero: the rows of dX (and a_out) that belong to dropped data are left unwritten instead
+ *                of being set to zero - for a consumer that takes kept_out as its alive_in and therefore never
+ *                reads them (tensor-core path; the fp32 path always writes them).
+ * alive_in / alive_cnt_in and kept_out / kept_cnt_out come in pairs; the lists must not alias.  A length
+ * outside [0, N] or an entry outside [0, N) is not followed: it is reported as VCAS_ERR_BAD_ARG by
+ * vcas_last_device_status (the call's outputs are then undefined).
  */
 typedef struct {
   const void* H;
@@ -142,6 +147,7 @@ typedef struct {
   float* a_out;
   int32_t* kept_out;
   int32_t* kept_cnt_out;
+  int32_t skip_dropped_rows;
 } vcas_chain_args;
 int vcas_linear_bwd_chain(vcas_handle h, const void* X, const void* dY, const void* W,
                           float rho, float nu, uint64_t seed, const vcas_chain_args* chain,
@@ -230,7 +236,7 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
                        const vcas_config* cfg);
 
 /* Synchronises the device and returns the handle's device status word in *status
- * (VCAS_OK or VCAS_ERR_TIMEOUT / VCAS_ERR_INTERNAL); the word is then cleared.  After an
+ * (VCAS_OK or VCAS_ERR_TIMEOUT / VCAS_ERR_INTERNAL / VCAS_ERR_BAD_ARG); the word is then cleared.  After an
  * error the outputs of the calls since the last check are undefined; the workspace counters
  * that a kernel which gave up may have left behind are reset, so the handle stays usable.  No kernel of the
  * library waits for another kernel or for another CTA; the only waits are those of vcas_set_wait_limit. */

@@ -52,7 +52,7 @@ class State(C.Structure):
 class ChainArgs(C.Structure):
     _fields_ = [("H", C.c_void_p), ("a_in", C.c_void_p), ("a_in_parts", C.c_int32), ("alive_in", C.c_void_p),
                 ("alive_cnt_in", C.c_void_p), ("a_out", C.c_void_p), ("kept_out", C.c_void_p),
-                ("kept_cnt_out", C.c_void_p)]
+                ("kept_cnt_out", C.c_void_p), ("skip_dropped_rows", C.c_int32)]
 
 
 _lib = None
@@ -151,12 +151,12 @@ class Layer:
 
     def linear_bwd_chain(self, X, dY, W, rho: float, nu: float, seed: int, dX, dW, *, H=None, a_in=None,
                          a_in_parts: int = 1, alive_in=None, alive_cnt_in=None, a_out=None, kept_out=None,
-                         kept_cnt_out=None):
+                         kept_cnt_out=None, skip_dropped_rows: bool = False):
         """vcas_linear_bwd_chain: scores handed down from the layer above (a_in, alive_in) and to the layer
         below (a_out, kept_out); every extra is an optional device tensor."""
         dp = lambda t: None if t is None else t.data_ptr()
         args = ChainArgs(dp(H), dp(a_in), a_in_parts, dp(alive_in), dp(alive_cnt_in), dp(a_out), dp(kept_out),
-                         dp(kept_cnt_out))
+                         dp(kept_cnt_out), 1 if skip_dropped_rows else 0)
         _check(lib().vcas_linear_bwd_chain(self._h, _ptr(X), _ptr(dY), _ptr(W), C.c_float(rho), C.c_float(nu),
                                            C.c_uint64(seed), C.byref(args), _ptr(dX), _ptr(dW), _stream()),
                "vcas_linear_bwd_chain")

@@ -265,7 +265,7 @@ namespace {
 // One sampled backward (Eq. 2).  `a` carries the ratios, the seed, the optional given probabilities and the
 // optional scores handed down from the layer above; a_out: optional row square-norms of dX for the layer below.
 int run_sampled(Handle* h, const void* X, const void* dY, const void* W, const SamplerArgs& a, const void* Hpre,
-                void* dX, float* dW, float* a_out, cudaStream_t st) {
+                void* dX, float* dW, float* a_out, bool skip_dropped, cudaStream_t st) {
   const int hint = (int)(a.rho * a.nu * (float)(h->desc.N * h->desc.T)) + 1;
   // The sampled dX grid leaves one SM free: SampleW's single-CTA kernel, which runs beside it on the side
   // stream, needs a whole SM's shared memory.
@@ -282,9 +282,9 @@ int run_sampled(Handle* h, const void* X, const void* dY, const void* W, const S
     VCAS_CUDA(launch_sample_w(h, a, st));
     mark(h, 2, st);
     if (h->tensor_path) {
-      VCAS_CUDA(launch_umma_dx(h, dY, W, false, a.rho, Hpre, dX, a_out, spare, &px, st));
+      VCAS_CUDA(launch_umma_dx(h, dY, W, false, a.rho, Hpre, dX, a_out, skip_dropped, spare, &px, st));
     } else {
-      VCAS_CUDA(launch_fma_dx(h, dY, W, h->ws.scaleA, Hpre, dX, st));
+      VCAS_CUDA(launch_fma_dx(h, dY, W, h->ws.scaleA, Hpre, dX, st));     // always writes the zero rows
       if (a_out != nullptr) VCAS_CUDA(launch_rownorm_out(h, dX, a_out, st));
     }
     mark(h, 3, st);
@@ -306,7 +306,7 @@ int run_sampled(Handle* h, const void* X, const void* dY, const void* W, const S
     VCAS_CUDA(launch_sample_a(h, a, a.a_in == nullptr, st));
     VCAS_CUDA(cudaEventRecord(h->ev_fork, st));
     VCAS_CUDA(cudaStreamWaitEvent(h->side_stream, h->ev_fork, 0));
-    VCAS_CUDA(launch_umma_dx(h, dY, W, false, a.rho, Hpre, dX, a_out, spare, &px, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, false, a.rho, Hpre, dX, a_out, skip_dropped, spare, &px, st));
     const int rc = sample_w_and_dw(h, X, dY, a, false, &pw, dW, h->side_stream);
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
@@ -325,7 +325,7 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
   SamplerArgs a = sampler_args(rho, nu, seed);
   a.p_in = p_in; a.q_in = q_in;
-  return run_sampled(H(hh), X, dY, W, a, Hpre, dX, dW, nullptr, S(stream));
+  return run_sampled(H(hh), X, dY, W, a, Hpre, dX, dW, nullptr, false, S(stream));
 }
 
 int vcas_linear_bwd_chain(vcas_handle hh, const void* X, const void* dY, const void* W, float rho, float nu,
@@ -340,7 +340,7 @@ int vcas_linear_bwd_chain(vcas_handle hh, const void* X, const void* dY, const v
   a.a_in = c->a_in; a.a_parts = c->a_in != nullptr ? c->a_in_parts : 1;
   a.alive = c->alive_in; a.alive_cnt = c->alive_cnt_in;
   a.kept_out = c->kept_out; a.kept_cnt_out = c->kept_cnt_out;
-  return run_sampled(H(hh), X, dY, W, a, c->H, dX, dW, c->a_out, S(stream));
+  return run_sampled(H(hh), X, dY, W, a, c->H, dX, dW, c->a_out, c->skip_dropped_rows != 0, S(stream));
 }
 
 int vcas_chain_parts(vcas_handle hh, int32_t* parts) {
@@ -371,7 +371,7 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
   if (h->tensor_path) plan_products(h, true, 1.0f, h->desc.N * h->desc.T, 0, false, &px, &pw);
   mark_dense(h, 0, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, nullptr, 0, &px, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, nullptr, false, 0, &px, st));
   } else {
     VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
   }

@@ -340,8 +340,10 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 // pair_plan: the tiling chosen by plan_products for a call whose two products run at the same time
 // (nullptr: chosen here, for this product alone)
 // a_out: optional [R][a_out_parts(d_in)] partial row square-norms of the stored dX, written by the epilogue
+// skip_dropped: the rows of dropped data are not written (a consumer with the kept-data list never reads them)
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
-                           const void* H, void* dX, float* a_out, int spare_sms, const Plan* pair_plan, cudaStream_t st);
+                           const void* H, void* dX, float* a_out, bool skip_dropped, int spare_sms,
+                           const Plan* pair_plan, cudaStream_t st);
 inline int a_out_parts(int d_in) { return (d_in + 255) / 256; }
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling

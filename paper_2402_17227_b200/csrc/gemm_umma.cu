@@ -116,6 +116,7 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void*
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // at most one group of this thread may still be READING its shared-memory source
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // all groups of this thread are complete (their global writes are performed)
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -237,12 +238,13 @@ __device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid
 
 // GELU'(x) = Phi(x) + x phi(x) (erf form).  Both terms share E = exp(-x^2 / 2): phi = E / sqrt(2 pi), and
 // erf(|x| / sqrt 2) = 1 - (a1 t + ... + a5 t^5) E with t = 1 / (1 + p |x| / sqrt 2) (Abramowitz & Stegun 7.1.26,
-// absolute error below 1.5e-7, far inside the bf16 rounding of the result).  One exponential and one reciprocal
+// absolute error below 1.5e-7, far inside the bf16 rounding of the result).  One exponential and one approximate reciprocal
 // per element: the epilogue has only four warps per SM, so this arithmetic is on the critical path of the tile.
 __device__ __forceinline__ float gelu_prime(float x) {
   const float ax = fabsf(x);
   const float E = __expf(-0.5f * x * x);
-  const float t = __frcp_rn(fmaf(0.3275911f * 0.70710678118654752f, ax, 1.0f));
+  float t;      // approximate reciprocal (one instruction, no special-case branch; 1 ulp is far below the rest)
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f * 0.70710678118654752f, ax, 1.0f)));
   const float poly = t * fmaf(t, fmaf(t, fmaf(t, fmaf(t, 1.061405429f, -1.453152027f), 1.421413741f), -0.284496736f), 0.254829592f);
   const float erf_abs = fmaf(-poly, E, 1.0f);
   const float Phi = 0.5f * (1.0f + copysignf(erf_abs, x));
@@ -292,6 +294,7 @@ struct GemmParams {
   int a_parts;             // tile (unsliced 256-wide tiles only); the layer below adds the partials in order
   int N, T;
   int dense;               // 1: every datum kept with scale 1
+  int skip_dropped;        // 1: the rows of dropped data are left unwritten (the consumer knows they are zero)
   int a_tx_bytes;          // bytes one A box delivers (min(T, 128) token rows of 128 B)
   // dW: A = rows x d_out, B = rows x d_in (both MN-major, gathered along k by the pack step)
   const int32_t* cnt;      // number of valid rows (the contraction length)
@@ -315,7 +318,7 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
     const int cntA = P.dense ? P.N : P.counts[0];
     d.per_datum = ((P.T + BMT - 1) / BMT) * d.ntiles;
     d.gemm_tiles = cntA * d.per_datum;
-    d.zero_tiles = (P.N - cntA) * d.per_datum;
+    d.zero_tiles = P.skip_dropped ? 0 : (P.N - cntA) * d.per_datum;
     d.kblocks = (P.d_out + BK - 1) / BK;
   } else {
     d.per_datum = 0;
@@ -590,7 +593,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     };
 
-    uint8_t* stage0 = s.epi + warp * (2 * EPI_WARP_BYTES);       // this warp's two staging buffers
     const uint32_t swz = (uint32_t)(lane & 7);                   // 128-byte swizzle: 16-byte slot ^= row & 7
     int lt = 0;
     bool ok = true;
@@ -610,25 +612,38 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         return ((int)blockIdx.x < D.upi && u < D.units) ? u : -1;
       }
     };
-    // writes the zero tile z (rows of dropped data; nothing kept at all)
+    // Writes the zero tile z (rows of dropped data; nothing kept at all): every warp clears one of its staging
+    // buffers and stores it, by TMA, to each 32-row x 128-byte piece of its slab of the tile.  The tensor map
+    // clips rows beyond T and columns beyond d_in.  No per-element work: the epilogue warps are free again at once.
+    uint8_t* stage0 = s.epi + warp * (2 * EPI_WARP_BYTES);       // this warp's two staging buffers
     auto zero_tile = [&](int z) {
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(z, false, row0, rows_valid, col0, sc, n_out, t_out);
+      reinterpret_cast<uint4*>(stage0)[lane] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int k8 = 1; k8 < EPI_WARP_BYTES / 512; ++k8)
+        reinterpret_cast<uint4*>(stage0)[k8 * 32 + lane] = make_uint4(0u, 0u, 0u, 0u);
+      fence_async_smem();
+      __syncwarp();
+      constexpr int COLS = MODE == MODE_DX ? 64 : 32;             // columns per 128-byte staged row
+      if (lane == 0) {
 #pragma unroll 1
-      for (int hh = 0; hh < MH; ++hh) {
-        const int hrow = hh * BM + row;
-        if (hrow >= rows_valid) continue;
-        const size_t off = (row0 + hrow) * ld + col0;
-        if (MODE == MODE_DX) {
-#pragma unroll
-          for (int j = 0; j < BN / 8; ++j)
-            if (col0 + j * 8 < P.d_in) *reinterpret_cast<uint4*>(P.dX + off + j * 8) = make_uint4(0u, 0u, 0u, 0u);
-          if (P.a_out != nullptr) P.a_out[(row0 + hrow) * P.a_parts + col0 / 256] = 0.f;
-        } else {
-#pragma unroll
-          for (int j = 0; j < BN / 4; ++j)
-            if (col0 + j * 4 < P.d_in) *reinterpret_cast<uint4*>(P.dW + off + j * 4) = make_uint4(0u, 0u, 0u, 0u);
+        for (int hh = 0; hh < MH; ++hh) {
+          if (hh * BM + warp * 32 >= rows_valid) break;
+          for (int j = 0; j < BN / COLS; ++j) {
+            if (col0 + j * COLS >= P.d_in) break;
+            if (MODE == MODE_DX) tma_store_3d(&tmC, stage0, col0 + j * COLS, t_out + hh * BM + warp * 32, n_out);
+            else tma_store_2d(&tmC, stage0, col0 + j * COLS, (int)row0 + hh * BM + warp * 32);
+          }
         }
+        bulk_commit();
+        bulk_wait_read_0();                  // the buffer may be rewritten; the global writes finish on their own
+      }
+      __syncwarp();
+      if (MODE == MODE_DX && P.a_out != nullptr) {
+#pragma unroll 1
+        for (int hh = 0; hh < MH; ++hh)
+          if (hh * BM + row < rows_valid) P.a_out[(row0 + hh * BM + row) * P.a_parts + col0 / 256] = 0.f;
       }
     };
     for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
@@ -859,6 +874,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int z = (int)gridDim.x - 1 - (int)blockIdx.x; z < D.zero_tiles && ok; z += gridDim.x) zero_tile(z);
     }
   }
+  if (warp < 4 && lane == 0) bulk_wait_all();     // the bulk stores of zero tiles are only waited for here
   __syncwarp();
   tc_fence_before();
   __syncthreads();
@@ -1136,7 +1152,8 @@ void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spar
 }
 
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint, const void* H,
-                           void* dX, float* a_out, int spare_sms, const Plan* pair_plan, cudaStream_t st) {
+                           void* dX, float* a_out, bool skip_dropped, int spare_sms, const Plan* pair_plan,
+                           cudaStream_t st) {
   const vcas_layer_desc& d = h->desc;
   CUtensorMap tmA, tmB, tmC;
   {
@@ -1163,6 +1180,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
   P.a_out = a_out; P.a_parts = a_out_parts(d.d_in);
   P.H = (const __nv_bfloat16*)H; P.dX = (__nv_bfloat16*)dX;
   P.N = d.N; P.T = d.T; P.dense = dense ? 1 : 0;
+  P.skip_dropped = skip_dropped ? 1 : 0;
   P.a_tx_bytes = (d.T < BM ? d.T : BM) * BK * 2;
   const int chunks = (d.T + BM - 1) / BM, chunks2 = (d.T + 2 * BM - 1) / (2 * BM);
   const int ctas = h->num_sms - spare_sms > 1 ? h->num_sms - spare_sms : 1;

@@ -154,10 +154,23 @@ __global__ void __launch_bounds__(SAMPLE_A_THREADS) sample_a_kernel(SampleAParam
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int n = threadIdx.x; n < 32 * SLOTS; n += SAMPLE_A_THREADS) s_g[n] = 0.f;
   __syncthreads();
-  const int nd = P.alive != nullptr ? *P.alive_cnt : P.N;
+  // a caller's list of alive data is not trusted: a length outside [0, N] or an entry outside [0, N) is reported
+  // as VCAS_ERR_BAD_ARG in the status word and not followed
+  int nd = P.N;
+  if (P.alive != nullptr) {
+    nd = *P.alive_cnt;
+    if (nd < 0 || nd > P.N) {
+      if (threadIdx.x == 0) atomicExch(P.status, (int32_t)VCAS_ERR_BAD_ARG);
+      nd = min(max(nd, 0), P.N);
+    }
+  }
   const int len = P.T * P.a_parts;
   for (int k = warp; k < nd; k += SAMPLE_A_THREADS / 32) {
     const int n = P.alive != nullptr ? P.alive[k] : k;
+    if ((unsigned)n >= (unsigned)P.N) {
+      if (lane == 0) atomicExch(P.status, (int32_t)VCAS_ERR_BAD_ARG);
+      continue;
+    }
     const float s = datum_sqnorm_warp(P.a + (size_t)n * len, len, lane);
     if (lane == 0) s_g[n] = sqrtf(s);
   }
@@ -183,10 +196,21 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_a_big_kernel(SampleAPa
   const int N = P.N;
   for (int n = tid; n < N; n += nt) P.g[n] = 0.f;
   __syncthreads();
-  const int nd = P.alive != nullptr ? *P.alive_cnt : N;
+  int nd = N;
+  if (P.alive != nullptr) {
+    nd = *P.alive_cnt;
+    if (nd < 0 || nd > N) {
+      if (tid == 0) atomicExch(P.status, (int32_t)VCAS_ERR_BAD_ARG);
+      nd = min(max(nd, 0), N);
+    }
+  }
   const int len = P.T * P.a_parts;
   for (int k = warp; k < nd; k += nw) {
     const int n = P.alive != nullptr ? P.alive[k] : k;
+    if ((unsigned)n >= (unsigned)N) {
+      if (lane == 0) atomicExch(P.status, (int32_t)VCAS_ERR_BAD_ARG);
+      continue;
+    }
     const float s = datum_sqnorm_warp(P.a + (size_t)n * len, len, lane);
     if (lane == 0) P.g[n] = sqrtf(s);
   }

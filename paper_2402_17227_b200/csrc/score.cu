@@ -80,13 +80,24 @@ __global__ void __launch_bounds__(256) rownorm_dy_kernel(const T* __restrict__ d
   pdl_trigger();   // the next kernel may be scheduled now; it waits for this grid before reading
   const int lane = threadIdx.x & 31;
   const int wpb = blockDim.x >> 5;
-  const int rows = alive != nullptr ? *alive_cnt * Tn : R;
+  const int N = R / Tn;
+  // a caller's list is not trusted: its length is clamped and entries outside [0, N) are skipped (SampleA
+  // reports them in the status word)
+  const int rows = alive != nullptr ? min(max(*alive_cnt, 0), N) * Tn : R;
   for (int c = blockIdx.x * wpb + (threadIdx.x >> 5); c < rows; c += gridDim.x * wpb) {
     int r = c;
-    if (alive != nullptr) { const int k = c / Tn; r = alive[k] * Tn + (c - k * Tn); }
+    bool valid = true;
+    if (alive != nullptr) {
+      const int k = c / Tn;
+      const int n = alive[k];
+      valid = (unsigned)n < (unsigned)N;
+      r = valid ? n * Tn + (c - k * Tn) : 0;
+    }
     const float sa = warp_sum(row_partial<T>(dY + (size_t)r * d_out, d_out, lane));
-    if (lane == 0) a[(size_t)r * stride] = sa;
-    else if (lane < stride) a[(size_t)r * stride + lane] = 0.f;
+    if (valid) {
+      if (lane == 0) a[(size_t)r * stride] = sa;
+      else if (lane < stride) a[(size_t)r * stride + lane] = 0.f;
+    }
   }
 }
 

@@ -44,8 +44,11 @@ class LinearStack:
     the calls of a pass follow one another on one stream)."""
 
     def __init__(self, layers: list[StackLayer], N: int, T: int, dtype=torch.bfloat16, config=None,
-                 gemm_path: int = vb.GEMM_AUTO):
+                 gemm_path: int = vb.GEMM_AUTO, skip_dropped_rows: bool = False):
+        """skip_dropped_rows: the rows of dX that belong to dropped data are not written (every consumer in the
+        stack takes the kept-data list and never reads them); the dX buffers then hold stale rows there."""
         self.layers, self.N, self.T, self.dtype = layers, N, T, dtype
+        self.skip_dropped_rows = skip_dropped_rows
         self.R = N * T
         self.handles: dict = {}
         dev = layers[0].W.device
@@ -88,7 +91,8 @@ class LinearStack:
             if hook is not None:
                 hook(i, L, False)
             L.handle.linear_bwd_chain(L.X[v], dY, L.W, float(rho[i]), float(nu[i]), seed * len(self.layers) + i,
-                                      L.dX, L.dW, H=H, a_out=L.a_out, kept_out=L.kept, kept_cnt_out=L.kept_cnt, **kw)
+                                      L.dX, L.dW, H=H, a_out=L.a_out, kept_out=L.kept, kept_cnt_out=L.kept_cnt,
+                                      skip_dropped_rows=self.skip_dropped_rows, **kw)
             if hook is not None:
                 hook(i, L, True)
             prev = L

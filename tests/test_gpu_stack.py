@@ -149,3 +149,50 @@ def test_stack_adaptation_follows_the_oracle():
         assert stack.device_status() == 0
     assert moved
     stack.close()
+
+
+def test_bad_alive_list_is_reported_not_followed():
+    """A caller's alive list with a length beyond N or an entry outside [0, N) is skipped by the kernels' own
+    checks and reported through the status word."""
+    vbuild.build()
+    N, T, d_in, d_out = 8, 64, 128, 192
+    case = inputs.LayerCase("bad", N, T, d_in, d_out, BF16, 1.0, 0.5, 0.5, 0.5)
+    X, dY, W = [t.cuda() for t in inputs.make_layer(case)]
+    lay = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
+    dX = torch.empty(N * T, d_in, dtype=BF16, device="cuda")
+    dW = torch.empty(d_out, d_in, dtype=torch.float32, device="cuda")
+    alive = torch.tensor([0, 3, N + 5, -2, 6, 7, 1, 2], dtype=torch.int32, device="cuda")
+    for cnt in (5, N + 3):
+        c = torch.tensor([cnt], dtype=torch.int32, device="cuda")
+        lay.linear_bwd_chain(X, dY, W, 0.5, 0.5, 1, dX, dW, alive_in=alive, alive_cnt_in=c)
+        assert lay.device_status() == -1
+    good = torch.tensor([0, 3, 6], dtype=torch.int32, device="cuda")
+    lay.linear_bwd_chain(X, dY, W, 0.9, 0.5, 1, dX, dW, alive_in=good,
+                         alive_cnt_in=torch.tensor([3], dtype=torch.int32, device="cuda"))
+    assert lay.device_status() == 0
+    s = lay.last_sampling()
+    assert set(s.idxA.cpu().tolist()) <= {0, 3, 6}
+    lay.close()
+
+
+def test_skip_dropped_rows_leaves_them_untouched():
+    """With skip_dropped_rows the rows of dX of dropped data are not written; the kept rows are the same bits."""
+    vbuild.build()
+    N, T, d_in, d_out = 10, 197, 320, 192
+    case = inputs.LayerCase("skip", N, T, d_in, d_out, BF16, 1.0, 0.5, 0.5, 0.5)
+    X, dY, W = [t.cuda() for t in inputs.make_layer(case)]
+    lay = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
+    ref = torch.empty(N * T, d_in, dtype=BF16, device="cuda")
+    dW = torch.empty(d_out, d_in, dtype=torch.float32, device="cuda")
+    kept = torch.zeros(N, dtype=torch.int32, device="cuda"); cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lay.linear_bwd_chain(X, dY, W, 0.5, 0.5, 4, ref, dW, kept_out=kept, kept_cnt_out=cnt)
+    dX = torch.full((N * T, d_in), 7.0, dtype=BF16, device="cuda")
+    lay.linear_bwd_chain(X, dY, W, 0.5, 0.5, 4, dX, dW, kept_out=kept, kept_cnt_out=cnt, skip_dropped_rows=True)
+    k = kept[:int(cnt.item())].cpu().numpy()
+    keep = np.zeros(N, bool); keep[k] = True
+    assert 0 < keep.sum() < N
+    rows = torch.from_numpy(np.repeat(keep, T)).cuda()
+    assert torch.equal(dX[rows], ref[rows]) and not ref[~rows].any()
+    assert torch.all(dX[~rows] == 7.0)
+    assert lay.device_status() == 0
+    lay.close()
