@@ -262,9 +262,29 @@ def sparsity_p(g, s: float) -> float:
     return n / g.shape[0]
 
 
+def param_subset(d_out: int, k: int, seed: int):
+    """A uniformly random subset of k of the layer's d_out output features (rows of theta), ascending.
+
+    App. D estimates the variances on a small random sample of the parameters.  Contract of this
+    repository: feature i gets the Philox word of counter (i, 0, 2, 0) under the key (seed low, seed high)
+    (sampler id 2), and the k features with the smallest words are taken (ties by index)."""
+    idx = np.arange(d_out, dtype=np.uint64)
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    zero = np.zeros_like(idx)
+    u = philox4x32_10((idx, zero, zero + np.uint64(2), zero),
+                      (zero + np.uint64(seed & 0xFFFFFFFF), zero + np.uint64(seed >> 32)))[0]
+    order = np.lexsort((np.arange(d_out), u))            # by word, then by index
+    return np.sort(order[:k]).astype(np.int64)
+
+
 def variance_probe(Xs, dYs, W, N: int, T: int, rho: float, nu: float, s: float,
-                   alpha: float, seed: int):
+                   alpha: float, seed: int, param_rows=None):
     """The Monte-Carlo probe of Alg. 1 for one linear layer's parameter gradient.
+
+    param_rows (App. D: the variances are estimated on a sample of the parameters): if given, V_s and V_act
+    are taken over these rows of the parameter gradient only and scaled by d_out / len(param_rows) - an
+    unbiased estimate of the full sums when the rows are a uniformly random subset.  V_w is analytic (Eq. 3)
+    and needs no gradient.
 
     Xs, dYs: M batches.  For every batch i the exact gradient G_s,i = dY_i^T X_i; for
     every repetition j a SampleA-only gradient G_act,ij = G_hat_ij^T X_i and the analytic
@@ -275,26 +295,28 @@ def variance_probe(Xs, dYs, W, N: int, T: int, rho: float, nu: float, s: float,
     M = len(Xs)
     assert M >= 2 and len(dYs) == M
     W = np.asarray(W, dtype=np.float64)
+    rows = slice(None) if param_rows is None else np.asarray(param_rows)
+    scale = 1.0 if param_rows is None else W.shape[0] / len(param_rows)
     G_s = []
     v_act, v_w, p_lo, p_hi = 0.0, 0.0, 0.0, 0.0
     for i in range(M):
         X = np.asarray(Xs[i], dtype=np.float64)
         dY = np.asarray(dYs[i], dtype=np.float64)
-        G_s.append(dY.T @ X)
+        G_s.append((dY.T @ X)[rows])
         g = datum_norms(row_sqnorms(dY), N, T)
         p_lo += sparsity_p(g, max(0.0, s - alpha))
         p_hi += sparsity_p(g, min(1.0, s + alpha))
         for j in range(M):
             sd = probe_seed(seed, i, j, M)
             sa = sample_a(dY, N, T, rho, sd)
-            G_act = sa["G_hat"].T @ X
+            G_act = (sa["G_hat"].T @ X)[rows]
             v_act += float(np.sum((G_act - G_s[i]) ** 2))
             w = np.sqrt(row_sqnorms(sa["G_hat"])) * np.sqrt(row_sqnorms(X))
             q32 = capped_prop(w, nu * T * int(np.count_nonzero(sa["keepA"]))).astype(np.float32)
             v_w += var_sample_w(sa["G_hat"], X, q32)
     mean = sum(G_s) / M
     V_s = sum(float(np.sum((G - mean) ** 2)) for G in G_s) / (M - 1)
-    return dict(V_s=V_s, V_act=v_act / (M * M), V_w=v_w / (M * M), p_lo=p_lo / M, p_hi=p_hi / M)
+    return dict(V_s=scale * V_s, V_act=scale * v_act / (M * M), V_w=v_w / (M * M), p_lo=p_lo / M, p_hi=p_hi / M)
 
 
 def update_ratios(s, rho, nu, V_s, V_act, V_w, p_lo, p_hi, *, tau_act, tau_w, alpha, beta,

@@ -457,3 +457,39 @@ def test_kept_row_forms_agree_with_whole_matrix_forms():
         dX, dW = o.products_on_kept_rows(X, dY, W, sm["p32"], sm["q32"], sm["keepA"], sm["keepW"], T)
         assert np.allclose(dX, ref["dX"], rtol=1e-12, atol=1e-13) and np.allclose(dW, ref["dW"], rtol=1e-12, atol=1e-13)
         assert 0 < sm["keepA"].sum() < N and 0 < sm["keepW"].sum() < sm["keepA"].sum() * T
+
+
+def test_probe_on_a_parameter_subset_is_unbiased_for_the_full_sums():
+    """App. D: variances estimated on a random sample of the parameters.  Averaged over ALL subsets of k of the
+    d_out rows, the scaled subset estimates equal the full V_s and V_act exactly (each row is in the same
+    share k/d_out of the subsets); V_w and the sparsity candidates do not depend on the subset."""
+    r = rng(31)
+    N, T, di, do, M, k = 5, 3, 4, 5, 2, 2
+    W = r.standard_normal((do, di))
+    Xs = [r.standard_normal((N * T, di)) for _ in range(M)]
+    dYs = [r.standard_normal((N * T, do)) * np.repeat(np.exp(r.standard_normal(N)), T)[:, None] for _ in range(M)]
+    full = o.variance_probe(Xs, dYs, W, N, T, 0.6, 0.5, s=0.8, alpha=0.05, seed=3)
+    subs = list(itertools.combinations(range(do), k))
+    outs = [o.variance_probe(Xs, dYs, W, N, T, 0.6, 0.5, s=0.8, alpha=0.05, seed=3, param_rows=list(c)) for c in subs]
+    assert np.isclose(np.mean([x["V_s"] for x in outs]), full["V_s"], rtol=1e-12)
+    assert np.isclose(np.mean([x["V_act"] for x in outs]), full["V_act"], rtol=1e-12)
+    assert all(x["V_w"] == full["V_w"] and x["p_lo"] == full["p_lo"] and x["p_hi"] == full["p_hi"] for x in outs)
+    assert len({round(x["V_s"], 9) for x in outs}) > 1                     # the subsets do differ
+    # one subset, by hand: rows {1, 3} of the gradients, scaled by d_out / 2
+    Gs = np.stack([dY.T @ X for X, dY in zip(Xs, dYs)])[:, [1, 3]]
+    one = o.variance_probe(Xs, dYs, W, N, T, 0.6, 0.5, s=0.8, alpha=0.05, seed=3, param_rows=[1, 3])
+    assert np.isclose(one["V_s"], do / 2 * np.var(Gs, axis=0, ddof=1).sum(), rtol=1e-12)
+
+
+def test_param_subset_is_a_uniform_random_subset():
+    k, d = 8, 40
+    seen = np.zeros(d)
+    for seed in range(3000):
+        sub = o.param_subset(d, k, seed)
+        assert len(sub) == k and len(set(sub)) == k and np.all(np.diff(sub) > 0) and 0 <= sub[0] and sub[-1] < d
+        seen[sub] += 1
+    expect = 3000 * k / d                               # every feature in a share k/d of the subsets
+    chi2 = np.sum((seen - expect) ** 2 / (expect * (1 - k / d)))
+    assert chi2 < (d - 1) + 6 * np.sqrt(2 * (d - 1))
+    assert np.array_equal(o.param_subset(d, d, 5), np.arange(d))           # k = d: everything
+    assert not np.array_equal(o.param_subset(d, k, 1), o.param_subset(d, k, 1 + (1 << 32)))   # both key words
