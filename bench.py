@@ -32,6 +32,7 @@ WORKLOAD = "llm_mlp_up"
 RHO = NU = 0.3
 F_CALLS = 100
 PROBE_M = 2
+PROBE_ROWS = 128       # rows of the parameter gradient the probe samples (App. D), of the layer's 11008
 N_BATCHES = 2
 METRIC = "sampled linear-bwd ms/layer"
 SLAB = 1024            # d_out columns of the layer that one oracle sample computes (CPU baseline)
@@ -496,6 +497,8 @@ def measure_bert_large_stack(vb, inputs, torch, dev, steps=200, F=50, M=2):
             Xs, dYs, H = pool[name]
             layers.append(StackLayer(f"b{blk}.{name}", d_in, d_out, W, Xs, dYs, H=H, chained=chained))
     stack = LinearStack(layers, N, T, config=cfg, skip_dropped_rows=True)    # every consumer takes the kept-data list
+    for hd in stack.handles.values():
+        hd.set_probe_subsample(128, 0)          # App. D: the probe's variances on a sample of the parameter rows
     L = len(layers)
     # Alg. 1's state in layer order (index 0 = lowest layer); the stack runs in backward order (top first)
     state = dict(s=0.75, rho=list(np.linspace(0.2, 0.8, L)), nu=[0.3] * L)
@@ -605,7 +608,7 @@ def measure_bert_large_stack(vb, inputs, torch, dev, steps=200, F=50, M=2):
         "initial": {"s": 0.75, "rho_top": 0.8, "rho_bottom": 0.2, "nu": 0.3},
         "trajectory": traj, "final": {"s": state["s"], "rho": [round(float(x), 4) for x in state["rho"]],
                                       "nu": [round(float(x), 4) for x in state["nu"]]},
-        "workspace_bytes": stack.workspace_bytes(), "handles": len(stack.handles),
+        "workspace_bytes": stack.workspace_bytes(), "handles": len(stack.handles), "probe_sampled_rows": 128,
     }
     assert stack.device_status() == 0
     stack.close()
@@ -729,6 +732,15 @@ def main():
     with torch.cuda.graph(graph_dense):
         dense_only()
     probe_launches = [0]
+
+    # the probe on all rows of the parameter gradient and on a sample of them (App. D); the steps use the sample
+    def probe_ms():
+        for _ in range(2):
+            layer.variance_probe(Xs[:PROBE_M], dYs[:PROBE_M], W, RHO, NU, 1.0, 1, out=probe_out)
+        return timed(lambda: layer.variance_probe(Xs[:PROBE_M], dYs[:PROBE_M], W, RHO, NU, 1.0, 1, out=probe_out), 3) / 3
+    probe_full_ms = probe_ms()
+    layer.set_probe_subsample(PROBE_ROWS, 0)
+    probe_sub_ms = probe_ms()
 
     def step():
         # Alg. 1: every F calls probe the variances on M batches and update (s, rho_l, nu_l) ...
@@ -883,6 +895,8 @@ def main():
         "dense_tflops": 4.0 * R * d_in * d_out / ms_dense / 1e9,
         "kept_rows": {"kept_A": kept_A, "kept_W": kept_W, "R": R, "note": "mean over the 40 profiled calls"},
         "workspace_bytes": layer.workspace_bytes(),
+        "probe": {"M": PROBE_M, "ms_all_parameter_rows": probe_full_ms, "ms_sampled_rows": probe_sub_ms,
+                  "sampled_rows": PROBE_ROWS, "of_rows": d_out, "used_in_steps": "sampled rows"},
         "adaptation_state": state,
         "other_workloads": extra,
     }

@@ -225,6 +225,19 @@ int vcas_variance_probe(vcas_handle h, int32_t M, const void* const* X_i, const 
                         vcas_stream stream);
 
 /*
+ * App. D: the probe's variances may be estimated on a random sample of the parameters.  With rows > 0 the
+ * probe forms G_s,i and G_act,ij only on `rows` of the d_out rows of the parameter gradient - a uniformly
+ * random subset fixed here: row i gets the Philox word of counter (i, 0, 2, 0) under the key (seed low, seed
+ * high), the `rows` smallest words win, ties by index - and scales V_s and V_act by d_out / rows (unbiased for
+ * the sums over all rows); V_w (Eq. 3) and p_lo / p_hi need no gradient and are unchanged.  The probe's two
+ * products then cost rows / d_out of their full size.  rows: a multiple of 64 (8 on the fp32-FMA path), at most
+ * 256 and below d_out; 0 switches the sample off (default).  Synchronous.
+ */
+int vcas_set_probe_subsample(vcas_handle h, int32_t rows, uint64_t seed);
+/* The rows chosen (host out, ascending; rows_host may be NULL) and their number. */
+int vcas_get_probe_subsample(vcas_handle h, int32_t* rows_host, int32_t* count);
+
+/*
  * One adaptation step of Alg. 1 (host only, all pointers host, arrays of length L):
  *   Eq. 5: s <- clip(s + alpha sign(sum_l V_act,l - tau_act sum_l V_s,l), 0, 1), sign(0) = +1;
  *   Eq. 4: rho_l <- max(rho_min, max_{j<=l} p_j) with p_j = p_hi[j] if s went up else p_lo[j];

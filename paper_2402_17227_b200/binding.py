@@ -24,7 +24,8 @@ GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
 EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
            "vcas_linear_bwd_ex", "vcas_linear_bwd_chain", "vcas_chain_parts", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
-           "vcas_set_profiling", "vcas_stage_times", "vcas_set_wait_limit", "vcas_score_static", "vcas_set_tuning",
+           "vcas_set_profiling", "vcas_stage_times", "vcas_set_wait_limit",
+           "vcas_set_probe_subsample", "vcas_get_probe_subsample", "vcas_score_static", "vcas_set_tuning",
            "vcas_version"]
 
 
@@ -237,6 +238,17 @@ class Layer:
                    tile_m: int = 0) -> None:
         _check(lib().vcas_set_tuning(self._h, C.c_int32(dx_tile_n), C.c_int32(dw_tile_n), C.c_int32(dx_split_k),
                                      C.c_int32(dw_split_k), C.c_int32(tile_m)), "vcas_set_tuning")
+
+    def set_probe_subsample(self, rows: int, seed: int = 0) -> None:
+        _check(lib().vcas_set_probe_subsample(self._h, C.c_int32(rows), C.c_uint64(seed)), "vcas_set_probe_subsample")
+
+    def probe_subsample(self):
+        """The rows of the parameter gradient the probe samples (host list; empty when it uses all rows)."""
+        n = C.c_int32(0)
+        _check(lib().vcas_get_probe_subsample(self._h, None, C.byref(n)), "vcas_get_probe_subsample")
+        rows = (C.c_int32 * max(1, n.value))()
+        _check(lib().vcas_get_probe_subsample(self._h, rows, C.byref(n)), "vcas_get_probe_subsample")
+        return list(rows)[:n.value]
 
     def set_wait_limit(self, limit_ns: int, stall_once: bool = False) -> None:
         _check(lib().vcas_set_wait_limit(self._h, C.c_uint64(limit_ns), C.c_int32(1 if stall_once else 0)),

@@ -98,6 +98,8 @@ size_t layout(Handle* h, uint8_t* base) {
     v.sched = w.sched + 2;
   }
   v.Gact = carve<float>(cur, DW);
+  h->sub_rows = carve<int32_t>(cur, SUB_MAX);
+  h->sub_dY = carve<float>(cur, R * SUB_MAX * (d.dtype == VCAS_DTYPE_BF16 ? 2 : 4) / 4);
   return (size_t)(cur - base);
 }
 
@@ -197,6 +199,7 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->tune_tile_m = 0;
   h->plan_valid = false;
   h->wait_limit_ns = 2000000000ull;
+  h->sub_k = 0;
   h->stall_once = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&h->device) != cudaSuccess || cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
@@ -430,11 +433,25 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
   double s_lo = (double)s - alpha, s_hi = (double)s + alpha;
   if (s_lo < 0.0) s_lo = 0.0;
   if (s_hi > 1.0) s_hi = 1.0;
+  // App. D: with a subsample set (vcas_set_probe_subsample) the exact and the SampleA-only gradients are formed
+  // on sub_k rows of the parameter gradient only: the products run through a copy of the handle whose d_out is
+  // sub_k, on those columns of dY; scoring and sampling still see the whole of dY.
+  const bool sub = h->sub_k > 0;
+  Handle hs = *h;
+  if (sub) hs.desc.d_out = h->sub_k;
+  hs.plan_valid = false;
+  Handle* hp = sub ? &hs : h;
+  const uint64_t launches0 = hs.launches;
   VCAS_CUDA(launch_probe_reset(h, st));
   for (int i = 0; i < M; ++i) {
-    int rc = dense_dw(h, X_i[i], dY_i[i], nullptr, h->ws.Gs, st);   // G_s,i
+    const void* dYp = dY_i[i];
+    if (sub) {
+      VCAS_CUDA(launch_gather_cols(h, dY_i[i], h->desc.d_out, h->sub_rows, h->sub_k, h->sub_dY, st));
+      dYp = h->sub_dY;
+    }
+    int rc = dense_dw(hp, X_i[i], dYp, nullptr, h->ws.Gs, st);   // G_s,i
     if (rc != VCAS_OK) return rc;
-    VCAS_CUDA(launch_probe_welford(h, i, st));
+    VCAS_CUDA(launch_probe_welford(hp, i, st));
     SamplerArgs a = sampler_args(rho, nu, 0);
     a.sample_w = 0;          // the probe draws no SampleW mask: G_act keeps every row of the kept data,
     a.accumulate_vw = 1;     // and Eq. 3 is accumulated analytically at ratio nu
@@ -451,19 +468,23 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
       cudaStream_t sj = second ? h->side_stream : st;
       h->ws = second ? h->ws2 : first;
       h->ws.a = first.a;
+      hs.ws = h->ws;
       a.seed = seed + (uint64_t)(i * M + j + 1) * 0x9E3779B97F4A7C15ull;
       cudaError_t e = launch_sample_a(h, a, !second, sj);
       if (e == cudaSuccess && j == 0) e = launch_probe_sparsity(h, s_lo, s_hi, sj);
-      if (e == cudaSuccess) rc = sample_w_and_dw(h, X_i[i], dY_i[i], a, true, nullptr, h->ws.Gact, sj);   // G_act,ij
-      if (e == cudaSuccess && rc == VCAS_OK) e = launch_probe_sqdiff(h, sj);
+      if (e == cudaSuccess) rc = sample_w_and_dw(hp, X_i[i], dYp, a, true, nullptr, h->ws.Gact, sj);   // G_act,ij
+      if (e == cudaSuccess && rc == VCAS_OK) e = launch_probe_sqdiff(hp, sj);
       h->ws = first;
+      hs.ws = first;
       if (e != cudaSuccess) return VCAS_ERR_CUDA;
       if (rc != VCAS_OK) return rc;
     }
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
     VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   }
-  VCAS_CUDA(launch_probe_finalize(h, M, V_s, V_act, V_w, p_lo, p_hi, st));
+  const double scale = sub ? (double)h->desc.d_out / (double)h->sub_k : 1.0;
+  VCAS_CUDA(launch_probe_finalize(hp, M, scale, V_s, V_act, V_w, p_lo, p_hi, st));
+  if (sub) h->launches += hs.launches - launches0;
   return VCAS_OK;
 }
 
@@ -513,6 +534,29 @@ int vcas_set_tuning(vcas_handle hh, int32_t dx_tile_n, int32_t dw_tile_n, int32_
   h->tune_dx_split_k = dx_split_k;
   h->tune_dw_split_k = dw_split_k;
   h->tune_tile_m = tile_m;
+  return VCAS_OK;
+}
+
+int vcas_set_probe_subsample(vcas_handle hh, int32_t rows, uint64_t seed) {
+  if (hh == nullptr || rows < 0) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  if (rows == 0) { h->sub_k = 0; return VCAS_OK; }
+  const int unit = h->tensor_path ? 64 : 8;
+  if (rows > SUB_MAX || (rows % unit) != 0 || rows >= h->desc.d_out) return VCAS_ERR_BAD_ARG;
+  // scratch: the probe's gradient buffers are free between probes
+  VCAS_CUDA(launch_param_subset(h, rows, seed, reinterpret_cast<uint32_t*>(h->ws.Gs),
+                                reinterpret_cast<int32_t*>(h->ws.Gact), h->sub_rows, nullptr));
+  VCAS_CUDA(cudaDeviceSynchronize());
+  h->sub_k = rows;
+  return VCAS_OK;
+}
+
+int vcas_get_probe_subsample(vcas_handle hh, int32_t* rows_host, int32_t* count) {
+  if (hh == nullptr || count == nullptr) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  *count = h->sub_k;
+  if (rows_host != nullptr && h->sub_k > 0)
+    VCAS_CUDA(cudaMemcpy(rows_host, h->sub_rows, (size_t)h->sub_k * sizeof(int32_t), cudaMemcpyDeviceToHost));
   return VCAS_OK;
 }
 

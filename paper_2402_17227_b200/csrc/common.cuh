@@ -85,12 +85,17 @@ struct Handle {
   bool plan_valid;
   int plan_key[PLAN_KEY_INTS];
   Plan plan_dx, plan_dw;
+  // the probe's sample of the parameters (App. D): sub_k rows of the parameter gradient (0: all of them)
+  int sub_k;
+  int32_t* sub_rows;   // [SUB_MAX] device, ascending
+  void* sub_dY;        // [R, SUB_MAX] those columns of the current batch's dY, compact
   unsigned long long wait_limit_ns;   // bound of every device-side wait (default 2 s)
   int stall_once;    // test hook, see vcas_set_wait_limit
   int tune_tile_m;   // 0 auto, 1: 128-row tiles only, 2: 256-row tiles whenever the width is 256, 3: 256-row tiles for
                      // whole waves of CTAs and 128-row tiles, their contraction sliced, for the rest
 };
 constexpr int PROF_RING = 2048;
+constexpr int SUB_MAX = 256;     // most parameter rows the probe's subsample may hold
 
 // ---------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies.
@@ -361,7 +366,13 @@ cudaError_t launch_probe_welford(Handle* h, int i, cudaStream_t st);
 cudaError_t launch_probe_sqdiff(Handle* h, cudaStream_t st);
 cudaError_t launch_probe_sparsity(Handle* h, double s_lo, double s_hi, cudaStream_t st);
 // adds the accumulators of the second set to the first (fixed order), then Alg. 1's averages
-cudaError_t launch_probe_finalize(Handle* h, int M, float* V_s, float* V_act, float* V_w,
+// scale: factor of V_s and V_act (d_out / sampled parameter rows)
+cudaError_t launch_probe_finalize(Handle* h, int M, double scale, float* V_s, float* V_act, float* V_w,
                                   float* p_lo, float* p_hi, cudaStream_t st);
+// out[r, c] = in[r, cols[c]] for the R rows of a [R, d] matrix of the layer dtype
+cudaError_t launch_gather_cols(Handle* h, const void* in, int d, const int32_t* cols, int k, void* out, cudaStream_t st);
+// k of the d_out output features chosen by Philox (ascending) into rows; scratch_u, scratch_flag: d_out words each
+cudaError_t launch_param_subset(Handle* h, int k, uint64_t seed, uint32_t* scratch_u, int32_t* scratch_flag,
+                                int32_t* rows, cudaStream_t st);
 
 }  // namespace vcas

@@ -110,15 +110,50 @@ __global__ void __launch_bounds__(1024) sparsity_kernel(const float* __restrict_
   }
 }
 
-__global__ void finalize_kernel(const double* __restrict__ acc, const double* __restrict__ acc2, int M, float* V_s,
-                                float* V_act, float* V_w, float* p_lo, float* p_hi) {
+// scale: d_out / (rows of the parameter gradient the sums were taken over) (App. D: a sample of the parameters)
+__global__ void finalize_kernel(const double* __restrict__ acc, const double* __restrict__ acc2, int M, double scale,
+                                float* V_s, float* V_act, float* V_w, float* p_lo, float* p_hi) {
   if (threadIdx.x == 0 && blockIdx.x == 0) {
     const double mm = (double)M * (double)M;
-    if (V_s) *V_s = (float)(acc[4] / (double)(M - 1));
-    if (V_act) *V_act = (float)((acc[0] + acc2[0]) / mm);     // even draws + odd draws
+    if (V_s) *V_s = (float)(scale * acc[4] / (double)(M - 1));
+    if (V_act) *V_act = (float)(scale * (acc[0] + acc2[0]) / mm);     // even draws + odd draws
     if (V_w) *V_w = (float)((acc[1] + acc2[1]) / mm);
     if (p_lo) *p_lo = (float)(acc[2] / (double)M);
     if (p_hi) *p_hi = (float)(acc[3] / (double)M);
+  }
+}
+
+// The columns `cols` of a row-major [R, d] matrix, compact: out[r, c] = in[r, cols[c]] (one warp per row).
+template <typename T>
+__global__ void __launch_bounds__(256) gather_cols_kernel(const T* __restrict__ in, int R, int d,
+                                                          const int32_t* __restrict__ cols, int k, T* __restrict__ out) {
+  const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+  for (int r = blockIdx.x * wpb + (threadIdx.x >> 5); r < R; r += gridDim.x * wpb)
+    for (int c = lane; c < k; c += 32) out[(size_t)r * k + c] = in[(size_t)r * d + cols[c]];
+}
+
+// A uniformly random subset of k of the d_out output features, ascending: feature i gets the Philox word of
+// counter (i, 0, 2, 0) (sampler id 2) under the key (seed low, seed high); the k features with the smallest
+// words are taken, ties by index.  One CTA; u is scratch of d_out words.
+__global__ void __launch_bounds__(1024) subset_kernel(int d_out, int k, uint64_t seed, uint32_t* __restrict__ u,
+                                                      int32_t* __restrict__ flag, int32_t* __restrict__ rows) {
+  for (int i = threadIdx.x; i < d_out; i += blockDim.x)
+    u[i] = philox_word0((uint32_t)i, 0u, 2u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+  __syncthreads();
+  for (int i = threadIdx.x; i < d_out; i += blockDim.x) {
+    const uint32_t x = u[i];
+    int rank = 0;
+    for (int j = 0; j < d_out; ++j) {
+      const uint32_t y = u[j];
+      rank += (y < x) || (y == x && j < i);
+    }
+    flag[i] = rank < k ? 1 : 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int i = 0; i < d_out; ++i)
+      if (flag[i]) rows[n++] = i;
   }
 }
 
@@ -161,12 +196,31 @@ cudaError_t launch_probe_sparsity(Handle* h, double s_lo, double s_hi, cudaStrea
   return cudaGetLastError();
 }
 
-cudaError_t launch_probe_finalize(Handle* h, int M, float* V_s, float* V_act, float* V_w, float* p_lo,
+cudaError_t launch_gather_cols(Handle* h, const void* in, int d, const int32_t* cols, int k, void* out, cudaStream_t st) {
+  const int R = h->desc.N * h->desc.T;
+  int blocks = (R + 7) / 8;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (h->desc.dtype == VCAS_DTYPE_BF16)
+    gather_cols_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)in, R, d, cols, k, (__nv_bfloat16*)out);
+  else
+    gather_cols_kernel<float><<<blocks, 256, 0, st>>>((const float*)in, R, d, cols, k, (float*)out);
+  h->launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_param_subset(Handle* h, int k, uint64_t seed, uint32_t* scratch_u, int32_t* scratch_flag,
+                                int32_t* rows, cudaStream_t st) {
+  subset_kernel<<<1, 1024, 0, st>>>(h->desc.d_out, k, seed, scratch_u, scratch_flag, rows);
+  h->launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_probe_finalize(Handle* h, int M, double scale, float* V_s, float* V_act, float* V_w, float* p_lo,
                                   float* p_hi, cudaStream_t st) {
   const size_t n4 = (size_t)h->desc.d_out * h->desc.d_in / 4;
   reduce_kernel<<<reduce_blocks(n4), 256, 0, st>>>((const float4*)h->ws.m2, nullptr, n4, 1, h->ws.partial,
                                                    h->ws.counts + 4, h->ws.acc + 4);
-  finalize_kernel<<<1, 32, 0, st>>>(h->ws.acc, h->ws2.acc, M, V_s, V_act, V_w, p_lo, p_hi);
+  finalize_kernel<<<1, 32, 0, st>>>(h->ws.acc, h->ws2.acc, M, scale, V_s, V_act, V_w, p_lo, p_hi);
   h->launches += 2;
   return cudaGetLastError();
 }
