@@ -223,6 +223,28 @@ def dense_bwd(X, dY, W):
     return dY @ W, dY.T @ X
 
 
+def layernorm_bwd(X, gamma, dY, N: int, T: int, rho: float, seed: int, eps: float = 1e-5, p_override=None):
+    """Backward of Y = LayerNorm(X) * gamma + beta over the last axis with SampleA in front of it
+    (Eq. 2 for a layer without a weight-gradient sampler; App. E: the sampled, rescaled gradient G_hat is
+    multiplied by the layer's exact Jacobian).  Returns dict(p32, keepA, dX, dgamma, dbeta, g).
+
+    With x_hat = (x - mean) / sqrt(var + eps) per row and g_hat = G_hat * gamma:
+      dX = (g_hat - mean(g_hat) - x_hat * mean(g_hat * x_hat)) / sqrt(var + eps)     (row-wise means),
+      dgamma = sum_r G_hat_r * x_hat_r,   dbeta = sum_r G_hat_r.
+    Rows of dropped data have G_hat = 0, hence dX = 0 and no contribution to dgamma, dbeta."""
+    X = np.asarray(X, dtype=np.float64)
+    gamma = np.asarray(gamma, dtype=np.float64)
+    sa = sample_a(dY, N, T, rho, seed, p_override)
+    G = sa["G_hat"]
+    mean = X.mean(axis=1, keepdims=True)
+    var = ((X - mean) ** 2).mean(axis=1, keepdims=True)
+    rstd = 1.0 / np.sqrt(var + eps)
+    xh = (X - mean) * rstd
+    gh = G * gamma
+    dX = (gh - gh.mean(axis=1, keepdims=True) - xh * (gh * xh).mean(axis=1, keepdims=True)) * rstd
+    return dict(p32=sa["p32"], keepA=sa["keepA"], g=sa["g"], dX=dX, dgamma=(G * xh).sum(axis=0), dbeta=G.sum(axis=0))
+
+
 # --------------------------------------------------------------------------------------
 # Closed-form variances (Sec. 4.1 and Eq. 3)
 # --------------------------------------------------------------------------------------

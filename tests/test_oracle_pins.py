@@ -493,3 +493,46 @@ def test_param_subset_is_a_uniform_random_subset():
     assert chi2 < (d - 1) + 6 * np.sqrt(2 * (d - 1))
     assert np.array_equal(o.param_subset(d, d, 5), np.arange(d))           # k = d: everything
     assert not np.array_equal(o.param_subset(d, k, 1), o.param_subset(d, k, 1 + (1 << 32)))   # both key words
+
+
+def test_layernorm_bwd_is_autograd_at_ratio_one_and_unbiased():
+    import torch
+    r = rng(41)
+    N, T, d = 4, 3, 6
+    X = r.standard_normal((N * T, d)) * 2 + 0.5
+    gamma, beta = r.standard_normal(d), r.standard_normal(d)
+    dY = r.standard_normal((N * T, d)) * np.repeat(np.exp(r.standard_normal(N)), T)[:, None]
+    # ratio 1: exact backward of the library LayerNorm (float64 autograd)
+    xt = torch.tensor(X, requires_grad=True); gt = torch.tensor(gamma, requires_grad=True)
+    bt = torch.tensor(beta, requires_grad=True)
+    y = torch.nn.functional.layer_norm(xt, (d,), gt, bt, eps=1e-5)
+    y.backward(torch.tensor(dY))
+    out = o.layernorm_bwd(X, gamma, dY, N, T, 1.0, seed=0)
+    assert out["keepA"].all()
+    assert np.allclose(out["dX"], xt.grad.numpy(), rtol=1e-10, atol=1e-12)
+    assert np.allclose(out["dgamma"], gt.grad.numpy(), rtol=1e-10, atol=1e-12)
+    assert np.allclose(out["dbeta"], bt.grad.numpy(), rtol=1e-10, atol=1e-12)
+    # sampled: all three are linear in G_hat, so the exact enumeration over the 2^N masks gives the exact backward
+    g = o.datum_norms(o.row_sqnorms(dY), N, T)
+    p = o.capped_prop(g, N * 0.5).astype(np.float32)
+    mean = {k: 0 for k in ("dX", "dgamma", "dbeta")}
+    for mask in itertools.product([0, 1], repeat=N):
+        keep = np.array(mask, bool)
+        pr = np.prod(np.where(keep, p.astype(np.float64), 1 - p.astype(np.float64)))
+        G_hat = o.apply_data_mask(dY, p, keep, T)
+        xt2 = torch.tensor(X, requires_grad=True); gt2 = torch.tensor(gamma, requires_grad=True)
+        bt2 = torch.tensor(beta, requires_grad=True)
+        torch.nn.functional.layer_norm(xt2, (d,), gt2, bt2, eps=1e-5).backward(torch.tensor(G_hat))
+        for k, v in (("dX", xt2.grad), ("dgamma", gt2.grad), ("dbeta", bt2.grad)):
+            mean[k] = mean[k] + pr * v.numpy()
+    assert np.allclose(mean["dX"], xt.grad.numpy(), rtol=1e-9, atol=1e-12)
+    assert np.allclose(mean["dgamma"], gt.grad.numpy(), rtol=1e-9, atol=1e-12)
+    # one seeded call: dropped data give exactly zero rows, kept data carry 1/p
+    out = o.layernorm_bwd(X, gamma, dY, N, T, 0.5, seed=3)
+    keep = out["keepA"]
+    assert 0 < keep.sum() < N
+    assert not out["dX"][np.repeat(~keep, T)].any()
+    xt3 = torch.tensor(X, requires_grad=True)
+    torch.nn.functional.layer_norm(xt3, (d,), torch.tensor(gamma), torch.tensor(beta), eps=1e-5).backward(
+        torch.tensor(o.apply_data_mask(dY, out["p32"], keep, T)))
+    assert np.allclose(out["dX"], xt3.grad.numpy(), rtol=1e-10, atol=1e-12)
