@@ -152,6 +152,22 @@ typedef struct {
 int vcas_linear_bwd_chain(vcas_handle h, const void* X, const void* dY, const void* W,
                           float rho, float nu, uint64_t seed, const vcas_chain_args* chain,
                           void* dX, float* dW, vcas_stream stream);
+/*
+ * SampleA in front of a layer that is not a matrix product (Sec. 4: SampleA is applied at every layer; App. E:
+ * for a non-linear layer the sampled, rescaled gradient G_hat is multiplied by the saved exact Jacobian):
+ * backward of Y = LayerNorm(X) * gamma + beta over the last axis, width d = d_in = d_out of the handle.
+ *   G_hat = SampleA(dY) as in vcas_linear_bwd (p_n ~ ||G_n||_F, sum p = N rho, kept data times 1/p_n);
+ *   dX = (g - mean(g) - x_hat mean(g x_hat)) / sqrt(var + eps) per row, g = G_hat * gamma, x_hat the normalised
+ *        row; [R, d] layer dtype; rows of dropped data are 0 and are not computed;
+ *   dgamma [d] = sum_r G_hat_r * x_hat_r,  dbeta [d] = sum_r G_hat_r   (fp32).
+ * gamma: [d], layer dtype.  chain may be NULL; its fields mean what they mean for vcas_linear_bwd_chain (H is
+ * ignored; a_out gets the row square-norms of dX in its first part, zeros in the others).  The kept data are
+ * read back with vcas_last_sampling (g, p, idxA, cntA; the row-wise outputs are not defined by this call).
+ */
+int vcas_layernorm_bwd(vcas_handle h, const void* X, const void* gamma, const void* dY, float eps,
+                       float rho, uint64_t seed, const vcas_chain_args* chain,
+                       void* dX, float* dgamma, float* dbeta, vcas_stream stream);
+
 /* Number of partial sums per row that this handle's dX product writes to a_out (host out). */
 int vcas_chain_parts(vcas_handle h, int32_t* parts);
 

@@ -22,7 +22,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
 
 EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
-           "vcas_linear_bwd_ex", "vcas_linear_bwd_chain", "vcas_chain_parts", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
+           "vcas_linear_bwd_ex", "vcas_linear_bwd_chain", "vcas_chain_parts", "vcas_layernorm_bwd", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
            "vcas_set_profiling", "vcas_stage_times", "vcas_set_wait_limit",
            "vcas_set_probe_subsample", "vcas_get_probe_subsample", "vcas_score_static", "vcas_set_tuning",
@@ -161,6 +161,23 @@ class Layer:
         _check(lib().vcas_linear_bwd_chain(self._h, _ptr(X), _ptr(dY), _ptr(W), C.c_float(rho), C.c_float(nu),
                                            C.c_uint64(seed), C.byref(args), _ptr(dX), _ptr(dW), _stream()),
                "vcas_linear_bwd_chain")
+
+    def layernorm_bwd(self, X, gamma, dY, rho: float, seed: int, eps: float = 1e-5, *, dX=None, a_in=None,
+                      a_in_parts: int = 1, alive_in=None, alive_cnt_in=None, a_out=None, kept_out=None,
+                      kept_cnt_out=None, skip_dropped_rows: bool = False):
+        """vcas_layernorm_bwd on a handle made with d_in = d_out = the normalised width.  Returns (dX, dgamma, dbeta)."""
+        dev = X.device
+        if dX is None:
+            dX = torch.empty(self.R, self.d_in, dtype=self.dtype, device=dev)
+        dg = torch.empty(self.d_in, dtype=torch.float32, device=dev)
+        db = torch.empty(self.d_in, dtype=torch.float32, device=dev)
+        dp = lambda t: None if t is None else t.data_ptr()
+        args = ChainArgs(None, dp(a_in), a_in_parts, dp(alive_in), dp(alive_cnt_in), dp(a_out), dp(kept_out),
+                         dp(kept_cnt_out), 1 if skip_dropped_rows else 0)
+        _check(lib().vcas_layernorm_bwd(self._h, _ptr(X), _ptr(gamma), _ptr(dY), C.c_float(eps), C.c_float(rho),
+                                        C.c_uint64(seed), C.byref(args), _ptr(dX), _ptr(dg), _ptr(db), _stream()),
+               "vcas_layernorm_bwd")
+        return dX, dg, db
 
     def chain_parts(self) -> int:
         n = C.c_int32(0)

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvcas.so")
-SOURCES = ["api.cu", "score.cu", "sampler.cu", "gemm_fma.cu", "gemm_umma.cu", "probe.cu", "score_static.cu"]
+SOURCES = ["api.cu", "score.cu", "sampler.cu", "gemm_fma.cu", "gemm_umma.cu", "probe.cu", "score_static.cu", "layernorm.cu"]
 
 
 def _stale() -> bool:

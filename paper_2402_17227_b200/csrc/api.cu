@@ -346,6 +346,36 @@ int vcas_linear_bwd_chain(vcas_handle hh, const void* X, const void* dY, const v
   return run_sampled(H(hh), X, dY, W, a, c->H, dX, dW, c->a_out, c->skip_dropped_rows != 0, S(stream));
 }
 
+int vcas_layernorm_bwd(vcas_handle hh, const void* X, const void* gamma, const void* dY, float eps, float rho,
+                       uint64_t seed, const vcas_chain_args* c, void* dX, float* dgamma, float* dbeta,
+                       vcas_stream stream) {
+  if (hh == nullptr || X == nullptr || gamma == nullptr || dY == nullptr || dX == nullptr || dgamma == nullptr ||
+      dbeta == nullptr)
+    return VCAS_ERR_BAD_ARG;
+  if (!ratio_ok(rho) || !(eps >= 0.f)) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  if (h->desc.d_in != h->desc.d_out) return VCAS_ERR_SHAPE;      // a handle made with d_in = d_out = the normalised width
+  if (h->desc.d_in < 2 * a_out_parts(h->desc.d_in)) return VCAS_ERR_SHAPE;
+  SamplerArgs a = sampler_args(rho, 1.0f, seed);
+  float* a_out = nullptr;
+  bool skip = false;
+  if (c != nullptr) {
+    if ((c->alive_in == nullptr) != (c->alive_cnt_in == nullptr)) return VCAS_ERR_BAD_ARG;
+    if ((c->kept_out == nullptr) != (c->kept_cnt_out == nullptr)) return VCAS_ERR_BAD_ARG;
+    if (c->a_in != nullptr && c->a_in_parts < 1) return VCAS_ERR_BAD_ARG;
+    a.a_in = c->a_in; a.a_parts = c->a_in != nullptr ? c->a_in_parts : 1;
+    a.alive = c->alive_in; a.alive_cnt = c->alive_cnt_in;
+    a.kept_out = c->kept_out; a.kept_cnt_out = c->kept_cnt_out;
+    a_out = c->a_out;
+    skip = c->skip_dropped_rows != 0;
+  }
+  cudaStream_t st = S(stream);
+  VCAS_CUDA(launch_rownorm_dy(h, dY, a, st));
+  VCAS_CUDA(launch_sample_a(h, a, a.a_in == nullptr, st));
+  VCAS_CUDA(launch_layernorm_bwd(h, X, gamma, dY, eps, dX, a_out, skip, dgamma, dbeta, rho, st));
+  return VCAS_OK;
+}
+
 int vcas_chain_parts(vcas_handle hh, int32_t* parts) {
   if (hh == nullptr || parts == nullptr) return VCAS_ERR_BAD_ARG;
   *parts = a_out_parts(H(hh)->desc.d_in);

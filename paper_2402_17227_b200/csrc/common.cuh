@@ -360,6 +360,11 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
 void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spare_sms, bool row_norms_out, Plan* dx,
                    Plan* dw);
 
+// LayerNorm backward over the rows of kept data (after SampleA): dX, optional row square-norms of dX, dgamma, dbeta
+cudaError_t launch_layernorm_bwd(Handle* h, const void* X, const void* gamma, const void* dY, float eps, void* dX,
+                                 float* a_out, bool skip_dropped, float* dgamma, float* dbeta, float rho_hint,
+                                 cudaStream_t st);
+
 // probe reductions
 cudaError_t launch_probe_reset(Handle* h, cudaStream_t st);
 cudaError_t launch_probe_welford(Handle* h, int i, cudaStream_t st);
