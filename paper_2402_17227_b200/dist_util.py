@@ -1,6 +1,8 @@
 """Host-side helpers for running the sampled backward as data-parallel replicas (one process per
-GPU): which synthetic batches a rank owns, and how per-rank times combine into the job's metric.
-The paper's data-parallel runs sample per replica (App. C); there is no data-path exchange here."""
+GPU): which synthetic batches a rank owns, how per-rank times combine into the job's metric, and the
+sum of the replicas' parameter gradients.  The paper's data-parallel runs sample per replica (App. C):
+the sampled backward itself needs no exchange; the only exchange of a data-parallel step is the
+all-reduce of every layer's dW, which App. C names as what limits the time gained."""
 from __future__ import annotations
 
 import torch
@@ -25,3 +27,24 @@ def ms_per_layer(ms_per_step: float, calls_per_step: int, world: int) -> float:
     """Whole-job milliseconds per layer backward: `world` replicas each finish `calls_per_step`
     backward calls in `ms_per_step` (weak scaling: the work per GPU is fixed)."""
     return ms_per_step / (calls_per_step * world)
+
+
+class GradReducer:
+    """Sums the replicas' parameter gradients, overlapped with the backward of the layers below: a layer's
+    all-reduce is issued as soon as its backward call is enqueued (the collective runs on the communication
+    library's own stream, ordered after the work enqueued so far), and is only waited for at the end of the
+    pass, before an optimiser would read the gradients.  Every replica's estimator is unbiased for its shard,
+    so the sum over replicas is unbiased for the batch (divide by the world size for the mean)."""
+
+    def __init__(self):
+        self.works = []
+        self.active = dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1
+
+    def reduce_async(self, dW: torch.Tensor) -> None:
+        if self.active:
+            self.works.append(dist.all_reduce(dW, op=dist.ReduceOp.SUM, async_op=True))
+
+    def wait(self) -> None:
+        for w in self.works:
+            w.wait()
+        self.works.clear()
