@@ -802,6 +802,8 @@ def main():
         def ddp_period():
             for k in range(F_CALLS):
                 b = k % N_BATCHES
+                if len(red.works) >= 4:
+                    red.works.pop(0).wait()     # the buffer about to be rewritten has been reduced
                 layer.linear_bwd_plain(Xs[b], dYs[b], W, RHO, NU, 777000 + k, dX, dWs[k % 4])
                 red.reduce_async(dWs[k % 4])
             red.wait()
