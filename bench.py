@@ -496,7 +496,8 @@ def measure_bert_large_stack(vb, inputs, torch, dev, steps=200, F=50, M=2):
             W = (torch.randn(d_out, d_in, generator=gw, device=dev, dtype=torch.float32) * 0.02).to(bf)
             Xs, dYs, H = pool[name]
             layers.append(StackLayer(f"b{blk}.{name}", d_in, d_out, W, Xs, dYs, H=H, chained=chained))
-    stack = LinearStack(layers, N, T, config=cfg, skip_dropped_rows=True)    # every consumer takes the kept-data list
+    # every consumer takes the kept-data list; a layer's dW branch runs beside the layers below it
+    stack = LinearStack(layers, N, T, config=cfg, skip_dropped_rows=True, overlap_layers=True)
     for hd in stack.handles.values():
         hd.set_probe_subsample(128, 0)          # App. D: the probe's variances on a sample of the parameter rows
     L = len(layers)

@@ -133,7 +133,13 @@ int vcas_linear_bwd_ex(vcas_handle h, const void* X, const void* dY, const void*
  *   kept_out     [N] int32: ascending list of the data this call kept, kept_cnt_out [1] its length;
  *   skip_dropped_rows  non-zero: the rows of dX (and a_out) that belong to dropped data are left unwritten instead
  *                of being set to zero - for a consumer that takes kept_out as its alive_in and therefore never
- *                reads them (tensor-core path; the fp32 path always writes them).
+ *                reads them (tensor-core path; the fp32 path always writes them);
+ *   defer_join   non-zero: the call returns with its weight-gradient branch (SampleW, the kept-row operands, the
+ *                dW product, which run on a stream of the handle's own) not yet joined to `stream`: dX, a_out and
+ *                kept_out are ordered on `stream` as usual, but dW and the sampling record are complete only after
+ *                vcas_join(h, stream).  The next call on the same handle joins first by itself.  In a stack this
+ *                lets the scoring and the dX product of the next layer run beside this layer's dW branch.  Under
+ *                stream capture every handle must be joined before the capture ends.
  * alive_in / alive_cnt_in and kept_out / kept_cnt_out come in pairs; the lists must not alias.  A length
  * outside [0, N] or an entry outside [0, N) is not followed: it is reported as VCAS_ERR_BAD_ARG by
  * vcas_last_device_status (the call's outputs are then undefined).
@@ -148,6 +154,7 @@ typedef struct {
   int32_t* kept_out;
   int32_t* kept_cnt_out;
   int32_t skip_dropped_rows;
+  int32_t defer_join;
 } vcas_chain_args;
 int vcas_linear_bwd_chain(vcas_handle h, const void* X, const void* dY, const void* W,
                           float rho, float nu, uint64_t seed, const vcas_chain_args* chain,
@@ -167,6 +174,9 @@ int vcas_linear_bwd_chain(vcas_handle h, const void* X, const void* dY, const vo
 int vcas_layernorm_bwd(vcas_handle h, const void* X, const void* gamma, const void* dY, float eps,
                        float rho, uint64_t seed, const vcas_chain_args* chain,
                        void* dX, float* dgamma, float* dbeta, vcas_stream stream);
+
+/* Makes `stream` wait for the branch a call with defer_join left running (no-op otherwise).  Asynchronous. */
+int vcas_join(vcas_handle h, vcas_stream stream);
 
 /* Number of partial sums per row that this handle's dX product writes to a_out (host out). */
 int vcas_chain_parts(vcas_handle h, int32_t* parts);

@@ -22,7 +22,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
 
 EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
-           "vcas_linear_bwd_ex", "vcas_linear_bwd_chain", "vcas_chain_parts", "vcas_layernorm_bwd", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
+           "vcas_linear_bwd_ex", "vcas_linear_bwd_chain", "vcas_chain_parts", "vcas_layernorm_bwd", "vcas_join", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
            "vcas_set_profiling", "vcas_stage_times", "vcas_set_wait_limit",
            "vcas_set_probe_subsample", "vcas_get_probe_subsample", "vcas_score_static", "vcas_set_tuning",
@@ -53,7 +53,7 @@ class State(C.Structure):
 class ChainArgs(C.Structure):
     _fields_ = [("H", C.c_void_p), ("a_in", C.c_void_p), ("a_in_parts", C.c_int32), ("alive_in", C.c_void_p),
                 ("alive_cnt_in", C.c_void_p), ("a_out", C.c_void_p), ("kept_out", C.c_void_p),
-                ("kept_cnt_out", C.c_void_p), ("skip_dropped_rows", C.c_int32)]
+                ("kept_cnt_out", C.c_void_p), ("skip_dropped_rows", C.c_int32), ("defer_join", C.c_int32)]
 
 
 _lib = None
@@ -152,12 +152,12 @@ class Layer:
 
     def linear_bwd_chain(self, X, dY, W, rho: float, nu: float, seed: int, dX, dW, *, H=None, a_in=None,
                          a_in_parts: int = 1, alive_in=None, alive_cnt_in=None, a_out=None, kept_out=None,
-                         kept_cnt_out=None, skip_dropped_rows: bool = False):
+                         kept_cnt_out=None, skip_dropped_rows: bool = False, defer_join: bool = False):
         """vcas_linear_bwd_chain: scores handed down from the layer above (a_in, alive_in) and to the layer
         below (a_out, kept_out); every extra is an optional device tensor."""
         dp = lambda t: None if t is None else t.data_ptr()
         args = ChainArgs(dp(H), dp(a_in), a_in_parts, dp(alive_in), dp(alive_cnt_in), dp(a_out), dp(kept_out),
-                         dp(kept_cnt_out), 1 if skip_dropped_rows else 0)
+                         dp(kept_cnt_out), 1 if skip_dropped_rows else 0, 1 if defer_join else 0)
         _check(lib().vcas_linear_bwd_chain(self._h, _ptr(X), _ptr(dY), _ptr(W), C.c_float(rho), C.c_float(nu),
                                            C.c_uint64(seed), C.byref(args), _ptr(dX), _ptr(dW), _stream()),
                "vcas_linear_bwd_chain")
@@ -173,11 +173,14 @@ class Layer:
         db = torch.empty(self.d_in, dtype=torch.float32, device=dev)
         dp = lambda t: None if t is None else t.data_ptr()
         args = ChainArgs(None, dp(a_in), a_in_parts, dp(alive_in), dp(alive_cnt_in), dp(a_out), dp(kept_out),
-                         dp(kept_cnt_out), 1 if skip_dropped_rows else 0)
+                         dp(kept_cnt_out), 1 if skip_dropped_rows else 0, 0)
         _check(lib().vcas_layernorm_bwd(self._h, _ptr(X), _ptr(gamma), _ptr(dY), C.c_float(eps), C.c_float(rho),
                                         C.c_uint64(seed), C.byref(args), _ptr(dX), _ptr(dg), _ptr(db), _stream()),
                "vcas_layernorm_bwd")
         return dX, dg, db
+
+    def join(self) -> None:
+        _check(lib().vcas_join(self._h, _stream()), "vcas_join")
 
     def chain_parts(self) -> int:
         n = C.c_int32(0)

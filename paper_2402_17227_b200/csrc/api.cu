@@ -137,6 +137,16 @@ int sample_w_and_dw(Handle* h, const void* X, const void* dY, const SamplerArgs&
   return VCAS_OK;
 }
 
+// A call that deferred its join left work on the side stream: everything that touches the handle's workspace
+// or the outputs of that call waits for it first.
+int join_pending(Handle* h, cudaStream_t st) {
+  if (h->join_pending) {
+    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
+    h->join_pending = false;
+  }
+  return VCAS_OK;
+}
+
 // stage boundary k of the current sampled call (no-op unless profiling is on)
 inline void mark(Handle* h, int k, cudaStream_t st) {
   if (h->prof_enabled && h->prof_calls < PROF_RING) cudaEventRecord(h->ev[h->prof_calls * 8 + k], st);
@@ -200,6 +210,7 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->plan_valid = false;
   h->wait_limit_ns = 2000000000ull;
   h->sub_k = 0;
+  h->join_pending = false;
   h->stall_once = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&h->device) != cudaSuccess || cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) {
@@ -268,7 +279,8 @@ namespace {
 // One sampled backward (Eq. 2).  `a` carries the ratios, the seed, the optional given probabilities and the
 // optional scores handed down from the layer above; a_out: optional row square-norms of dX for the layer below.
 int run_sampled(Handle* h, const void* X, const void* dY, const void* W, const SamplerArgs& a, const void* Hpre,
-                void* dX, float* dW, float* a_out, bool skip_dropped, cudaStream_t st) {
+                void* dX, float* dW, float* a_out, bool skip_dropped, bool defer_join, cudaStream_t st) {
+  if (join_pending(h, st) != VCAS_OK) return VCAS_ERR_CUDA;
   const int hint = (int)(a.rho * a.nu * (float)(h->desc.N * h->desc.T)) + 1;
   // The sampled dX grid leaves one SM free: SampleW's single-CTA kernel, which runs beside it on the side
   // stream, needs a whole SM's shared memory.
@@ -313,7 +325,8 @@ int run_sampled(Handle* h, const void* X, const void* dY, const void* W, const S
     const int rc = sample_w_and_dw(h, X, dY, a, false, &pw, dW, h->side_stream);
     if (rc != VCAS_OK) return rc;
     VCAS_CUDA(cudaEventRecord(h->ev_join, h->side_stream));
-    VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
+    if (defer_join) h->join_pending = true;       // dW and the sampling record are complete only after vcas_join
+    else VCAS_CUDA(cudaStreamWaitEvent(st, h->ev_join, 0));
   }
   if (h->prof_enabled && h->prof_calls < PROF_RING) h->prof_calls += 1;
   return VCAS_OK;
@@ -328,7 +341,7 @@ int vcas_linear_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
   SamplerArgs a = sampler_args(rho, nu, seed);
   a.p_in = p_in; a.q_in = q_in;
-  return run_sampled(H(hh), X, dY, W, a, Hpre, dX, dW, nullptr, false, S(stream));
+  return run_sampled(H(hh), X, dY, W, a, Hpre, dX, dW, nullptr, false, false, S(stream));
 }
 
 int vcas_linear_bwd_chain(vcas_handle hh, const void* X, const void* dY, const void* W, float rho, float nu,
@@ -343,7 +356,8 @@ int vcas_linear_bwd_chain(vcas_handle hh, const void* X, const void* dY, const v
   a.a_in = c->a_in; a.a_parts = c->a_in != nullptr ? c->a_in_parts : 1;
   a.alive = c->alive_in; a.alive_cnt = c->alive_cnt_in;
   a.kept_out = c->kept_out; a.kept_cnt_out = c->kept_cnt_out;
-  return run_sampled(H(hh), X, dY, W, a, c->H, dX, dW, c->a_out, c->skip_dropped_rows != 0, S(stream));
+  return run_sampled(H(hh), X, dY, W, a, c->H, dX, dW, c->a_out, c->skip_dropped_rows != 0, c->defer_join != 0,
+                     S(stream));
 }
 
 int vcas_layernorm_bwd(vcas_handle hh, const void* X, const void* gamma, const void* dY, float eps, float rho,
@@ -370,10 +384,16 @@ int vcas_layernorm_bwd(vcas_handle hh, const void* X, const void* gamma, const v
     skip = c->skip_dropped_rows != 0;
   }
   cudaStream_t st = S(stream);
+  if (join_pending(h, st) != VCAS_OK) return VCAS_ERR_CUDA;
   VCAS_CUDA(launch_rownorm_dy(h, dY, a, st));
   VCAS_CUDA(launch_sample_a(h, a, a.a_in == nullptr, st));
   VCAS_CUDA(launch_layernorm_bwd(h, X, gamma, dY, eps, dX, a_out, skip, dgamma, dbeta, rho, st));
   return VCAS_OK;
+}
+
+int vcas_join(vcas_handle hh, vcas_stream stream) {
+  if (hh == nullptr) return VCAS_ERR_BAD_ARG;
+  return join_pending(H(hh), S(stream));
 }
 
 int vcas_chain_parts(vcas_handle hh, int32_t* parts) {
@@ -393,6 +413,7 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
     return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
+  if (join_pending(h, st) != VCAS_OK) return VCAS_ERR_CUDA;
   cudaStream_t sw = st;
   const bool fork = h->tensor_path && !h->prof_enabled;
   if (fork) {
@@ -427,6 +448,7 @@ int vcas_score(vcas_handle hh, const void* X, const void* dY, float rho, float n
   if (!ratio_ok(rho) || !ratio_ok(nu)) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
+  if (join_pending(h, st) != VCAS_OK) return VCAS_ERR_CUDA;
   const SamplerArgs a = sampler_args(rho, nu, seed);
   VCAS_CUDA(launch_rownorm_dy(h, dY, a, st));
   VCAS_CUDA(launch_sample_a(h, a, true, st));
@@ -439,6 +461,7 @@ int vcas_score(vcas_handle hh, const void* X, const void* dY, float rho, float n
 int vcas_last_sampling(vcas_handle hh, float* g, float* p, float* w, float* q, int32_t* idxA, int32_t* cntA,
                        int32_t* idxW, int32_t* cntW, vcas_stream stream) {
   if (hh == nullptr) return VCAS_ERR_BAD_ARG;
+  if (join_pending(H(hh), S(stream)) != VCAS_OK) return VCAS_ERR_CUDA;
   return copy_out(H(hh), g, p, w, q, idxA, cntA, idxW, cntW, S(stream));
 }
 
@@ -459,6 +482,7 @@ int vcas_variance_probe(vcas_handle hh, int32_t M, const void* const* X_i, const
     if (X_i[i] == nullptr || dY_i[i] == nullptr) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   cudaStream_t st = S(stream);
+  if (join_pending(h, st) != VCAS_OK) return VCAS_ERR_CUDA;
   const double alpha = (double)h->cfg.alpha;
   double s_lo = (double)s - alpha, s_hi = (double)s + alpha;
   if (s_lo < 0.0) s_lo = 0.0;
@@ -643,6 +667,7 @@ int vcas_last_device_status(vcas_handle hh, int32_t* status) {
   if (hh == nullptr || status == nullptr) return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   VCAS_CUDA(cudaDeviceSynchronize());
+  h->join_pending = false;
   VCAS_CUDA(cudaMemcpy(status, h->ws.status, sizeof(int32_t), cudaMemcpyDeviceToHost));
   VCAS_CUDA(cudaMemset(h->ws.status, 0, sizeof(int32_t)));
   if (*status != VCAS_OK && h->tensor_path) {

@@ -74,6 +74,7 @@ struct Handle {
   // second stream and fork/join events: the dW branch (pack + product) runs beside the dX product
   cudaStream_t side_stream;
   cudaEvent_t ev_fork, ev_join;
+  bool join_pending;   // the last call left its side-stream branch unjoined (vcas_chain_args::defer_join)
   // optional stage timing (vcas_set_profiling): rings of CUDA events around the stages
   bool prof_enabled;
   cudaEvent_t* ev;        // [PROF_RING][8]: stage boundaries of a sampled call (see vcas_stage_times)

@@ -429,7 +429,6 @@ struct EmitParams {
 };
 
 // Row k of packG = scaleW[k] * dY[idxW[k]] (G_tilde of Sec. 4.2, rounded to bf16), row k of packX = X[idxW[k]].
-// Four independent 16-byte loads per thread are in flight.
 __device__ __forceinline__ uint4 scale8(const uint4& v, float sc) {
   const uint32_t u[4] = {v.x, v.y, v.z, v.w};
   uint32_t o[4];
@@ -440,24 +439,6 @@ __device__ __forceinline__ uint4 scale8(const uint4& v, float sc) {
   }
   return make_uint4(o[0], o[1], o[2], o[3]);
 }
-__device__ __forceinline__ void pack_row(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int d,
-                                         float sc, bool scaled) {
-  const uint4* __restrict__ in = reinterpret_cast<const uint4*>(src);
-  uint4* __restrict__ out = reinterpret_cast<uint4*>(dst);
-  const int nv = d / 8, nt = blockDim.x;
-  int i = threadIdx.x;
-  for (; i + 3 * nt < nv; i += 4 * nt) {
-    uint4 v0 = __ldg(in + i), v1 = __ldg(in + i + nt), v2 = __ldg(in + i + 2 * nt), v3 = __ldg(in + i + 3 * nt);
-    if (scaled) { v0 = scale8(v0, sc); v1 = scale8(v1, sc); v2 = scale8(v2, sc); v3 = scale8(v3, sc); }
-    out[i] = v0; out[i + nt] = v1; out[i + 2 * nt] = v2; out[i + 3 * nt] = v3;
-  }
-  for (; i < nv; i += nt) {
-    uint4 v = __ldg(in + i);
-    if (scaled) v = scale8(v, sc);
-    out[i] = v;
-  }
-}
-
 // One CTA per (chunk of 32 compact rows, part) (grid-strided): the chunk's kept rows go to positions
 // chunk_off[ch]... of the ascending kept-row list with their rescale factors 1/(p_n q_r); q and w are written by
 // global row (by part 0); the operands of the chunk's kept rows j with j % parts == part are packed for the dW
@@ -507,11 +488,39 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
     }
     if (pack) {
       __syncthreads();
+      // this part's rows j = part, part + parts, ...: their 16-byte pieces of both operands are spread over the
+      // CTA's threads, four independent loads per thread in flight whatever the width of a row
       const int m = s_cnt;
-      for (int j = part; j < m; j += parts) {
-        const size_t r = (size_t)s_r[j], pos = (size_t)s_pos[j];
-        pack_row(P.dY + r * P.d_out, P.packG + pos * P.d_out, P.d_out, s_sc[j], true);
-        pack_row(P.X + r * P.d_in, P.packX + pos * P.d_in, P.d_in, 1.f, false);
+      const int mp = m > part ? (m - part + parts - 1) / parts : 0;
+      const int vo = P.d_out / 8, vt = vo + P.d_in / 8;
+      const int total = mp * vt;
+      for (int it0 = tid; it0 < total; it0 += 4 * EMIT_THREADS) {
+        uint4 v[4];
+        uint4* dst[4];
+        float scl[4];
+        bool isg[4];
+#pragma unroll
+        for (int u4 = 0; u4 < 4; ++u4) {
+          const int it = it0 + u4 * EMIT_THREADS;
+          dst[u4] = nullptr;
+          if (it < total) {
+            const int jj = it / vt, piece = it - jj * vt;
+            const int j = part + jj * parts;
+            const size_t r = (size_t)s_r[j], pos = (size_t)s_pos[j];
+            isg[u4] = piece < vo;
+            scl[u4] = s_sc[j];
+            if (isg[u4]) {
+              v[u4] = __ldg(reinterpret_cast<const uint4*>(P.dY + r * P.d_out) + piece);
+              dst[u4] = reinterpret_cast<uint4*>(P.packG + pos * P.d_out) + piece;
+            } else {
+              v[u4] = __ldg(reinterpret_cast<const uint4*>(P.X + r * P.d_in) + (piece - vo));
+              dst[u4] = reinterpret_cast<uint4*>(P.packX + pos * P.d_in) + (piece - vo);
+            }
+          }
+        }
+#pragma unroll
+        for (int u4 = 0; u4 < 4; ++u4)
+          if (dst[u4] != nullptr) *dst[u4] = isg[u4] ? scale8(v[u4], scl[u4]) : v[u4];
       }
       __syncthreads();
     }

@@ -44,11 +44,14 @@ class LinearStack:
     the calls of a pass follow one another on one stream)."""
 
     def __init__(self, layers: list[StackLayer], N: int, T: int, dtype=torch.bfloat16, config=None,
-                 gemm_path: int = vb.GEMM_AUTO, skip_dropped_rows: bool = False):
+                 gemm_path: int = vb.GEMM_AUTO, skip_dropped_rows: bool = False, overlap_layers: bool = False):
         """skip_dropped_rows: the rows of dX that belong to dropped data are not written (every consumer in the
         stack takes the kept-data list and never reads them); the dX buffers then hold stale rows there."""
         self.layers, self.N, self.T, self.dtype = layers, N, T, dtype
         self.skip_dropped_rows = skip_dropped_rows
+        # overlap_layers: a layer's weight-gradient branch is left running while the next layers are scored and
+        # their dX products run (vcas_chain_args::defer_join); all handles are joined at the end of the pass
+        self.overlap_layers = overlap_layers
         self.R = N * T
         self.handles: dict = {}
         dev = layers[0].W.device
@@ -92,10 +95,13 @@ class LinearStack:
                 hook(i, L, False)
             L.handle.linear_bwd_chain(L.X[v], dY, L.W, float(rho[i]), float(nu[i]), seed * len(self.layers) + i,
                                       L.dX, L.dW, H=H, a_out=L.a_out, kept_out=L.kept, kept_cnt_out=L.kept_cnt,
-                                      skip_dropped_rows=self.skip_dropped_rows, **kw)
+                                      skip_dropped_rows=self.skip_dropped_rows, defer_join=self.overlap_layers, **kw)
             if hook is not None:
                 hook(i, L, True)
             prev = L
+        if self.overlap_layers:
+            for h in self.handles.values():
+                h.join()
 
     def dense_backward(self, variant: int = 0, hook=None) -> None:
         """The exact backward of the same layers (no sampling, no Jacobian factor): the dense comparison."""

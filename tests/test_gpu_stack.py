@@ -196,3 +196,37 @@ def test_skip_dropped_rows_leaves_them_untouched():
     assert torch.all(dX[~rows] == 7.0)
     assert lay.device_status() == 0
     lay.close()
+
+
+def test_overlapped_layers_give_the_same_bits():
+    """With defer_join a layer's weight-gradient branch runs beside the next layers; results are unchanged, also when
+    a pass is replayed from a CUDA graph."""
+    vbuild.build()
+    dev = torch.device("cuda")
+    N, T, d, ffn, qkv = 8, 64, 256, 512, 384
+    outs = []
+    for overlap in (False, True):
+        layers = []
+        for block in (2, 1, 0):
+            layers += make_block_layers(N, T, d, ffn, qkv, block, 1, dev)
+        stack = LinearStack(layers, N, T, gemm_path=vb.GEMM_TENSOR, overlap_layers=overlap, skip_dropped_rows=True)
+        L = len(layers)
+        rho, nu = np.linspace(0.8, 0.4, L), np.full(L, 0.5)
+        stack.backward(rho, nu, seed=5)
+        torch.cuda.synchronize()
+        res = [(l.dW.clone(), l.kept.clone(), l.kept_cnt.clone()) for l in layers]
+        if overlap:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                stack.backward(rho, nu, seed=5)
+            for l in layers:
+                l.dW.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            for l, (dW, kept, cnt) in zip(layers, res):
+                assert torch.equal(l.dW, dW) and torch.equal(l.kept_cnt, cnt)
+        outs.append(res)
+        assert stack.device_status() == 0
+        stack.close()
+    for (dW0, k0, c0), (dW1, k1, c1) in zip(*outs):
+        assert torch.equal(dW0, dW1) and torch.equal(c0, c1) and torch.equal(k0[:int(c0.item())], k1[:int(c1.item())])
