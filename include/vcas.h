@@ -292,13 +292,19 @@ int vcas_set_wait_limit(vcas_handle h, uint64_t limit_ns, int32_t stall_once);
 /* Tuning overrides for the tensor-core products (the paper has no counterpart): output tile
  * width of the dX and dW kernels (64, 128 or 256), the number of slices each contraction is
  * split into (1..16; slices are combined in a fixed order, so results stay reproducible), and
- * the tile height (tile_m = 1: 128 rows, 2: 256 rows whenever the width is 256 and the
+ * the tile height of each product (dx_tile_m, dw_tile_m = 1: 128 rows, 2: 256 rows whenever the width is 256 and the
  * contraction is not sliced, 3: 256 rows for as many tiles as fill all SMs a whole number of
  * times and 128 rows with a sliced contraction, in a second launch, for the rest).
  * 0 = let the library choose from the shapes and ratios.  VCAS_ERR_BAD_ARG for a value outside
  * these sets. */
 int vcas_set_tuning(vcas_handle h, int32_t dx_tile_n, int32_t dw_tile_n, int32_t dx_split_k, int32_t dw_split_k,
-                    int32_t tile_m);
+                    int32_t dx_tile_m, int32_t dw_tile_m);
+
+/* The tilings the library chose for the two products of the handle's last sampled or dense call (the paper has
+ * no counterpart): plan[0..2] = tile width, contraction slices, tile-height code (as in vcas_set_tuning) of the dX
+ * product, plan[3..5] the same for the dW product (host out).  VCAS_ERR_BAD_ARG before the first call or on the
+ * fp32-FMA path. */
+int vcas_last_plan(vcas_handle h, int32_t* plan);
 
 /* Stage timing for benchmarks (the paper has no counterpart; Sec. 6 only reports end-to-end
  * hours).  While enabled, vcas_linear_bwd(_ex) and vcas_dense_bwd record CUDA events on the

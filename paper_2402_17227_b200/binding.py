@@ -26,7 +26,7 @@ EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
            "vcas_set_profiling", "vcas_stage_times", "vcas_set_wait_limit",
            "vcas_set_probe_subsample", "vcas_get_probe_subsample", "vcas_score_static", "vcas_set_tuning",
-           "vcas_version"]
+           "vcas_last_plan", "vcas_version"]
 
 
 class VcasError(RuntimeError):
@@ -255,9 +255,17 @@ class Layer:
         return st.value
 
     def set_tuning(self, dx_tile_n: int = 0, dw_tile_n: int = 0, dx_split_k: int = 0, dw_split_k: int = 0,
-                   tile_m: int = 0) -> None:
+                   tile_m: int = 0, dw_tile_m: int | None = None) -> None:
+        """tile_m: tile height of the dX product, and of the dW product too unless dw_tile_m is given."""
         _check(lib().vcas_set_tuning(self._h, C.c_int32(dx_tile_n), C.c_int32(dw_tile_n), C.c_int32(dx_split_k),
-                                     C.c_int32(dw_split_k), C.c_int32(tile_m)), "vcas_set_tuning")
+                                     C.c_int32(dw_split_k), C.c_int32(tile_m),
+                                     C.c_int32(tile_m if dw_tile_m is None else dw_tile_m)), "vcas_set_tuning")
+
+    def last_plan(self):
+        """((width, slices, height code) of the dX product, the same of the dW product) of the last call."""
+        a = (C.c_int32 * 6)()
+        _check(lib().vcas_last_plan(self._h, a), "vcas_last_plan")
+        return tuple(a[0:3]), tuple(a[3:6])
 
     def set_probe_subsample(self, rows: int, seed: int = 0) -> None:
         _check(lib().vcas_set_probe_subsample(self._h, C.c_int32(rows), C.c_uint64(seed)), "vcas_set_probe_subsample")

@@ -206,7 +206,7 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->ev_dense = nullptr;
   h->prof_calls = h->prof_dense_calls = 0;
   h->tune_dx_tile_n = h->tune_dw_tile_n = h->tune_dx_split_k = h->tune_dw_split_k = 0;
-  h->tune_tile_m = 0;
+  h->tune_dx_tile_m = h->tune_dw_tile_m = 0;
   h->plan_valid = false;
   h->wait_limit_ns = 2000000000ull;
   h->sub_k = 0;
@@ -577,17 +577,28 @@ int vcas_update_ratios(vcas_state* state, int32_t L, const float* V_s, const flo
 }
 
 int vcas_set_tuning(vcas_handle hh, int32_t dx_tile_n, int32_t dw_tile_n, int32_t dx_split_k, int32_t dw_split_k,
-                    int32_t tile_m) {
+                    int32_t dx_tile_m, int32_t dw_tile_m) {
   if (hh == nullptr) return VCAS_ERR_BAD_ARG;
   auto tile_ok = [](int32_t t) { return t == 0 || t == 64 || t == 128 || t == 256; };
   if (!tile_ok(dx_tile_n) || !tile_ok(dw_tile_n) || dx_split_k < 0 || dx_split_k > 16 ||
-      dw_split_k < 0 || dw_split_k > 16 || tile_m < 0 || tile_m > 3) return VCAS_ERR_BAD_ARG;
+      dw_split_k < 0 || dw_split_k > 16 || dx_tile_m < 0 || dx_tile_m > 3 || dw_tile_m < 0 || dw_tile_m > 3)
+    return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
   h->tune_dx_tile_n = dx_tile_n;
   h->tune_dw_tile_n = dw_tile_n;
   h->tune_dx_split_k = dx_split_k;
   h->tune_dw_split_k = dw_split_k;
-  h->tune_tile_m = tile_m;
+  h->tune_dx_tile_m = dx_tile_m;
+  h->tune_dw_tile_m = dw_tile_m;
+  return VCAS_OK;
+}
+
+int vcas_last_plan(vcas_handle hh, int32_t* plan) {
+  if (hh == nullptr || plan == nullptr) return VCAS_ERR_BAD_ARG;
+  Handle* h = H(hh);
+  if (!h->tensor_path || !h->plan_valid) return VCAS_ERR_BAD_ARG;
+  plan[0] = h->plan_dx.bn; plan[1] = h->plan_dx.split; plan[2] = h->plan_dx.mh;
+  plan[3] = h->plan_dw.bn; plan[4] = h->plan_dw.split; plan[5] = h->plan_dw.mh;
   return VCAS_OK;
 }
 

@@ -92,7 +92,7 @@ struct Handle {
   void* sub_dY;        // [R, SUB_MAX] those columns of the current batch's dY, compact
   unsigned long long wait_limit_ns;   // bound of every device-side wait (default 2 s)
   int stall_once;    // test hook, see vcas_set_wait_limit
-  int tune_tile_m;   // 0 auto, 1: 128-row tiles only, 2: 256-row tiles whenever the width is 256, 3: 256-row tiles for
+  int tune_dx_tile_m, tune_dw_tile_m;   // per product; 0 auto, 1: 128-row tiles only, 2: 256-row tiles whenever the width is 256, 3: 256-row tiles for
                      // whole waves of CTAs and 128-row tiles, their contraction sliced, for the rest
 };
 constexpr int PROF_RING = 2048;

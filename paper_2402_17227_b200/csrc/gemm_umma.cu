@@ -912,13 +912,16 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tile shape and number of contraction slices from a small cost model, calibrated on B200 with
-// in-kernel timestamps: a k-block costs about 0.5 / 0.45 / 0.43 us for 256 / 128 / 64 wide tiles
-// (the shared-memory fill rate of one SM bounds it, so narrow tiles only pay off when they fill
-// more SMs); a unit costs about 4 us of set-up, pipeline fill and output store; a sliced unit
-// about 3 us more for its partial store, and the unit that comes last adds the S partial tiles of the whole
-// tile (about 2.5 us per slice); a 256 x 256 tile (mh = 2) costs
-// about 0.62 us per k-block for twice the work, and 7 us per tile.
+// Tile shape and number of contraction slices from a small cost model of the kernel instances (per
+// unit of work, so independent of the layer's shape), fitted to serialised stage times of every tiling
+// on five layer shapes on B200: a k-block costs about 0.50 / 0.45 / 0.43 us for 256 / 128 / 64 wide
+// 128-row tiles (the shared-memory fill rate of one SM bounds it, so narrow tiles only pay off when
+// they fill more SMs); a unit costs about 4 us of set-up, pipeline fill and output store; a sliced unit
+// pays for its partial store and the unit that comes last adds the S partial tiles of the whole tile
+// through L2: about 20 us + 1.5 us per slice on the critical path, so that slicing only pays for long
+// contractions with few tiles; a 256 x 256 tile (mh = 2) costs about 0.66 us per k-block for twice the
+// work, and 7 us per tile.
+constexpr double SLICED_US = 20.0, SLICED_PER_SLICE_US = 1.5;
 struct Cand {
   Plan plan;
   long units;      // (tile, slice) units
@@ -947,12 +950,12 @@ int enumerate_plans(long row_tiles128, long row_tiles256, int n_extent, int kblo
       if (sp > 1 && force_split == 0 && kblocks / sp < 4) continue;   // slices too short to pay off
       const long units = tiles * sp;
       const double waves = (double)((units + num_sms - 1) / num_sms);
-      const double unit = (double)((kblocks + sp - 1) / sp) * c_kb[i] + (sp > 1 ? 7.0 + 2.5 * sp : 4.0);
+      const double unit = (double)((kblocks + sp - 1) / sp) * c_kb[i] + (sp > 1 ? SLICED_US + SLICED_PER_SLICE_US * sp : 4.0);
       if (n < MAX_CANDS) out[n++] = {{widths[i], sp, 1}, units, unit, waves * unit};
     }
     if (widths[i] == 256 && force_split <= 1) {                        // 256 x 256 tiles, never sliced
       const long units = row_tiles256 * ntiles;
-      const double wave = (double)kblocks * 0.62 + 7.0;
+      const double wave = (double)kblocks * 0.66 + 7.0;
       if (n < MAX_CANDS) out[n++] = {{256, 1, 2}, units, wave, (double)((units + num_sms - 1) / num_sms) * wave};
       const long frac = units % num_sms;
       if (remainder_ok && frac > 0 && 2 * frac <= num_sms) {            // whole waves, then the rest as sliced 128-row tiles
@@ -960,7 +963,9 @@ int enumerate_plans(long row_tiles128, long row_tiles256, int n_extent, int kblo
         if (sp > 8) sp = 8;
         if (sp > kblocks / 4) sp = kblocks / 4;
         if (sp < 1) sp = 1;
-        const double tail = (double)((kblocks + sp - 1) / sp) * 0.50 + (sp > 1 ? 7.0 + 2.5 * (double)sp : 4.0) + 4.0;
+        // the second launch always runs the sliced instance (its tiles go through the slice exchange even when
+        // a contraction ends up in one slice), and costs a launch of its own
+        const double tail = (double)((kblocks + sp - 1) / sp) * 0.50 + SLICED_US + SLICED_PER_SLICE_US * (double)sp + 4.0;
         if (n < MAX_CANDS) out[n++] = {{256, 1, 3}, units, wave, (double)(units / num_sms) * wave + tail};
       }
     }
@@ -970,10 +975,10 @@ int enumerate_plans(long row_tiles128, long row_tiles256, int n_extent, int kblo
 }
 
 // the tile-height override of vcas_set_tuning, applied to a chosen plan
-Plan apply_tile_m(const Handle* h, Plan plan, bool remainder_ok) {
-  if (h->tune_tile_m == 1) plan.mh = 1;
-  if (h->tune_tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
-  if (h->tune_tile_m == 3 && plan.bn == 256 && remainder_ok) { plan.mh = 3; plan.split = 1; }
+Plan apply_tile_m(int tile_m, Plan plan, bool remainder_ok) {
+  if (tile_m == 1) plan.mh = 1;
+  if (tile_m == 2 && plan.bn == 256) { plan.mh = 2; plan.split = 1; }
+  if (tile_m == 3 && plan.bn == 256 && remainder_ok) { plan.mh = 3; plan.split = 1; }
   return plan;
 }
 
@@ -985,11 +990,54 @@ Plan best_alone(const Cand* c, int n) {
 }
 
 // The two products of one call run at the same time on two streams.  Model: the first product's CTAs are
-// resident from time 0, the second's become ready `offset` us later and take the SMs that are free then, or,
-// if those are too few, wait for the first product's CTAs to leave.  (Measured on the benchmark layer: a
-// dense call takes 63 us when the two grids together exceed the SMs, 52 us when the dW product runs as 36
-// tiles of 256 x 256 beside the 96 CTAs of the dX product.)
+// resident from time 0 and leave after their last unit (a grid whose last wave is partial frees the CTAs without
+// a unit in it one unit time earlier); the second product becomes ready `offset` us later and works its units
+// off on the SMs that are free at the time - a persistent CTA of the second grid simply starts when an SM frees
+// up and draws units until none are left.  (Measured on the BERT-base layer: a dense call takes 63 us when the
+// two grids together exceed the SMs and every unit of the second waits for the first, 52 us when the dW product
+// runs as 36 tiles of 256 x 256 beside the 96 CTAs of the dX product.)
 constexpr double KERNEL_US = 3.0;   // launch ramp and exit of a product kernel, on top of its units (timeline measurements)
+
+// Finish time of the second product: `units` units of `unit` us each, ready at `ready`, on the SMs the first
+// product (g1 CTAs, `units1` units of `unit1` us) leaves free.
+// slices > 1: the sliced instance assigns its units to CTAs in advance (CTA i takes units i, i + upi, ...), so the
+// CTAs that start first are also the ones with the most units.
+double second_end(long units, double unit, long g2, int slices, double ready, long g1, long units1, double unit1,
+                  int num_sms) {
+  const long full = units1 / g1, rest = units1 % g1;
+  // phases of the first product: [0, full * unit1) all g1 CTAs busy; [full * unit1, (full + 1) * unit1) only
+  // `rest` of them (if any); afterwards none
+  const double t_a = (double)full * unit1 + KERNEL_US;
+  const double t_b = rest > 0 ? t_a + unit1 : t_a;
+  const long busy[3] = {g1, rest, 0};
+  const double from[3] = {0.0, t_a, t_b};
+  const double to[3] = {t_a, t_b, 1e30};
+  long left = units;
+  double end = ready;
+  bool started = false;
+  for (int ph = 0; ph < 3 && left > 0; ++ph) {
+    long sms = num_sms - busy[ph];
+    if (sms > g2) sms = g2;
+    const double t0 = ready > from[ph] ? ready : from[ph];
+    if (sms <= 0 || t0 >= to[ph]) continue;
+    if (!started && slices > 1) {
+      const long upi = (g2 / slices) * slices;
+      const long most = upi > 0 ? (units + upi - 1) / upi : units;
+      end = t0 + (double)most * unit;
+    }
+    started = true;
+    // units that start in this phase (a unit started before the phase ends is finished by its CTA)
+    const double span = to[ph] - t0;
+    long rounds = ph == 2 ? (left + sms - 1) / sms : (long)(span / unit) + 1;
+    long can = rounds * sms;
+    if (can > left) { can = left; rounds = (left + sms - 1) / sms; }
+    left -= can;
+    const double e = t0 + (double)rounds * unit;
+    if (e > end) end = e;
+  }
+  return end + KERNEL_US;
+}
+
 void best_pair(const Cand* c1, int n1, int ctas1, const Cand* c2, int n2, int ctas2, int num_sms, double offset,
                Plan* p1, Plan* p2) {
   double best = 1e30;
@@ -1001,10 +1049,19 @@ void best_pair(const Cand* c1, int n1, int ctas1, const Cand* c2, int n2, int ct
     for (int j = 0; j < n2; ++j) {
       const bool split2 = c2[j].plan.mh == 3;
       const long g2 = split2 || c2[j].units > ctas2 ? ctas2 : c2[j].units;
-      const double d2 = (split2 ? c2[j].alone : (double)((c2[j].units + g2 - 1) / g2) * c2[j].unit) + KERNEL_US;
-      const double start2 = g2 <= num_sms - g1 ? offset : (offset > d1 ? offset : d1);
-      const double end = d1 > start2 + d2 ? d1 : start2 + d2;
-      const double t = end + 1e-3 * ((double)g1 * d1 + (double)g2 * d2) / num_sms;    // ties: less SM time
+      double end2;
+      if (split1 || split2) {
+        // a product in two launches: its time alone, after the first product unless both grids fit side by side
+        const double d2 = (split2 ? c2[j].alone : (double)((c2[j].units + g2 - 1) / g2) * c2[j].unit) + KERNEL_US;
+        const double start2 = g2 <= num_sms - g1 ? offset : (offset > d1 ? offset : d1);
+        end2 = start2 + d2;
+      } else {
+        end2 = second_end(c2[j].units, c2[j].unit, g2, c2[j].plan.split, offset, g1, c1[i].units, c1[i].unit, num_sms);
+      }
+      const double end = d1 > end2 ? d1 : end2;
+      // ties: the pair whose products finish earlier, then the one with less SM time
+      const double sm_time = (double)c1[i].units * c1[i].unit + (double)c2[j].units * c2[j].unit;
+      const double t = end + 0.02 * (d1 + end2) + 1e-3 * sm_time / num_sms;
       if (t < best - 1e-9) { best = t; *p1 = c1[i].plan; *p2 = c2[j].plan; }
     }
   }
@@ -1107,12 +1164,12 @@ DxShape dx_shape(const Handle* h, bool dense, float rho_hint) {
   g.row_tiles256 = nk * ((d.T + 2 * BM - 1) / (2 * BM));
   g.kblocks = (d.d_out + BK - 1) / BK;
   // the halves of a 256-row tile must both hold rows for the remainder launch to take them over
-  g.rem_ok = h->tune_tile_m != 2 && ((d.T % (2 * BM)) == 0 || (d.T % (2 * BM)) > BM);
+  g.rem_ok = h->tune_dx_tile_m != 2 && ((d.T % (2 * BM)) == 0 || (d.T % (2 * BM)) > BM);
   return g;
 }
 bool dw_remainder_ok(const Handle* h) {
   const int d_out = h->desc.d_out;
-  return h->tune_tile_m != 2 && ((d_out % (2 * BM)) == 0 || (d_out % (2 * BM)) > BM);
+  return h->tune_dw_tile_m != 2 && ((d_out % (2 * BM)) == 0 || (d_out % (2 * BM)) > BM);
 }
 }  // namespace
 
@@ -1123,7 +1180,7 @@ void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spar
   const int kb_w = (cnt_hint + BK - 1) / BK;
   const int key[PLAN_KEY_INTS] = {(dense ? 1 : 0) | (row_norms_out ? 2 : 0), (int)g.row_tiles128, kb_w, spare_sms,
                                   h->tune_dx_tile_n, h->tune_dw_tile_n, h->tune_dx_split_k, h->tune_dw_split_k,
-                                  h->tune_tile_m};
+                                  h->tune_dx_tile_m + 4 * h->tune_dw_tile_m};
   bool hit = h->plan_valid;
   for (int i = 0; i < PLAN_KEY_INTS && hit; ++i) hit = h->plan_key[i] == key[i];
   if (!hit) {
@@ -1136,14 +1193,22 @@ void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spar
     const bool rem_w = dw_remainder_ok(h);
     const int nw = enumerate_plans((d.d_out + BM - 1) / BM, (d.d_out + 2 * BM - 1) / (2 * BM), d.d_in, kb_w, h->num_sms,
                                    h->max_units, h->tune_dw_tile_n, h->tune_dw_split_k, rem_w, cw);
-    // a sampled dW product becomes ready about this much later than the dX product (sampling and pack
-    // against the SampleA-only kernel: 20.7 against 10.2 us after the call's start on the benchmark
-    // layer); the dense products start together
-    const double offset = dense ? 0.0 : 10.5;
+    // A sampled dW product becomes ready later than the dX product by the time of the kernels in front of it
+    // on the side stream (fitted to their ncu durations on three layer shapes): the norms of the kept rows of X
+    // (HBM-bound), SampleW's single-CTA fixed point over the rows of kept data, and the emit + pack pass, which
+    // moves the kept rows of both operands twice.  The dense products start together.
+    double offset = 0.0;
+    if (!dense) {
+      const double rows_a = (double)rho_hint * d.N * d.T;
+      const double scores_us = 4.0 + rows_a * d.d_in * 2.0 / 3.5e6;
+      const double sample_w_us = 6.0 + rows_a * 0.0013;
+      const double pack_us = 6.0 + 2.0 * (double)cnt_hint * (d.d_in + d.d_out) * 2.0 / 3.0e6;
+      offset = scores_us + sample_w_us + pack_us;
+    }
     Plan px, pw;
     best_pair(cx, nx, ctas, cw, nw, h->num_sms, h->num_sms, offset, &px, &pw);
-    h->plan_dx = apply_tile_m(h, px, g.rem_ok && !row_norms_out);
-    h->plan_dw = apply_tile_m(h, pw, rem_w);
+    h->plan_dx = apply_tile_m(h->tune_dx_tile_m, px, g.rem_ok && !row_norms_out);
+    h->plan_dw = apply_tile_m(h->tune_dw_tile_m, pw, rem_w);
     for (int i = 0; i < PLAN_KEY_INTS; ++i) h->plan_key[i] = key[i];
     h->plan_valid = true;
   }
@@ -1193,7 +1258,7 @@ cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense,
     const bool rn = a_out != nullptr;
     const int n = enumerate_plans(g.row_tiles128, g.row_tiles256, d.d_in, g.kblocks, ctas, h->max_units,
                                   rn ? 256 : h->tune_dx_tile_n, rn ? 1 : h->tune_dx_split_k, g.rem_ok && !rn, cands);
-    plan = apply_tile_m(h, best_alone(cands, n), g.rem_ok && !rn);
+    plan = apply_tile_m(h->tune_dx_tile_m, best_alone(cands, n), g.rem_ok && !rn);
   }
   P.split_k = plan.split;
   // upper bound of work items: every datum kept and split, or every datum a zero tile
@@ -1235,7 +1300,7 @@ cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, in
     Cand cands[MAX_CANDS];
     const int n = enumerate_plans(mtiles, mtiles2, d.d_in, (cnt_hint + BK - 1) / BK, h->num_sms, h->max_units,
                                   h->tune_dw_tile_n, h->tune_dw_split_k, rem_ok, cands);
-    plan = apply_tile_m(h, best_alone(cands, n), rem_ok);
+    plan = apply_tile_m(h->tune_dw_tile_m, best_alone(cands, n), rem_ok);
   }
   P.split_k = plan.split;
   const long max_items = (plan.mh >= 2 ? mtiles2 : mtiles) * ((d.d_in + plan.bn - 1) / plan.bn) * plan.split;
