@@ -6,11 +6,11 @@
 // shared memory -> global), warp 4 issues TMA loads into a ring of shared-memory stages, warp 5
 // issues tcgen05.mma into TMEM accumulators (two of 128 rows, so that the epilogue of a tile overlaps
 // the main loop of the next one, or one of 256 rows).  bf16 operands, fp32 accumulation.  Outputs leave
-// through 128-byte-swizzled shared-memory staging and TMA / bulk stores.  Two instances per tile
-// shape: the unsliced one draws its tiles from a device-wide counter; the sliced one cuts each
-// contraction into slices worked on by neighbouring CTAs and adds the slices in a fixed order.
-// Every wait (mbarrier or sibling CTA) is bounded: when it runs out the CTA records
-// VCAS_ERR_TIMEOUT in the status word and leaves.
+// through 128-byte-swizzled shared-memory staging and TMA / bulk stores.  Three instances per tile
+// shape: two unsliced ones (tiles in CTA order, or drawn from a device-wide counter); the sliced one cuts
+// each contraction into slices, stores every slice's fp32 partial tile, and a reduction launch that follows
+// it adds the slices in a fixed order on all SMs.  No CTA waits for another CTA.  Every wait on an mbarrier
+// is bounded: when it runs out the CTA records VCAS_ERR_TIMEOUT in the status word and leaves.
 #include <cuda.h>
 
 #include <atomic>
@@ -260,19 +260,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 //
 // Work decomposition (all derived on the device from the kept counts): `gemm_tiles` output
 // tiles, each cut along the contraction into S slices of kb_per k-blocks -> units; a unit is
-// (tile, slice).  With S > 1 every unit stores its fp32 partial tile to the workspace and takes a
-// ticket on its tile; the unit that takes the last of the S tickets adds the S partials of the
-// share of the tile's rows in slice order (a fixed order: results do not depend on timing) and
-// writes that share of the output.
+// (tile, slice).  In the sliced instance every unit stores its fp32 partial tile to the workspace;
+// slice_reduce_kernel, launched behind the product, adds the S partials of every tile in slice order
+// (a fixed order: results do not depend on timing) and writes the output.
 constexpr int MODE_DX = 0, MODE_DW = 1;
 constexpr int KIND_SLICED = 0, KIND_STATIC = 1, KIND_DYNAMIC = 2;
 
 struct GemmParams {
   int32_t* status;
   float* partial;          // [max_units][128 * BN] fp32 partial tiles (split contraction)
-  int32_t* tickets;        // [2 * max_units]: slices stored / slices finished per tile; zero between launches
   int32_t* sched;          // [2]: next work item, CTAs that have finished (unsliced instance); zero between launches
   int split_k;             // slices requested by the host
+  int grid_ctas;           // CTAs of the product launch (the slicing is derived from it, also by the reduction launch)
   int max_units;
   unsigned long long wait_limit_ns;   // every mbarrier wait gives up after this long
   int stall_once;          // test hook: CTA 0 leaves out the loads of its first k-block, so that a wait runs out
@@ -346,7 +345,7 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
     } else {
       d.gemm_tiles = 2 * tail256;
       d.zero_tiles = 0;                      // part 1 writes them
-      split_req = d.gemm_tiles > 0 ? (int)gridDim.x / d.gemm_tiles : 1;
+      split_req = d.gemm_tiles > 0 ? P.grid_ctas / d.gemm_tiles : 1;
       if (split_req > 8) split_req = 8;
       if (split_req > d.kblocks / 4) split_req = d.kblocks / 4;      // slices of at least four k-blocks
     }
@@ -354,12 +353,12 @@ __device__ __forceinline__ Decomp decompose(const GemmParams& P) {
   int S = (split_req < 1 || MH == 2 || LEAN) ? 1 : split_req;
   if (S > d.kblocks) S = d.kblocks > 0 ? d.kblocks : 1;
   if (d.gemm_tiles > 0 && (long)d.gemm_tiles * S > P.max_units) S = P.max_units / d.gemm_tiles;
-  if (S > (int)gridDim.x) S = (int)gridDim.x;
+  if (S > P.grid_ctas) S = P.grid_ctas;
   if (S < 1) S = 1;
   d.kb_per = d.kblocks > 0 ? (d.kblocks + S - 1) / S : 0;
   d.S = d.kb_per > 0 ? (d.kblocks + d.kb_per - 1) / d.kb_per : 1;   // every slice non-empty
   d.units = d.gemm_tiles * d.S;
-  d.upi = ((int)gridDim.x / d.S) * d.S;
+  d.upi = (P.grid_ctas / d.S) * d.S;
   return d;
 }
 
@@ -386,7 +385,6 @@ __device__ __forceinline__ void tile_coords(const GemmParams& P, const Decomp& D
   }
 }
 
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // KIND: three instances per tile shape.  KIND_STATIC and KIND_DYNAMIC are for unsliced contractions (S = 1)
 // and carry no code of the slice exchange; the static one takes work items blockIdx.x, + gridDim.x, ...,
@@ -568,31 +566,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         col0 = nt * BN;
       }
     };
-    // finishes 8 consecutive columns of one output row: rescale, optional GELU', convert, store
-    auto store8 = [&](size_t off, float sc, const float* f) {
-      if (MODE == MODE_DX) {
-        float r[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) r[e] = sc * f[e];
-        if (P.H != nullptr) {
-          const uint4 hv = *reinterpret_cast<const uint4*>(P.H + off);
-          const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            r[2 * e] *= gelu_prime(__uint_as_float(hu[e] << 16));
-            r[2 * e + 1] *= gelu_prime(__uint_as_float(hu[e] & 0xffff0000u));
-          }
-        }
-        uint4 o;
-        o.x = pack_bf16(r[0], r[1]); o.y = pack_bf16(r[2], r[3]);
-        o.z = pack_bf16(r[4], r[5]); o.w = pack_bf16(r[6], r[7]);
-        *reinterpret_cast<uint4*>(P.dX + off) = o;
-      } else {
-        *reinterpret_cast<float4*>(P.dW + off) = make_float4(f[0], f[1], f[2], f[3]);
-        *reinterpret_cast<float4*>(P.dW + off + 4) = make_float4(f[4], f[5], f[6], f[7]);
-      }
-    };
-
     const uint32_t swz = (uint32_t)(lane & 7);                   // 128-byte swizzle: 16-byte slot ^= row & 7
     int lt = 0;
     bool ok = true;
@@ -649,7 +622,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
       if (LEAN && u >= D.units) { zero_tile(u - D.units); continue; }
       const int lt_now = lt++;
-      const int tile = u / D.S, slice = u % D.S;
+      const int tile = u / D.S;
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(tile, true, row0, rows_valid, col0, sc, n_out, t_out);
       const int buf = lt_now % NACC; const uint32_t use = (uint32_t)(lt_now / NACC) & 1u;
@@ -668,52 +641,6 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (!got) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * BN);
-      // Adds the slices of this unit's share of the tile's rows in slice order and writes that share of the
-      // output.  A partial tile is laid out [32-column chunk][row][32 floats] with the eight 16-byte slots of
-      // a row swizzled by (row & 7); load4(slice, float offset) fetches one slot of one slice.
-      auto reduce_tile = [&](auto load4) {
-        const int r_begin = 0;
-        const int r_end = min(BM, rows_valid);
-        const int c8n = min(BN, P.d_in - col0) / 8;               // 8-column groups per row inside the tensor
-        const int n_items = max(0, r_end - r_begin) * c8n;
-        auto slot_off = [&](int r, int c8, int half) {
-          const int slot = ((c8 & 3) * 2 + half) ^ (r & 7);
-          return (size_t)(c8 >> 2) * (BM * 32) + (size_t)r * 32 + (size_t)slot * 4;
-        };
-        for (int it0 = tid; it0 < n_items; it0 += 256) {
-          // two items per thread in flight
-          const int it1 = it0 + 128;
-          const bool has1 = it1 < n_items;
-          const int ra = r_begin + it0 / c8n, ca = it0 % c8n;
-          const int rb = has1 ? r_begin + it1 / c8n : ra, cb = has1 ? it1 % c8n : ca;
-          const size_t oa0 = slot_off(ra, ca, 0), oa1 = slot_off(ra, ca, 1);
-          const size_t ob0 = slot_off(rb, cb, 0), ob1 = slot_off(rb, cb, 1);
-          float fa[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          float fb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          for (int sl0 = 0; sl0 < D.S; sl0 += 4) {           // slices in order, four at a time in flight
-            float4 x[4][4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int sl = min(sl0 + q, D.S - 1);
-              x[q][0] = load4(sl, oa0);
-              x[q][1] = load4(sl, oa1);
-              x[q][2] = load4(sl, ob0);
-              x[q][3] = load4(sl, ob1);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              if (sl0 + q < D.S) {
-                fa[0] += x[q][0].x; fa[1] += x[q][0].y; fa[2] += x[q][0].z; fa[3] += x[q][0].w;
-                fa[4] += x[q][1].x; fa[5] += x[q][1].y; fa[6] += x[q][1].z; fa[7] += x[q][1].w;
-                fb[0] += x[q][2].x; fb[1] += x[q][2].y; fb[2] += x[q][2].z; fb[3] += x[q][2].w;
-                fb[4] += x[q][3].x; fb[5] += x[q][3].y; fb[6] += x[q][3].z; fb[7] += x[q][3].w;
-              }
-            }
-          }
-          store8((row0 + ra) * ld + col0 + ca * 8, sc, fa);
-          if (has1) store8((row0 + rb) * ld + col0 + cb * 8, sc, fb);
-        }
-      };
       if constexpr (LEAN) {
         // ---- whole contraction in this unit: accumulator -> (rescale, GELU', convert) -> swizzled
         // shared memory -> TMA store of 32 rows x 128 bytes per warp (rows / columns outside the
@@ -844,29 +771,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
       tc_fence_before();
       mbar_arrive(&s.tmem_empty[buf]);          // the accumulator is free again
-      if (lane == 0) bulk_wait_all();           // this warp's part of the partial tile is in global memory
-      __syncwarp();
-      // ... announce it.  The unit that finds the other S - 1 slices of its tile already announced adds the S
-      // partial tiles in slice order (a fixed order: results do not depend on which unit comes last) and writes
-      // the output; the others are done.  No unit waits for another one, so the S units of a tile need not be
-      // resident at the same time.
-      __threadfence();
-      epi_bar();
-      if (tid == 0) {
-        const int arrived = atomicAdd(&P.tickets[tile], 1);
-        const int last = arrived == D.S - 1 ? 1 : 0;
-        if (last) P.tickets[tile] = 0;            // all S have arrived: re-armed for the next launch
-        *s.flag = last;
-      }
-      epi_bar();
-      if (*(volatile int*)s.flag != 0) {
-        __threadfence();
-        const float* tile_part = P.partial + (size_t)(tile * D.S) * (BM * BN);
-        reduce_tile([&](int sl, size_t off) {
-          return __ldcg(reinterpret_cast<const float4*>(tile_part + (size_t)sl * (BM * BN) + off));
-        });
-      }
-      epi_bar();                                  // s.flag is rewritten by the next unit
+      if (lane == 0) bulk_wait_all();           // this warp's part of the partial tile is in global memory;
+      __syncwarp();                             // the launch that follows adds the slices (slice_reduce_kernel)
       }  // !LEAN
     }
     // sliced instance: zero tiles are taken from the far end of the grid first, where CTAs have no product units
@@ -879,6 +785,90 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (warp == 5) { tc_fence_after(); tmem_dealloc(tmem_base, TMEM_COLS); }
+}
+
+// Adds the S partial tiles of every product tile of a sliced launch in slice order and writes the output
+// (dX: rescaled by 1/p_n, optional GELU', rounded to bf16; dW: fp32).  Launched behind the product kernel as a
+// programmatic dependent; it derives the same tiles and slices from the device-resident counts.  One thread per
+// 8 consecutive columns of one output row: it reads two 16-byte slots of every slice (through L2, where the
+// product has just put them) and stores 16 or 32 bytes, so consecutive threads write consecutive bytes.  A partial
+// tile is laid out [32-column chunk][row][32 floats] with the eight 16-byte slots of a row swizzled by (row & 7),
+// as the product's epilogue staged it.
+constexpr int REDUCE_THREADS = 256;
+template <int MODE, int BN>
+__global__ void __launch_bounds__(REDUCE_THREADS) slice_reduce_kernel(GemmParams P) {
+  pdl_wait();      // the partial tiles come from the product kernel before this one
+  pdl_trigger();
+  const Decomp D = decompose<MODE, BN, 1, false>(P);
+  if (D.gemm_tiles <= 0) return;
+  constexpr int C8 = BN / 8;                       // 8-column groups per tile row
+  constexpr int PER_TILE = BM * C8;
+  const long total = (long)D.gemm_tiles * PER_TILE;
+  const size_t ld = (size_t)P.d_in;
+  for (long it = (long)blockIdx.x * REDUCE_THREADS + threadIdx.x; it < total; it += (long)gridDim.x * REDUCE_THREADS) {
+    const int tile = (int)(it / PER_TILE);
+    const int rem = (int)(it - (long)tile * PER_TILE);
+    const int r = rem / C8, c8 = rem - r * C8;
+    int k, c0, c1;
+    tile_coords<MODE>(P, D, tile, k, c0, c1);
+    size_t row0;
+    int rows_valid;
+    float sc = 1.0f;
+    if (MODE == MODE_DX) {
+      const int n = P.dense ? k : P.idxA[k];
+      row0 = (size_t)n * P.T + (size_t)c0 * BM;
+      rows_valid = min(BM, P.T - c0 * BM);
+      if (!P.dense) sc = P.scaleA[n];
+    } else {
+      row0 = (size_t)c0 * BM;
+      rows_valid = min(BM, P.d_out - c0 * BM);
+    }
+    const int col = c1 * BN + c8 * 8;
+    if (r >= rows_valid || col >= P.d_in) continue;
+    const float* tile_part = P.partial + (size_t)tile * D.S * (BM * BN);
+    const size_t chunk = (size_t)(c8 >> 2) * (BM * 32) + (size_t)r * 32;
+    const size_t o0 = chunk + (size_t)((((c8 & 3) * 2 + 0) ^ (r & 7)) * 4);
+    const size_t o1 = chunk + (size_t)((((c8 & 3) * 2 + 1) ^ (r & 7)) * 4);
+    float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int sl0 = 0; sl0 < D.S; sl0 += 4) {         // slices in order, four at a time in flight
+      float4 x[4][2];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float* src = tile_part + (size_t)min(sl0 + q, D.S - 1) * (BM * BN);
+        x[q][0] = __ldcg(reinterpret_cast<const float4*>(src + o0));
+        x[q][1] = __ldcg(reinterpret_cast<const float4*>(src + o1));
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (sl0 + q < D.S) {
+          f[0] += x[q][0].x; f[1] += x[q][0].y; f[2] += x[q][0].z; f[3] += x[q][0].w;
+          f[4] += x[q][1].x; f[5] += x[q][1].y; f[6] += x[q][1].z; f[7] += x[q][1].w;
+        }
+      }
+    }
+    const size_t off = (row0 + r) * ld + col;
+    if (MODE == MODE_DX) {
+      float v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = sc * f[e];
+      if (P.H != nullptr) {
+        const uint4 hv = __ldg(reinterpret_cast<const uint4*>(P.H + off));
+        const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          v[2 * e] *= gelu_prime(__uint_as_float(hu[e] << 16));
+          v[2 * e + 1] *= gelu_prime(__uint_as_float(hu[e] & 0xffff0000u));
+        }
+      }
+      uint4 o;
+      o.x = pack_bf16(v[0], v[1]); o.y = pack_bf16(v[2], v[3]);
+      o.z = pack_bf16(v[4], v[5]); o.w = pack_bf16(v[6], v[7]);
+      *reinterpret_cast<uint4*>(P.dX + off) = o;
+    } else {
+      *reinterpret_cast<float4*>(P.dW + off) = make_float4(f[0], f[1], f[2], f[3]);
+      *reinterpret_cast<float4*>(P.dW + off + 4) = make_float4(f[4], f[5], f[6], f[7]);
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------ host side
@@ -917,11 +907,10 @@ bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, 
 // on five layer shapes on B200: a k-block costs about 0.50 / 0.45 / 0.43 us for 256 / 128 / 64 wide
 // 128-row tiles (the shared-memory fill rate of one SM bounds it, so narrow tiles only pay off when
 // they fill more SMs); a unit costs about 4 us of set-up, pipeline fill and output store; a sliced unit
-// pays for its partial store and the unit that comes last adds the S partial tiles of the whole tile
-// through L2: about 20 us + 1.5 us per slice on the critical path, so that slicing only pays for long
-// contractions with few tiles; a 256 x 256 tile (mh = 2) costs about 0.66 us per k-block for twice the
-// work, and 7 us per tile.
-constexpr double SLICED_US = 20.0, SLICED_PER_SLICE_US = 1.5;
+// stores its partial tile instead, and the reduction launch that follows adds the slices on all SMs:
+// together about 11 us + 1 us per slice; a 256 x 256 tile (mh = 2) costs about 0.66 us per k-block for
+// twice the work, and 7 us per tile.
+constexpr double SLICED_US = 11.0, SLICED_PER_SLICE_US = 1.0;
 struct Cand {
   Plan plan;
   long units;      // (tile, slice) units
@@ -1080,6 +1069,7 @@ cudaError_t run_gemm_k(Handle* h, const CUtensorMap& a, const CUtensorMap& b, co
     attr_set[h->device].store(true, std::memory_order_release);
   }
   GemmParams P = P0;
+  P.grid_ctas = (int)(max_items < ctas ? max_items : ctas);
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
   cfg.blockDim = dim3(NUM_THREADS);
@@ -1096,7 +1086,20 @@ cudaError_t run_gemm_k(Handle* h, const CUtensorMap& a, const CUtensorMap& b, co
   cfg.gridDim = dim3((unsigned)grid);
   cudaError_t e = cudaLaunchKernelEx(&cfg, umma_kernel<MODE, BN, MH, KIND>, a, b, c, P);
   h->launches += 1;
-  return e != cudaSuccess ? e : cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if constexpr (KIND == KIND_SLICED) {
+    // the slices are added by a launch of their own on all SMs: one thread per 8 columns of an output row of the
+    // most tiles the product can have (the kernel strides over what the device-resident counts leave)
+    const long max_tiles = P.split_k > 0 ? max_items / P.split_k : max_items;
+    long blocks = (max_tiles * BM * (BN / 8) + REDUCE_THREADS - 1) / REDUCE_THREADS;
+    const long cap = (long)h->num_sms * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    e = launch_after(slice_reduce_kernel<MODE, BN>, dim3((unsigned)blocks), dim3(REDUCE_THREADS), 0, st, P);
+    h->launches += 1;
+    if (e != cudaSuccess) return e;
+  }
+  return cudaGetLastError();
 }
 
 template <int MODE, int BN, int MH>
@@ -1141,7 +1144,6 @@ void common_params(Handle* h, GemmParams& P, int which) {
   P = GemmParams();
   P.status = h->ws.status;
   P.partial = h->ws.partial_tiles + (size_t)which * h->max_units * (BM * 256);
-  P.tickets = h->ws.tickets + (size_t)which * 2 * h->max_units;
   P.sched = h->ws.sched + which * 2;
   P.max_units = h->max_units;
   P.wait_limit_ns = h->wait_limit_ns;

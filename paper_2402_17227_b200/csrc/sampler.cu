@@ -372,18 +372,32 @@ __global__ void __launch_bounds__(SAMPLER_THREADS) sample_w_kernel(SampleWParams
     __syncthreads();
   }
 
-  // kept rows per chunk of 32 compact rows: chunk_off[ch] = count for now
+  // kept rows per chunk of 32 compact rows: chunk_off[ch] = count for now.  A warp takes four chunks at a time
+  // and issues their loads together (one memory latency per four chunks instead of one per chunk).
   const int nchunks = (n + 31) >> 5;
-  for (int ch = warp; ch < nchunks; ch += SAMPLER_THREADS / 32) {
-    const int i = (ch << 5) + lane;
-    bool keep = false;
-    if (i < n) {
-      const int k = i / T;
-      const float q = q_of(mode, c, w[i], P.q_in, P.q_in != nullptr ? P.idxA[k] * T + (i - k * T) : 0);
-      keep = row_kept(P.sample_w, q, P.sample_w ? P.uc[i] : 0u);
+  for (int ch0 = warp; ch0 < nchunks; ch0 += 4 * (SAMPLER_THREADS / 32)) {
+    float wv[4];
+    uint32_t uv[4];
+#pragma unroll
+    for (int k4 = 0; k4 < 4; ++k4) {
+      const int i = ((ch0 + k4 * (SAMPLER_THREADS / 32)) << 5) + lane;
+      wv[k4] = i < n ? w[i] : 0.f;
+      uv[k4] = (i < n && P.sample_w) ? __ldg(P.uc + i) : 0u;
     }
-    const unsigned b = __ballot_sync(0xffffffffu, keep);
-    if (lane == 0) P.chunk_off[ch] = __popc(b);
+#pragma unroll
+    for (int k4 = 0; k4 < 4; ++k4) {
+      const int ch = ch0 + k4 * (SAMPLER_THREADS / 32);
+      if (ch >= nchunks) break;                    // warp-uniform
+      const int i = (ch << 5) + lane;
+      bool keep = false;
+      if (i < n) {
+        const int k = i / T;
+        const float q = q_of(mode, c, wv[k4], P.q_in, P.q_in != nullptr ? P.idxA[k] * T + (i - k * T) : 0);
+        keep = row_kept(P.sample_w, q, uv[k4]);
+      }
+      const unsigned b = __ballot_sync(0xffffffffu, keep);
+      if (lane == 0) P.chunk_off[ch] = __popc(b);
+    }
   }
   __syncthreads();
   // exclusive prefix sums over the chunk counts: every thread owns a contiguous segment
@@ -488,39 +502,37 @@ __global__ void __launch_bounds__(EMIT_THREADS) emit_pack_kernel(EmitParams P) {
     }
     if (pack) {
       __syncthreads();
-      // this part's rows j = part, part + parts, ...: their 16-byte pieces of both operands are spread over the
-      // CTA's threads, four independent loads per thread in flight whatever the width of a row
+      // This part's rows j = part, part + parts, ...  A row's 16-byte pieces (first those of dY, then those of X)
+      // are cut into segments of 128; a warp takes (row, segment) items in turn and moves a segment with four
+      // independent loads per lane in flight.  One integer division per 2 KB moved, none per piece.
       const int m = s_cnt;
       const int mp = m > part ? (m - part + parts - 1) / parts : 0;
       const int vo = P.d_out / 8, vt = vo + P.d_in / 8;
-      const int total = mp * vt;
-      for (int it0 = tid; it0 < total; it0 += 4 * EMIT_THREADS) {
+      const int nseg = (vt + 127) >> 7;
+      for (int item = warp; item < mp * nseg; item += EMIT_THREADS / 32) {
+        const int jj = item / nseg, seg = item - jj * nseg;
+        const int j = part + jj * parts;
+        const size_t r = (size_t)s_r[j], pos = (size_t)s_pos[j];
+        const float sc = s_sc[j];
+        const uint4* srcG = reinterpret_cast<const uint4*>(P.dY + r * P.d_out);
+        const uint4* srcX = reinterpret_cast<const uint4*>(P.X + r * P.d_in) - vo;
+        uint4* dstG = reinterpret_cast<uint4*>(P.packG + pos * P.d_out);
+        uint4* dstX = reinterpret_cast<uint4*>(P.packX + pos * P.d_in) - vo;
+        const int p0 = (seg << 7) + lane;
         uint4 v[4];
-        uint4* dst[4];
-        float scl[4];
-        bool isg[4];
 #pragma unroll
-        for (int u4 = 0; u4 < 4; ++u4) {
-          const int it = it0 + u4 * EMIT_THREADS;
-          dst[u4] = nullptr;
-          if (it < total) {
-            const int jj = it / vt, piece = it - jj * vt;
-            const int j = part + jj * parts;
-            const size_t r = (size_t)s_r[j], pos = (size_t)s_pos[j];
-            isg[u4] = piece < vo;
-            scl[u4] = s_sc[j];
-            if (isg[u4]) {
-              v[u4] = __ldg(reinterpret_cast<const uint4*>(P.dY + r * P.d_out) + piece);
-              dst[u4] = reinterpret_cast<uint4*>(P.packG + pos * P.d_out) + piece;
-            } else {
-              v[u4] = __ldg(reinterpret_cast<const uint4*>(P.X + r * P.d_in) + (piece - vo));
-              dst[u4] = reinterpret_cast<uint4*>(P.packX + pos * P.d_in) + (piece - vo);
-            }
-          }
+        for (int q = 0; q < 4; ++q) {
+          const int piece = p0 + 32 * q;
+          if (piece < vt) v[q] = __ldg(piece < vo ? srcG + piece : srcX + piece);
         }
 #pragma unroll
-        for (int u4 = 0; u4 < 4; ++u4)
-          if (dst[u4] != nullptr) *dst[u4] = isg[u4] ? scale8(v[u4], scl[u4]) : v[u4];
+        for (int q = 0; q < 4; ++q) {
+          const int piece = p0 + 32 * q;
+          if (piece < vt) {
+            if (piece < vo) dstG[piece] = scale8(v[q], sc);
+            else dstX[piece] = v[q];
+          }
+        }
       }
       __syncthreads();
     }
