@@ -208,6 +208,7 @@ int vcas_create(vcas_handle* out, const vcas_layer_desc* desc, const vcas_config
   h->tune_dx_tile_n = h->tune_dw_tile_n = h->tune_dx_split_k = h->tune_dw_split_k = 0;
   h->tune_dx_tile_m = h->tune_dw_tile_m = 0;
   h->plan_valid = false;
+  h->plan_cache_used = h->plan_cache_next = 0;
   h->wait_limit_ns = 2000000000ull;
   h->sub_k = 0;
   h->join_pending = false;

@@ -54,6 +54,7 @@ constexpr int PARTIAL_SLOTS = 4096;
 // (mh: 1 = 128-row tiles, 2 = 256-row tiles, 3 = 256-row tiles for whole waves + 128-row tiles for the rest).
 struct Plan { int bn, split, mh; };
 constexpr int PLAN_KEY_INTS = 9;
+constexpr int PLAN_CACHE = 64;
 
 struct Handle {
   vcas_layer_desc desc;
@@ -86,6 +87,11 @@ struct Handle {
   bool plan_valid;
   int plan_key[PLAN_KEY_INTS];
   Plan plan_dx, plan_dw;
+  // ... and the pairs made before it (a handle shared by the layers of a stack sees a few dozen different
+  // expected counts in turn): a small table replaced in round-robin order
+  int plan_cache_key[PLAN_CACHE][PLAN_KEY_INTS];
+  Plan plan_cache_dx[PLAN_CACHE], plan_cache_dw[PLAN_CACHE];
+  int plan_cache_used, plan_cache_next;
   // the probe's sample of the parameters (App. D): sub_k rows of the parameter gradient (0: all of them)
   int sub_k;
   int32_t* sub_rows;   // [SUB_MAX] device, ascending

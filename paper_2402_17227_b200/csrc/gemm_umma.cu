@@ -935,6 +935,7 @@ int enumerate_plans(long row_tiles128, long row_tiles256, int n_extent, int kblo
     const long tiles = row_tiles128 * ntiles;
     for (int sp = 1; sp <= 16; ++sp) {
       if (force_split != 0 && sp != force_split) continue;
+      if (force_split == 0 && sp > 4 && (sp & 1) != 0) continue;       // 1, 2, 3, 4, 6, 8, ... 16
       if (sp > 1 && tiles * sp > max_units) continue;
       if (sp > 1 && force_split == 0 && kblocks / sp < 4) continue;   // slices too short to pay off
       const long units = tiles * sp;
@@ -1186,6 +1187,19 @@ void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spar
   bool hit = h->plan_valid;
   for (int i = 0; i < PLAN_KEY_INTS && hit; ++i) hit = h->plan_key[i] == key[i];
   if (!hit) {
+    for (int e = 0; e < h->plan_cache_used && !hit; ++e) {
+      bool same = true;
+      for (int i = 0; i < PLAN_KEY_INTS && same; ++i) same = h->plan_cache_key[e][i] == key[i];
+      if (same) {
+        h->plan_dx = h->plan_cache_dx[e];
+        h->plan_dw = h->plan_cache_dw[e];
+        for (int i = 0; i < PLAN_KEY_INTS; ++i) h->plan_key[i] = key[i];
+        h->plan_valid = true;
+        hit = true;
+      }
+    }
+  }
+  if (!hit) {
     const int ctas = h->num_sms - spare_sms > 1 ? h->num_sms - spare_sms : 1;
     Cand cx[MAX_CANDS], cw[MAX_CANDS];
     // the epilogue emits row square-norms of dX only from unsliced 256-wide tiles (one partial sum per tile)
@@ -1213,6 +1227,12 @@ void plan_products(Handle* h, bool dense, float rho_hint, int cnt_hint, int spar
     h->plan_dw = apply_tile_m(h->tune_dw_tile_m, pw, rem_w);
     for (int i = 0; i < PLAN_KEY_INTS; ++i) h->plan_key[i] = key[i];
     h->plan_valid = true;
+    const int e = h->plan_cache_next;
+    for (int i = 0; i < PLAN_KEY_INTS; ++i) h->plan_cache_key[e][i] = key[i];
+    h->plan_cache_dx[e] = h->plan_dx;
+    h->plan_cache_dw[e] = h->plan_dw;
+    h->plan_cache_next = (e + 1) % PLAN_CACHE;
+    if (h->plan_cache_used < PLAN_CACHE) h->plan_cache_used += 1;
   }
   *dx = h->plan_dx;
   *dw = h->plan_dw;
