@@ -356,7 +356,7 @@ cudaError_t launch_fma_dw(Handle* h, const void* dY, const void* X, const int32_
 cudaError_t launch_umma_dx(Handle* h, const void* dY, const void* W, bool dense, float rho_hint,
                            const void* H, void* dX, float* a_out, bool skip_dropped, int spare_sms,
                            const Plan* pair_plan, cudaStream_t st);
-inline int a_out_parts(int d_in) { return (d_in + 255) / 256; }
+inline int a_out_parts(int d_in) { return 2 * ((d_in + 255) / 256); }    // one per 256-column tile and epilogue group
 // dW = A_rows^T B_rows over the first *cnt rows (A_rows [rows, d_out], B_rows [rows, d_in], bf16)
 // cnt_hint: the expected *cnt, used on the host to pick the tiling
 cudaError_t launch_umma_dw(Handle* h, const void* A_rows, const void* B_rows, int rows_capacity,

@@ -2,8 +2,9 @@
 //   dX[rows of kept data] = (1/p_n) dY[rows] W          (App. E; rows of dropped data are zero-filled)
 //   dW = A_rows^T B_rows over the compacted kept rows    (Sec. 4.2: G_tilde^T X)
 // One persistent CTA per SM works through tiles whose number depends on the kept counts, which
-// are read from device memory.  Per CTA: warps 0-3 are the epilogue (TMEM -> registers ->
-// shared memory -> global), warp 4 issues TMA loads into a ring of shared-memory stages, warp 5
+// are read from device memory.  Per CTA: warps 0-3 and 6-9 are the epilogue (TMEM -> registers ->
+// shared memory -> global; the two warps that reach the same TMEM lanes split a tile's columns), warp 4
+// issues TMA loads into a ring of shared-memory stages, warp 5
 // issues tcgen05.mma into TMEM accumulators (two of 128 rows, so that the epilogue of a tile overlaps
 // the main loop of the next one, or one of 256 rows).  bf16 operands, fp32 accumulation.  Outputs leave
 // through 128-byte-swizzled shared-memory staging and TMA / bulk stores.  Three instances per tile
@@ -25,10 +26,14 @@ constexpr int BK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN chunk of an MN-major operand
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;          // 8 epilogue warps, 1 TMA producer warp, 1 MMA warp
+constexpr int EPI_THREADS = 256;          // two groups of four epilogue warps
+// Register cap of the product kernels: a CTA of 320 threads must leave room on its SM for the CTAs of the
+// scoring and packing kernels of the call's other branch, which run beside it.
+constexpr int MAX_REGS = 128;
 constexpr int TMEM_COLS = 512;
 constexpr int EPI_WARP_BYTES = 32 * 128;                // one staging buffer: 32 rows of 128 bytes, 128B-swizzled
-constexpr int EPI_BYTES = 4 * 2 * EPI_WARP_BYTES;       // two buffers for each of the four epilogue warps
+constexpr int EPI_BYTES = 8 * EPI_WARP_BYTES;           // one buffer for each of the eight epilogue warps
 
 // MH = number of 128-row halves of a tile (1 or 2).  A 256-row tile reuses each B stage for two
 // accumulators, which cuts the shared-memory fill per FLOP by a third (the fill rate of one SM is
@@ -114,8 +119,6 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void*
                ::"l"(map), "r"(smem_u32(ssrc)), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// at most one group of this thread may still be READING its shared-memory source
-__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // all groups of this thread are complete (their global writes are performed)
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -221,9 +224,9 @@ __device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid
   using C = TileCfg<BN, MH>;
   if (tid == 0) {
     for (int i = 0; i < C::STAGES; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&s.tmem_full[i], 1); mbar_init(&s.tmem_empty[i], 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&s.tmem_full[i], 1); mbar_init(&s.tmem_empty[i], EPI_THREADS); }
     if (with_queue)
-      for (int i = 0; i < QD; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 129); }
+      for (int i = 0; i < QD; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], EPI_THREADS + 1); }
     *s.abort_flag = 0;
     *reinterpret_cast<unsigned long long*>(s.abort_flag + 5) = wait_limit_ns;   // read by mbar_wait
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -236,19 +239,80 @@ __device__ __forceinline__ uint32_t setup(const SmemLayout& s, int warp, int tid
   return *(volatile uint32_t*)s.tmem_holder;
 }
 
-// GELU'(x) = Phi(x) + x phi(x) (erf form).  Both terms share E = exp(-x^2 / 2): phi = E / sqrt(2 pi), and
-// erf(|x| / sqrt 2) = 1 - (a1 t + ... + a5 t^5) E with t = 1 / (1 + p |x| / sqrt 2) (Abramowitz & Stegun 7.1.26,
-// absolute error below 1.5e-7, far inside the bf16 rounding of the result).  One exponential and one approximate reciprocal
-// per element: the epilogue has only four warps per SM, so this arithmetic is on the critical path of the tile.
+// GELU'(x) = Phi(x) + x phi(x) (erf form) as a polynomial: GELU'(x) - 1/2 is odd, so GELU'(x) = 1/2 + x Q(x^2);
+// Q is a degree-11 polynomial in t = 2 x^2 / 25 - 1 (a Chebyshev least-squares fit on |x| <= 5, converted to
+// powers of t, whose coefficients stay below 0.15), and |x| is clamped to 5, beyond which GELU' is 0 or 1 to
+// within 1e-5.  Maximum absolute error 3e-5 in fp32 Horner form against the erf form in double precision, far
+// inside the bf16 rounding of the product it scales.  No special-function unit: with an exponential and a
+// reciprocal per element the epilogue of a wide dX tile took longer than its products (the exponential alone
+// cost as much as all other arithmetic); thirteen fused multiply-adds, issued for two elements at a time
+// (fma.rn.f32x2), cost less.
+#define VCAS_GELU_PRIME_COEFFS                                                                   \
+  {1.421275400e-01f, -7.508027066e-02f, 6.700628620e-02f, -7.250861119e-02f, 7.542644430e-02f,  \
+   -7.929997715e-02f, 1.003925139e-01f, -8.373814972e-02f, 1.450312277e-02f, -1.099747622e-02f, \
+   4.948262191e-02f, -2.731859035e-02f}
 __device__ __forceinline__ float gelu_prime(float x) {
-  const float ax = fabsf(x);
-  const float E = __expf(-0.5f * x * x);
-  float t;      // approximate reciprocal (one instruction, no special-case branch; 1 ulp is far below the rest)
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f * 0.70710678118654752f, ax, 1.0f)));
-  const float poly = t * fmaf(t, fmaf(t, fmaf(t, fmaf(t, 1.061405429f, -1.453152027f), 1.421413741f), -0.284496736f), 0.254829592f);
-  const float erf_abs = fmaf(-poly, E, 1.0f);
-  const float Phi = 0.5f * (1.0f + copysignf(erf_abs, x));
-  return fmaf(x, 0.39894228040143268f * E, Phi);
+  constexpr float GP_C[12] = VCAS_GELU_PRIME_COEFFS;
+  const float ax = fminf(fabsf(x), 5.0f);
+  const float t = fmaf(ax * ax, 0.08f, -1.0f);
+  float p = GP_C[11];
+#pragma unroll
+  for (int k = 10; k >= 0; --k) p = fmaf(p, t, GP_C[k]);
+  return fmaf(copysignf(ax, x), p, 0.5f);
+}
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// r[e] *= GELU'(h_e) for the eight bf16 pre-activations in hv: the same polynomial as gelu_prime, the four pairs
+// side by side and every step of Horner's rule issued for all of them before the next (independent chains).
+__device__ __forceinline__ void gelu_prime8(const uint4& hv, float (&r)[8]) {
+  constexpr float GP_C[12] = VCAS_GELU_PRIME_COEFFS;
+  const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
+  float x[8], ax[8];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    x[2 * e] = __uint_as_float(hu[e] << 16);
+    x[2 * e + 1] = __uint_as_float(hu[e] & 0xffff0000u);
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) ax[e] = fminf(fabsf(x[e]), 5.0f);
+  uint64_t t[4], p[4];
+  const uint64_t c08 = pack2(0.08f, 0.08f), cm1 = pack2(-1.0f, -1.0f);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const uint64_t a2 = pack2(ax[2 * e], ax[2 * e + 1]);
+    t[e] = fma2(mul2(a2, a2), c08, cm1);
+    p[e] = pack2(GP_C[11], GP_C[11]);
+  }
+#pragma unroll
+  for (int k = 10; k >= 0; --k) {
+    const uint64_t ck = pack2(GP_C[k], GP_C[k]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) p[e] = fma2(p[e], t[e], ck);
+  }
+  const uint64_t half2 = pack2(0.5f, 0.5f);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const uint64_t xc = pack2(copysignf(ax[2 * e], x[2 * e]), copysignf(ax[2 * e + 1], x[2 * e + 1]));
+    const uint64_t g = fma2(xc, p[e], half2);
+    const uint64_t o = mul2(pack2(r[2 * e], r[2 * e + 1]), g);
+    unpack2(o, r[2 * e], r[2 * e + 1]);
+  }
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -395,7 +459,7 @@ __device__ __forceinline__ void tile_coords(const GemmParams& P, const Decomp& D
 // Separate instances because the product kernels are short: code that a launch never runs still costs it
 // time.
 template <int MODE, int BN, int MH, int KIND>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __maxnreg__(MAX_REGS)
 umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, GemmParams P) {
   using C = TileCfg<BN, MH>;
@@ -536,8 +600,13 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
   } else {
     // -------------------------------------------------------------------- epilogue
-    // thread (warp, lane) owns accumulator lane warp*32 + lane = tile row
-    const int row = warp * 32 + lane;
+    // Two groups of four epilogue warps (warps 0-3 and 6-9).  A warp reaches the 32 TMEM lanes of quarter
+    // (warp % 4), so the two warps of a quarter share its rows and split the tile's column chunks between
+    // them (even chunks / odd chunks): two warps per scheduler hide each other's TMEM, arithmetic and store
+    // latencies, which a single warp per scheduler cannot.
+    const int eq = warp & 3;                  // TMEM lane quarter
+    const int eg = warp < 4 ? 0 : 1;          // epilogue group: which column chunks
+    const int row = eq * 32 + lane;           // this thread's row of a 128-row half
     const size_t ld = (size_t)P.d_in;
     // output rows [row0, row0 + rows_valid) x columns [col0, col0 + BN) of the tile; sc = 1/p_n
     auto geometry = [&](int tile, bool is_gemm, size_t& row0, int& rows_valid, int& col0, float& sc, int& n_out,
@@ -588,7 +657,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // Writes the zero tile z (rows of dropped data; nothing kept at all): every warp clears one of its staging
     // buffers and stores it, by TMA, to each 32-row x 128-byte piece of its slab of the tile.  The tensor map
     // clips rows beyond T and columns beyond d_in.  No per-element work: the epilogue warps are free again at once.
-    uint8_t* stage0 = s.epi + warp * (2 * EPI_WARP_BYTES);       // this warp's two staging buffers
+    uint8_t* stage0 = s.epi + (eg * 4 + eq) * EPI_WARP_BYTES;    // this warp's staging buffer
     auto zero_tile = [&](int z) {
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(z, false, row0, rows_valid, col0, sc, n_out, t_out);
@@ -602,11 +671,11 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (lane == 0) {
 #pragma unroll 1
         for (int hh = 0; hh < MH; ++hh) {
-          if (hh * BM + warp * 32 >= rows_valid) break;
-          for (int j = 0; j < BN / COLS; ++j) {
+          if (hh * BM + eq * 32 >= rows_valid) break;
+          for (int j = eg; j < BN / COLS; j += 2) {
             if (col0 + j * COLS >= P.d_in) break;
-            if (MODE == MODE_DX) tma_store_3d(&tmC, stage0, col0 + j * COLS, t_out + hh * BM + warp * 32, n_out);
-            else tma_store_2d(&tmC, stage0, col0 + j * COLS, (int)row0 + hh * BM + warp * 32);
+            if (MODE == MODE_DX) tma_store_3d(&tmC, stage0, col0 + j * COLS, t_out + hh * BM + eq * 32, n_out);
+            else tma_store_2d(&tmC, stage0, col0 + j * COLS, (int)row0 + hh * BM + eq * 32);
           }
         }
         bulk_commit();
@@ -616,7 +685,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       if (MODE == MODE_DX && P.a_out != nullptr) {
 #pragma unroll 1
         for (int hh = 0; hh < MH; ++hh)
-          if (hh * BM + row < rows_valid) P.a_out[(row0 + hh * BM + row) * P.a_parts + col0 / 256] = 0.f;
+          if (hh * BM + row < rows_valid) P.a_out[(row0 + hh * BM + row) * P.a_parts + (col0 / 256) * 2 + eg] = 0.f;
       }
     };
     for (int u = next_unit(-1); u >= 0 && ok; u = next_unit(u)) {
@@ -626,21 +695,37 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       size_t row0; int rows_valid, col0, n_out, t_out; float sc;
       geometry(tile, true, row0, rows_valid, col0, sc, n_out, t_out);
       const int buf = lt_now % NACC; const uint32_t use = (uint32_t)(lt_now / NACC) & 1u;
+      if constexpr (LEAN && MODE == MODE_DX) {
+        // GELU' epilogue: while the tile's products are still running, ask L2 for the pre-activations of this
+        // thread's rows
+        if (P.H != nullptr) {
+#pragma unroll
+          for (int hh = 0; hh < MH; ++hh) {
+            const int hrow = hh * BM + row;
+            if (hrow < rows_valid) {
+              const __nv_bfloat16* hp = P.H + (row0 + hrow) * ld + col0;
+#pragma unroll
+              for (int j = eg; j < BN / 64; j += 2)
+                if (col0 + j * 64 < P.d_in) asm volatile("prefetch.global.L2 [%0];" ::"l"(hp + j * 64));
+            }
+          }
+        }
+      }
       bool got = mbar_wait(&s.tmem_full[buf], use, abort_flag, P.status);
       if constexpr (!LEAN) {
-        // the 128 epilogue threads meet at barriers further down: they give up together or not at all
+        // the epilogue threads give up together or not at all
         uint32_t all;
         asm volatile(
             "{\n\t.reg .pred p, q;\n\t"
             "setp.ne.u32 p, %1, 0;\n\t"
-            "bar.red.and.pred q, 1, 128, p;\n\t"
+            "bar.red.and.pred q, 1, 256, p;\n\t"
             "selp.u32 %0, 1, 0, q;\n\t}"
             : "=r"(all) : "r"(got ? 1u : 0u) : "memory");
         got = all != 0;
       }
       if (!got) { ok = false; break; }
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * BN);
+      const uint32_t taddr = tmem_base + ((uint32_t)(eq * 32) << 16) + (uint32_t)(buf * BN);
       if constexpr (LEAN) {
         // ---- whole contraction in this unit: accumulator -> (rescale, GELU', convert) -> swizzled
         // shared memory -> TMA store of 32 rows x 128 bytes per warp (rows / columns outside the
@@ -651,56 +736,40 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
         for (int hh = 0; hh < MH; ++hh) rowsq[hh] = 0.f;
         // GELU' epilogue: this thread's 64 pre-activations of a chunk (eight 16-byte loads, its own row) are
-        // requested one chunk ahead, so that their latency hides behind the chunk before (a load per use was
-        // measured to double the time of the whole product)
-        uint4 hq[8], hn[8];
-        auto load_h = [&](int hj2, uint4 (&dst)[8]) {
-          const int hh2 = hj2 / (BN / COLS), j2 = hj2 % (BN / COLS);
-          const int hrow2 = hh2 * BM + row;
-          const bool okh = hj2 < MH * (BN / COLS) && hrow2 < rows_valid && col0 + j2 * COLS < P.d_in;
-          if (okh) {
-            const uint4* src = reinterpret_cast<const uint4*>(P.H + (row0 + hrow2) * ld + col0 + j2 * COLS);
-#pragma unroll
-            for (int k8 = 0; k8 < 8; ++k8) dst[k8] = __ldg(src + k8);
-          }
-        };
-        if (MODE == MODE_DX && P.H != nullptr) load_h(0, hq);
+        // requested at the top of the chunk, in front of the TMEM load; they were prefetched to L2 before the
+        // wait for the accumulator, and the other warp of this quarter covers what latency is left.  (Staging
+        // them through shared memory with coalesced copies was measured slower.)
+        uint4 hq[8];
 #pragma unroll 1
-        for (int hj = 0; hj < MH * (BN / COLS); ++hj, ++nbuf) {
+        for (int hj = eg; hj < MH * (BN / COLS); hj += 2, ++nbuf) {      // this group's chunks
           const int hh = hj / (BN / COLS), j = hj % (BN / COLS);    // 128-row half of the tile, column chunk
-          const int hrow = hh * BM + row;
-          const bool valid = hrow < rows_valid;
           const uint32_t taddr_h = taddr + (uint32_t)(hh * BN);
-          if (MODE == MODE_DX && P.H != nullptr) {
-            if (hj > 0) {
-#pragma unroll
-              for (int k8 = 0; k8 < 8; ++k8) hq[k8] = hn[k8];
-            }
-            load_h(hj + 1, hn);
-          }
           if (col0 + j * COLS >= P.d_in) { --nbuf; continue; }      // warp-uniform
-          uint8_t* buf8 = stage0 + (nbuf & 1) * EPI_WARP_BYTES;
-          if (nbuf >= 2) { if (lane == 0) bulk_wait_read_1(); __syncwarp(); }
+          uint8_t* buf8 = stage0;
           uint4* myrow = reinterpret_cast<uint4*>(buf8 + lane * 128);
+          // the store of this warp's chunk before must have read the buffer before it is refilled (the wait sits
+          // behind the TMEM load, where it costs little; the other warp of this quarter works meanwhile)
+          auto buffer_free = [&]() { if (nbuf >= 1) { if (lane == 0) bulk_wait_read_0(); __syncwarp(); } };
+          const bool with_h = MODE == MODE_DX && P.H != nullptr;
+          if (with_h) {
+            // rows beyond the tile's valid rows read a valid row instead: their outputs are clipped by the store
+            const int hrow = min(hh * BM + row, rows_valid - 1);
+            const uint4* src = reinterpret_cast<const uint4*>(P.H + (row0 + hrow) * ld + col0 + j * 64);
+#pragma unroll
+            for (int k8 = 0; k8 < 8; ++k8) hq[k8] = __ldg(src + k8);
+          }
           if (MODE == MODE_DX) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
               uint32_t v[32];
               tmem_ld32(taddr_h + (uint32_t)(j * 64 + half * 32), v);
+              if (half == 0) buffer_free();
 #pragma unroll
               for (int g8 = 0; g8 < 4; ++g8) {
                 float r[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) r[e] = sc * __uint_as_float(v[g8 * 8 + e]);
-                if (P.H != nullptr && valid) {
-                  const uint4 hv = hq[half * 4 + g8];
-                  const uint32_t hu[4] = {hv.x, hv.y, hv.z, hv.w};
-#pragma unroll
-                  for (int e = 0; e < 4; ++e) {
-                    r[2 * e] *= gelu_prime(__uint_as_float(hu[e] << 16));
-                    r[2 * e + 1] *= gelu_prime(__uint_as_float(hu[e] & 0xffff0000u));
-                  }
-                }
+                if (with_h) gelu_prime8(hq[half * 4 + g8], r);
                 uint4 o;
                 o.x = pack_bf16(r[0], r[1]); o.y = pack_bf16(r[2], r[3]);
                 o.z = pack_bf16(r[4], r[5]); o.w = pack_bf16(r[6], r[7]);
@@ -723,6 +792,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           } else {
             uint32_t v[32];
             tmem_ld32(taddr_h + (uint32_t)(j * 32), v);
+            buffer_free();
 #pragma unroll
             for (int g4 = 0; g4 < 8; ++g4)
               myrow[(uint32_t)g4 ^ swz] = make_uint4(v[g4 * 4], v[g4 * 4 + 1], v[g4 * 4 + 2], v[g4 * 4 + 3]);
@@ -730,8 +800,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           fence_async_smem();
           __syncwarp();
           if (lane == 0) {
-            if (MODE == MODE_DX) tma_store_3d(&tmC, buf8, col0 + j * 64, t_out + hh * BM + warp * 32, n_out);
-            else tma_store_2d(&tmC, buf8, col0 + j * 32, (int)row0 + hh * BM + warp * 32);
+            if (MODE == MODE_DX) tma_store_3d(&tmC, buf8, col0 + j * 64, t_out + hh * BM + eq * 32, n_out);
+            else tma_store_2d(&tmC, buf8, col0 + j * 32, (int)row0 + hh * BM + eq * 32);
             bulk_commit();
           }
         }
@@ -740,7 +810,8 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (MODE == MODE_DX && P.a_out != nullptr) {
 #pragma unroll
           for (int hh = 0; hh < MH; ++hh)
-            if (hh * BM + row < rows_valid) P.a_out[(row0 + hh * BM + row) * P.a_parts + col0 / 256] = rowsq[hh];
+            if (hh * BM + row < rows_valid)
+              P.a_out[(row0 + hh * BM + row) * P.a_parts + (col0 / 256) * 2 + eg] = rowsq[hh];
         }
         if (lane == 0) bulk_wait_all();        // staging buffers are reused by the next unit
         __syncwarp();
@@ -752,12 +823,12 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // staged in shared memory, so each warp moves its 32 rows of a chunk with one 4 KB bulk copy.
       float* part = P.partial + (size_t)u * (BM * BN);
 #pragma unroll 1
-      for (int j = 0; j < BN / 32; ++j) {
+      for (int j = eg; j < BN / 32; j += 2) {                       // this group's chunks
         if (col0 + j * 32 >= P.d_in) break;                         // warp-uniform
-        uint8_t* buf8 = stage0 + (j & 1) * EPI_WARP_BYTES;
-        if (j >= 2) { if (lane == 0) bulk_wait_read_1(); __syncwarp(); }
+        uint8_t* buf8 = stage0;
         uint32_t v[32];
         tmem_ld32(taddr + (uint32_t)(j * 32), v);
+        if (j >= 2) { if (lane == 0) bulk_wait_read_0(); __syncwarp(); }
         uint4* myrow = reinterpret_cast<uint4*>(buf8 + lane * 128);
 #pragma unroll
         for (int g4 = 0; g4 < 8; ++g4)
@@ -765,7 +836,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-          bulk_store(part + (size_t)j * (BM * 32) + (size_t)(warp * 32) * 32, buf8, EPI_WARP_BYTES);
+          bulk_store(part + (size_t)j * (BM * 32) + (size_t)(eq * 32) * 32, buf8, EPI_WARP_BYTES);
           bulk_commit();
         }
       }
@@ -780,7 +851,7 @@ umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       for (int z = (int)gridDim.x - 1 - (int)blockIdx.x; z < D.zero_tiles && ok; z += gridDim.x) zero_tile(z);
     }
   }
-  if (warp < 4 && lane == 0) bulk_wait_all();     // the bulk stores of zero tiles are only waited for here
+  if (warp != 4 && warp != 5 && lane == 0) bulk_wait_all();     // the bulk stores of zero tiles are only waited for here
   __syncwarp();
   tc_fence_before();
   __syncthreads();
