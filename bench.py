@@ -411,7 +411,10 @@ def measure_bert_base_with_probe(vb, inputs, torch, dev, pk):
 
 def measure_vit_block(vb, inputs, torch, dev, pk):
     """ViT-base MLP block (N=64, T=197, 768 -> 3072 -> 768): backward through fc2 with the GELU Jacobian fused
-    into its dX epilogue, then fc1 on the library's own output (data dropped by fc2 arrive as zero rows)."""
+    into its dX epilogue, then fc1 on the library's own output through the chain entry point: fc1 takes fc2's
+    kept-data list and the row norms its epilogue produced, so dZ1 is not read again for scoring.  The dense block
+    is the exact backward of both linears with the same GELU Jacobian in fc2's epilogue."""
+    from paper_2402_17227_b200.stack import LinearStack, StackLayer
     fc2, fc1 = inputs.CASES["vit_base_mlp_fc2"], inputs.CASES["vit_base_mlp_fc1"]
     N, T, hidden, d = fc2.N, fc2.T, fc2.d_in, fc2.d_out
     R = N * T
@@ -419,47 +422,41 @@ def measure_vit_block(vb, inputs, torch, dev, pk):
     A = torch.nn.functional.gelu(H.float()).to(torch.bfloat16)
     _, dZ2, W2 = [t.to(dev) for t in inputs.make_layer(fc2)]
     X1, _, W1 = [t.to(dev) for t in inputs.make_layer(fc1)]
-    l2, l1 = vb.Layer(N, T, hidden, d, torch.bfloat16), vb.Layer(N, T, d, hidden, torch.bfloat16)
-    dZ1 = torch.empty(R, hidden, dtype=torch.bfloat16, device=dev)
-    dW2 = torch.empty(d, hidden, dtype=torch.float32, device=dev)
-    dX1 = torch.empty(R, d, dtype=torch.bfloat16, device=dev)
-    dW1 = torch.empty(hidden, d, dtype=torch.float32, device=dev)
+    layers = [StackLayer("fc2", hidden, d, W2, [A], [dZ2], H=[H]),
+              StackLayer("fc1", d, hidden, W1, [X1], [None], chained=True)]
+    stack = LinearStack(layers, N, T, skip_dropped_rows=False, overlap_layers=True)
+    rho, nu = [fc2.rho, fc2.rho], [fc2.nu, fc2.nu]
     seeds = list(range(20))
-
-    def sampled(sd):
-        l2.linear_bwd(A, dZ2, W2, fc2.rho, fc2.nu, sd, H=H, dX=dZ1, dW=dW2)
-        l1.linear_bwd_plain(X1, dZ1, W1, fc2.rho, fc2.nu, sd + 1000, dX1, dW1)
-
-    def dense():
-        l2.dense_bwd(A, dZ2, W2, dX=dZ1, dW=dW2)
-        l1.dense_bwd(X1, dZ1, W1, dX=dX1, dW=dW1)
     for sd in seeds[:3]:
-        sampled(sd); dense()
+        stack.backward(rho, nu, seed=sd)
+        stack.dense_backward()
     torch.cuda.synchronize()
     e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
     e[0].record()
     for sd in seeds:
-        sampled(sd)
+        stack.backward(rho, nu, seed=sd)
     e[1].record()
     for _ in seeds:
-        dense()
+        stack.dense_backward()
     e[2].record()
     torch.cuda.synchronize()
     kept = []
     for sd in seeds:
-        sampled(sd)
-        s2, s1 = l2.last_sampling(), l1.last_sampling()
+        stack.backward(rho, nu, seed=sd)
+        s2, s1 = layers[0].handle.last_sampling(), layers[1].handle.last_sampling()
         kept.append((s2.cntA * T, s2.cntW, s1.cntA * T, s1.cntW))
     kA2, kW2, kA1, kW1 = [sum(k[i] for k in kept) / len(kept) for i in range(4)]
     t_s, t_d = e[0].elapsed_time(e[1]) / len(seeds), e[1].elapsed_time(e[2]) / len(seeds)
     ratio = 4.0 * R / max(1.0, kA2 + kW2 + kA1 + kW1)
-    assert l1.device_status() == 0 and l2.device_status() == 0
-    l1.close(); l2.close()
+    assert stack.device_status() == 0
+    stack.close()
     return {"N": N, "T": T, "d": d, "hidden": hidden, "rho": fc2.rho, "nu": fc2.nu, "seeds": len(seeds),
             "sampled_block_ms": t_s, "dense_block_ms": t_d, "speedup_vs_dense": t_d / t_s,
             "kept_rows": {"fc2_A": kA2, "fc2_W": kW2, "fc1_A": kA1, "fc1_W": kW1},
             "flops_reduction_ratio": ratio, "speedup_over_flops_ratio": t_d / t_s / ratio,
-            "note": "dense block: exact products of both linears, without the GELU Jacobian"}
+            "dense_tflops": 8.0 * R * d * hidden / t_d / 1e9,
+            "note": "fc1 is chained to fc2 (kept-data list and row norms handed down); dense block: exact products "
+                    "of both linears with the GELU Jacobian in fc2's epilogue"}
 
 
 def measure_bert_large_stack(vb, inputs, torch, dev, steps=200, F=50, M=2):
@@ -854,6 +851,12 @@ def main():
         # a BERT-large FFN linear at the keep ratios of a top, a middle and a bottom layer
         extra["bert_large_ffn_up"] = measure_layer(inputs.CASES["bert_large_ffn_up"], vb, inputs, torch, dev, pk,
                                                    [(0.8, 0.3), (0.5, 0.3), (0.2, 0.3)], list(range(20)))
+        torch.cuda.empty_cache()
+        # twice the rows of any other workload (N = 16, T = 2048: 32768 rows, more SampleW scores than fit one
+        # CTA's registers or a quarter of its shared memory)
+        long_case = inputs.LayerCase("long_seq_ffn_up", 16, 2048, 1024, 4096, torch.bfloat16, 1.0, 0.5, 0.5, 0.3)
+        extra["long_seq_ffn_up"] = measure_layer(long_case, vb, inputs, torch, dev, pk, [(0.5, 0.3), (0.3, 0.3)],
+                                                 list(range(10)))
 
     if rank != 0:
         if world > 1:

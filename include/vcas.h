@@ -184,6 +184,11 @@ int vcas_chain_parts(vcas_handle h, int32_t* parts);
 /* Exact backprop dX = dY W, dW = dY^T X with the same kernels at ratio 1 and no scoring. */
 int vcas_dense_bwd(vcas_handle h, const void* X, const void* dY, const void* W,
                    void* dX, float* dW, vcas_stream stream);
+/* vcas_dense_bwd for a layer whose input comes out of a GELU: with H [R, d_in] (layer dtype, the saved
+ * pre-activation, may be NULL) dX is multiplied elementwise by GELU'(H) in the product's epilogue, as
+ * vcas_linear_bwd_ex does - the exact backward through the activation, for comparisons with the sampled one. */
+int vcas_dense_bwd_ex(vcas_handle h, const void* X, const void* dY, const void* W, const void* H,
+                      void* dX, float* dW, vcas_stream stream);
 
 /*
  * Scores, keep probabilities, masks and compacted index lists only (Sec. 4.1, 4.2), exactly

@@ -22,7 +22,7 @@ DTYPE_F32, DTYPE_BF16 = 0, 1
 GEMM_AUTO, GEMM_FMA, GEMM_TENSOR = 0, 1, 2
 
 EXPORTS = ["vcas_default_config", "vcas_create", "vcas_destroy", "vcas_workspace_bytes", "vcas_linear_bwd",
-           "vcas_linear_bwd_ex", "vcas_linear_bwd_chain", "vcas_chain_parts", "vcas_layernorm_bwd", "vcas_join", "vcas_dense_bwd", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
+           "vcas_linear_bwd_ex", "vcas_linear_bwd_chain", "vcas_chain_parts", "vcas_layernorm_bwd", "vcas_join", "vcas_dense_bwd", "vcas_dense_bwd_ex", "vcas_score", "vcas_last_sampling", "vcas_mask_from_probs",
            "vcas_variance_probe", "vcas_update_ratios", "vcas_last_device_status", "vcas_launch_count",
            "vcas_set_profiling", "vcas_stage_times", "vcas_set_wait_limit",
            "vcas_set_probe_subsample", "vcas_get_probe_subsample", "vcas_score_static", "vcas_set_tuning",
@@ -192,10 +192,10 @@ class Layer:
         _check(lib().vcas_linear_bwd(self._h, _ptr(X), _ptr(dY), _ptr(W), C.c_float(rho), C.c_float(nu),
                                      C.c_uint64(seed), _ptr(dX), _ptr(dW), _stream()), "vcas_linear_bwd")
 
-    def dense_bwd(self, X, dY, W, *, dX=None, dW=None):
+    def dense_bwd(self, X, dY, W, *, H=None, dX=None, dW=None):
         dX, dW = self._outs(dX, dW, X.device)
-        _check(lib().vcas_dense_bwd(self._h, _ptr(X), _ptr(dY), _ptr(W), _ptr(dX), _ptr(dW), _stream()),
-               "vcas_dense_bwd")
+        _check(lib().vcas_dense_bwd_ex(self._h, _ptr(X), _ptr(dY), _ptr(W), _ptr(H), _ptr(dX), _ptr(dW), _stream()),
+               "vcas_dense_bwd_ex")
         return dX, dW
 
     # ------------------------------------------------------------------ sampling

@@ -410,6 +410,11 @@ int vcas_linear_bwd(vcas_handle hh, const void* X, const void* dY, const void* W
 
 int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W, void* dX, float* dW,
                    vcas_stream stream) {
+  return vcas_dense_bwd_ex(hh, X, dY, W, nullptr, dX, dW, stream);
+}
+
+int vcas_dense_bwd_ex(vcas_handle hh, const void* X, const void* dY, const void* W, const void* Hpre, void* dX,
+                      float* dW, vcas_stream stream) {
   if (hh == nullptr || X == nullptr || dY == nullptr || W == nullptr || dX == nullptr || dW == nullptr)
     return VCAS_ERR_BAD_ARG;
   Handle* h = H(hh);
@@ -426,9 +431,9 @@ int vcas_dense_bwd(vcas_handle hh, const void* X, const void* dY, const void* W,
   if (h->tensor_path) plan_products(h, true, 1.0f, h->desc.N * h->desc.T, 0, false, &px, &pw);
   mark_dense(h, 0, st);
   if (h->tensor_path) {
-    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, nullptr, dX, nullptr, false, 0, &px, st));
+    VCAS_CUDA(launch_umma_dx(h, dY, W, true, 1.0f, Hpre, dX, nullptr, false, 0, &px, st));
   } else {
-    VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, nullptr, dX, st));
+    VCAS_CUDA(launch_fma_dx(h, dY, W, nullptr, Hpre, dX, st));
   }
   mark_dense(h, 1, st);
   mark_dense(h, 3, sw);

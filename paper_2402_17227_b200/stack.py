@@ -104,14 +104,16 @@ class LinearStack:
                 h.join()
 
     def dense_backward(self, variant: int = 0, hook=None) -> None:
-        """The exact backward of the same layers (no sampling, no Jacobian factor): the dense comparison."""
+        """The exact backward of the same layers (no sampling; the GELU Jacobian where the sampled pass has it):
+        the dense comparison."""
         prev = None
         for i, L in enumerate(self.layers):
             v = variant % len(L.X)
             dY = prev.dX if L.chained else L.dY[v]
             if hook is not None:
                 hook(i, L, False)
-            L.handle.dense_bwd(L.X[v], dY, L.W, dX=L.dX, dW=L.dW)
+            H = L.H[v % len(L.H)] if L.H is not None else None
+            L.handle.dense_bwd(L.X[v], dY, L.W, H=H, dX=L.dX, dW=L.dW)
             if hook is not None:
                 hook(i, L, True)
             prev = L

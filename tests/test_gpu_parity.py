@@ -304,6 +304,11 @@ def test_gelu_jacobian_epilogue(name, dtype, path):
                               q_in=torch.from_numpy(ref["q32"]).cuda(), H=Hc)
     assert rel_fro(np64(dX), ref["dX"] * o.gelu_prime(np64(H))) <= tol_for(dtype)
     assert rel_fro(np64(dW), ref["dW"]) <= tol_for(dtype)
+    # the exact backward with the same Jacobian factor (vcas_dense_bwd_ex)
+    dXd, dWd = o.dense_bwd(np64(X), np64(dY), np64(W))
+    dX2, dW2 = layer.dense_bwd(Xc, dYc, Wc, H=Hc)
+    assert rel_fro(np64(dX2), dXd * o.gelu_prime(np64(H))) <= tol_for(dtype)
+    assert rel_fro(np64(dW2), dWd) <= tol_for(dtype)
     layer.close()
 
 
