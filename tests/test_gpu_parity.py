@@ -157,6 +157,15 @@ def test_tensor_path_split_contraction_and_tile_widths(tile_n, split, tile_m):
     dXd, dWd = o.dense_bwd(np64(X), np64(dY), np64(W))
     dX3, dW3 = layer.dense_bwd(Xc, dYc, Wc)
     assert rel_fro(np64(dX3), dXd) <= tol_for(BF16) and rel_fro(np64(dW3), dWd) <= tol_for(BF16)
+    # the GELU Jacobian under the same tiling (the slice reduction and the unsliced epilogue each apply it), with
+    # pre-activations on both sides of the polynomial's clamp at |x| = 5
+    H = (2.5 * torch.randn(N * T, d_in, generator=torch.Generator().manual_seed(8))).to(BF16)
+    gp = o.gelu_prime(np64(H))
+    dX5, dW5 = layer.linear_bwd(Xc, dYc, Wc, 0.5, 0.5, 4, p_in=p_in, q_in=q_in, H=H.cuda())
+    assert rel_fro(np64(dX5), ref["dX"] * gp) <= tol_for(BF16) and torch.equal(dW5, dW)
+    assert np.abs(np64(dX5) - ref["dX"] * gp).max() <= 2e-2 * np.abs(ref["dX"]).max()
+    dX6, _ = layer.dense_bwd(Xc, dYc, Wc, H=H.cuda())
+    assert rel_fro(np64(dX6), dXd * gp) <= tol_for(BF16)
     assert layer.device_status() == 0
     layer.close()
 
@@ -309,6 +318,27 @@ def test_gelu_jacobian_epilogue(name, dtype, path):
     dX2, dW2 = layer.dense_bwd(Xc, dYc, Wc, H=Hc)
     assert rel_fro(np64(dX2), dXd * o.gelu_prime(np64(H))) <= tol_for(dtype)
     assert rel_fro(np64(dW2), dWd) <= tol_for(dtype)
+    layer.close()
+
+
+def test_gelu_jacobian_values_on_the_tensor_path():
+    """The tensor path evaluates GELU' as a polynomial.  With dY = 1 and W = 1/d_out the product is exactly 1, so
+    the dense backward with H returns GELU'(H) rounded to bf16: every value, over -9 <= x <= 9 in steps of 2^-6,
+    must lie within the bf16 rounding (half a unit in the last of 8 significant bits: 2^-8 relative) plus 1e-4 of the erf form."""
+    N, T, d_in, d_out = 2, 128, 256, 64
+    xs = torch.arange(-9.0, 9.0, 2.0 ** -6)
+    H = xs.repeat((N * T * d_in + xs.numel() - 1) // xs.numel())[:N * T * d_in].reshape(N * T, d_in).to(BF16)
+    dY = torch.ones(N * T, d_out, dtype=BF16)
+    W = torch.full((d_out, d_in), 1.0 / d_out, dtype=BF16)
+    X = torch.zeros(N * T, d_in, dtype=BF16)
+    layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_TENSOR)
+    for tune in ((0, 0, 0, 0, 0), (256, 256, 1, 1, 2), (128, 128, 1, 1, 1)):
+        layer.set_tuning(*tune)
+        dX, _ = layer.dense_bwd(X.cuda(), dY.cuda(), W.cuda(), H=H.cuda())
+        ref = o.gelu_prime(np64(H))
+        err = np.abs(np64(dX) - ref)
+        assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 1e-4), float(err.max())
+    assert layer.device_status() == 0
     layer.close()
 
 
