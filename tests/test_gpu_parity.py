@@ -79,15 +79,16 @@ def test_score_matches_oracle(dtype, shape):
     layer.close()
 
 
-@pytest.mark.parametrize("N,T", [(40, 250), (64, 100), (33, 31), (20, 1000), (1100, 3)])
+@pytest.mark.parametrize("N,T", [(40, 250), (64, 100), (33, 31), (20, 1000), (1100, 3), (70, 1000)])
 def test_score_kernel_variants(N, T):
-    """Row counts that select each variant of the sampling kernel (4, 8, 16 rows per thread, more than
-    32 data, and the general kernel beyond 16384 rows or 1024 data)."""
+    """Sizes that select each variant of the sampling kernels: up to 32 data, up to 1024 data, more than 1024 data
+    (SampleA in one warp, in one warp with several data per lane, block-wide), and, with 70000 rows at rho = 0.95,
+    more SampleW scores than fit one CTA's shared memory (the water-filling then reads them from global memory)."""
     d_in = d_out = 64
-    X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.5, sigma_B=1.0, zero_fraction=0.1)
+    X, dY, W = small_case(BF16, N, T, d_in, d_out, sigma_A=1.5, sigma_B=1.0, zero_fraction=0.1 if N * T < 60000 else 0.0)
     layer = vb.Layer(N, T, d_in, d_out, BF16, vb.GEMM_FMA)
     Xc, dYc = cuda(X, dY)
-    for seed, rho, nu in [(1, 0.3, 0.4), (5, 0.6, 0.2)]:
+    for seed, rho, nu in [(1, 0.3, 0.4), (5, 0.6, 0.2)] + ([(2, 0.95, 0.3)] if N * T >= 60000 else []):
         s = layer.score(Xc, dYc, rho, nu, seed)
         ref = o.linear_bwd(np64(X), np64(dY), np64(W), N, T, f32(rho), f32(nu), seed)
         ref["seed"] = seed
