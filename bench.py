@@ -873,7 +873,7 @@ def main():
         sweep_seeds = list(range(20))
         grid = [(r, n) for r in SWEEP for n in SWEEP if args.sweep == "grid" or r == n]
         extra = {
-            # BASELINE configs[4]: the 5 x 5 grid of keep ratios on the headline layer, 20 seeds per point
+            # the 5 x 5 grid of keep ratios on the headline layer, 20 seeds per point
             "llm_mlp_up_ratio_sweep": measure_layer(case, vb, inputs, torch, dev, pk, grid, sweep_seeds,
                                                     tensors=(Xs[0], dYs[0], W), layer=layer),
         }
